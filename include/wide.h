@@ -1,0 +1,197 @@
+/*
+ * wide.h -- C ABI of the WIDE hot path for NVIDIA B200 (sm_100a).
+ *
+ * Token-wise dynamic-width execution of a transformer layer:
+ *   wide_route      router scores -> per-token group bitmask      (Section 3.1, Eq. 4)
+ *   wide_reorder    per-group mask reordering + tile predicates   (Section 3.3, Eq. 6-8, Algorithm 1)
+ *   wide_ffn        block-skipping SwiGLU FFN                     (Eq. 3; Algorithms 2 and 3)
+ *   wide_oproj      head-group-masked attention output projection (Eq. 2; Eq. 10, Algorithm 3)
+ *   wide_unpermute  the scatter epilogue as a standalone step     (Algorithm 2, epilogue)
+ *
+ * General rules
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library never
+ *     allocates, frees or keeps caller-visible memory.  Scratch memory is passed in as
+ *     `workspace` (size from wide_workspace_bytes).
+ *   - All work is enqueued on the caller's stream (`stream` is a cudaStream_t cast to
+ *     void*); no call synchronises the host or reads results back, except wide_status.
+ *   - Matrices are row-major and contiguous.  Base pointers must be 16-byte aligned.
+ *     Weights use the Linear layout C = A B^T with B in [N, K]:
+ *       w_gate, w_up [d_ff, hidden]   w_down [hidden, d_ff]   w_o [hidden, attn_dim]
+ *       w_router [n_groups, hidden]
+ *   - Masks are bit-packed: bit (g % 32) of word mask_bits[t * W + g / 32], W = ceil(n_groups/32),
+ *     is 1 iff token t executes group g; unused high bits are 0.
+ *   - Return value: WIDE_OK or a negative WIDE_ERR_* code.  Argument errors are found on the
+ *     host before anything is launched and leave all outputs untouched.
+ *   - Outputs are fully overwritten (no accumulate-into semantics).
+ *   - Device-side waits are bounded; if one expires the kernel records WIDE_ERR_TIMEOUT in
+ *     the context's device status word and returns (it never traps or spins forever).
+ */
+#ifndef WIDE_H_
+#define WIDE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define WIDE_VERSION 100
+
+#if defined(__GNUC__)
+#define WIDE_API __attribute__((visibility("default")))
+#else
+#define WIDE_API
+#endif
+
+/* error codes */
+#define WIDE_OK 0
+#define WIDE_ERR_INVALID_ARG (-1)
+#define WIDE_ERR_UNSUPPORTED_SHAPE (-2)
+#define WIDE_ERR_ALIGNMENT (-3)
+#define WIDE_ERR_WORKSPACE (-4)
+#define WIDE_ERR_CUDA (-5)
+#define WIDE_ERR_TIMEOUT (-6)
+
+/* element types of activations / weights / outputs */
+#define WIDE_BF16 0
+#define WIDE_F32 1
+
+/* router forms */
+#define WIDE_ROUTE_TOPK 0        /* one linear layer hidden -> n_groups, k largest per token   */
+#define WIDE_ROUTE_PAIR_ARGMAX 1 /* bottleneck W1 W2 -> 2 logits per group, Eq. 4 (inference)  */
+
+/* operations, for wide_workspace_bytes */
+#define WIDE_OP_ROUTE 0
+#define WIDE_OP_REORDER 1
+#define WIDE_OP_FFN 2
+#define WIDE_OP_OPROJ 3
+#define WIDE_OP_UNPERMUTE 4
+
+/* flags for wide_ffn / wide_oproj / wide_route */
+#define WIDE_FLAG_NONE 0u
+#define WIDE_FLAG_SIMT 1u        /* use the plain CUDA-core kernels (any shape; the only path for fp32) */
+#define WIDE_FLAG_FORCE_PREFILL 2u /* tokens <= WIDE_DECODE_MAX_TOKENS would normally take the decode path */
+#define WIDE_FLAG_FORCE_DECODE 4u  /* take the union-streaming decode path (tokens <= WIDE_DECODE_MAX_TOKENS) */
+
+#define WIDE_DECODE_MAX_TOKENS 64
+#define WIDE_MAX_GROUPS 256
+
+typedef struct wide_ctx wide_ctx;
+
+/* Create / destroy a context bound to CUDA device `device` (ordinal).  The context holds the
+ * device properties and a 4-byte device status word; nothing else.  Host-synchronous. */
+WIDE_API int wide_create(wide_ctx** ctx, int device);
+WIDE_API int wide_destroy(wide_ctx* ctx);
+
+/* Synchronise `stream`, read the device status word into *status (WIDE_OK or
+ * WIDE_ERR_TIMEOUT) and clear it.  The only call that blocks the host. */
+WIDE_API int wide_status(wide_ctx* ctx, void* stream, int* status);
+
+/* Override the bound of every device-side wait (nanoseconds; default 2e9). */
+WIDE_API int wide_set_wait_limit_ns(wide_ctx* ctx, uint64_t ns);
+
+WIDE_API const char* wide_strerror(int code);
+WIDE_API int wide_version(void);
+
+/* Bytes of scratch the given operation needs for these shapes (0 if none).
+ *   tokens T, hidden D, inner = d_ff (FFN) or attn_dim (O-proj), group G, n_groups N_G.
+ * The same size is valid for every flag combination of that operation. */
+WIDE_API size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, int inner, int group, int n_groups);
+
+/*
+ * wide_route -- Section 3.1 "Routing components" (Eq. 4) and the fixed-budget reading of
+ * Appendix A ("each token selects R groups").
+ *
+ *   mode WIDE_ROUTE_TOPK:        s[t,g] = sum_i x[t,i] * w_router[g,i];  token t executes the
+ *                                k_t groups with the largest score, equal scores -> lower g.
+ *                                k_t = k_per_token[t] if k_per_token != NULL else k.
+ *                                w2 must be NULL, rank 0.
+ *   mode WIDE_ROUTE_PAIR_ARGMAX: l = (x W1) W2 with w_router = W1 [hidden, rank] and
+ *                                w2 = W2 [rank, 2*n_groups]; token t executes group g iff
+ *                                l[t,2g] >= l[t,2g+1] (class 0 = execute, first index wins ties).
+ *
+ * The selection is decided on fp64 sums of the exact input products, so it does not depend on
+ * summation order.
+ *   x          [tokens, hidden]  dtype
+ *   mask_bits  out uint32 [tokens, W]
+ *   scores     out fp32 [tokens, n_groups] (TOPK) or [tokens, 2*n_groups] (PAIR), may be NULL
+ * Errors: INVALID_ARG (null pointer, k outside [0, n_groups], bad mode/dtype),
+ *         UNSUPPORTED_SHAPE (n_groups > WIDE_MAX_GROUPS, hidden % 8 != 0), ALIGNMENT, WORKSPACE.
+ */
+WIDE_API int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens, int hidden,
+               const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
+               const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* workspace,
+               size_t workspace_bytes, unsigned flags);
+
+/*
+ * wide_reorder -- mask reordering, Eq. 6 / Algorithm 1, and the level-0 predicate of Eq. 7-8.
+ * For each group g the rows are sorted by mask value, descending and STABLE (active rows in
+ * ascending token order, then inactive rows in ascending token order).
+ *
+ *   perm       out int32 [n_groups, tokens]   perm[g][j] = token at sorted position j
+ *   counts     out int32 [n_groups]           active tokens of group g
+ *   tile_map   out uint8 [n_tiles, n_groups]  1 iff sorted rows [m*tile_m, (m+1)*tile_m) of group g
+ *                                             contain an active row; n_tiles = ceil(tokens/tile_m)
+ *   work_list  out int32 [n_tiles*n_groups, 2] the active (tile, group) pairs, group-major with
+ *                                             tiles ascending; unused tail entries are (-1,-1)
+ *   n_work     out int32 [1]
+ *   union_list out int32 [n_groups]           groups with >= 1 active token, ascending; tail = -1
+ *   n_union    out int32 [1]
+ *   offsets    out int32 [n_groups + 1]       offsets[g] = sum_{g'<g} ceil(counts[g']/tile_m)*tile_m
+ *                                             (row offsets of the packed-sorted layout)
+ * tile_m must be a power of two >= 16.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE.
+ */
+WIDE_API int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
+                 int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map, int32_t* work_list,
+                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets);
+
+/*
+ * wide_ffn -- Eq. 3:  y = ((silu(x Wg^T) * (x Wu^T)) (.)_G M) Wd^T.
+ * Gate/up columns and down rows of inactive (token, group) pairs are skipped (block level) or
+ * contribute exact zeros (inside an active tile).
+ *
+ *   x [tokens, hidden], w_gate/w_up [d_ff, hidden], w_down [hidden, d_ff]: dtype
+ *   mask_bits [tokens, W], W = ceil((d_ff/group)/32)
+ *   perm, counts, work_list, n_work: outputs of wide_reorder for this mask with tile_m = 128.
+ *       Needed by the prefill tensor-core path; may all be NULL when tokens <=
+ *       WIDE_DECODE_MAX_TOKENS (decode path: union of active groups, no reordering) or with
+ *       WIDE_FLAG_SIMT.
+ *   y  out [tokens, hidden] of out_dtype
+ * Tensor-core paths need dtype bf16, hidden % 64 == 0, group in {64,128,256,512}; other shapes
+ * need WIDE_FLAG_SIMT (hidden % 4 == 0, group % 4 == 0).
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, ALIGNMENT, WORKSPACE, CUDA.
+ */
+WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
+             const void* w_down, int dtype, int tokens, int hidden, int d_ff, int group,
+             const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
+             const int32_t* work_list, const int32_t* n_work, void* y, int out_dtype,
+             void* workspace, size_t workspace_bytes, unsigned flags);
+
+/*
+ * wide_oproj -- Eq. 2 / Eq. 10:  y[t,:] = sum_{g : M[t,g]=1} a[t, gG:(g+1)G] Wo[:, gG:(g+1)G]^T,
+ * a = attention output flattened head-major [tokens, attn_dim], group g = channels [gG, (g+1)G).
+ *   perm, counts, work_list, n_work as for wide_ffn (same NULL rules).
+ */
+WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
+               int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,
+               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
+               const int32_t* n_work, void* y, int out_dtype, void* workspace,
+               size_t workspace_bytes, unsigned flags);
+
+/*
+ * wide_unpermute -- scatter epilogue of Algorithm 2 as its own call: packed-sorted rows back to
+ * the dense token-major layout.
+ *   dst[perm[g][j], g*G:(g+1)*G] = src_packed[offsets[g] + j, 0:G]   for j < counts[g]
+ *   every other element of dst = 0
+ *   src_packed [offsets[n_groups], group], dst [tokens, n_groups*group]; elem_bytes in {2, 4};
+ *   group*elem_bytes must be a multiple of 16.
+ */
+WIDE_API int wide_unpermute(wide_ctx* ctx, void* stream, const void* src_packed, const int32_t* perm,
+                   const int32_t* counts, const int32_t* offsets, int tokens, int n_groups,
+                   int group, int elem_bytes, void* dst);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WIDE_H_ */

@@ -1,0 +1,227 @@
+// C ABI of libwide: argument validation, workspace sizing and dispatch.  See include/wide.h.
+#include <new>
+
+#include "internal.h"
+
+namespace {
+
+bool valid_dtype(int d) { return d == WIDE_BF16 || d == WIDE_F32; }
+bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// Which implementation serves this FFN / O-proj call.
+enum Path { PATH_SIMT, PATH_PREFILL_TC, PATH_DECODE_TC, PATH_NONE };
+
+Path choose_path(int dtype, int tokens, int hidden, int inner, int group, unsigned flags) {
+    if (flags & WIDE_FLAG_SIMT) return PATH_SIMT;
+    const bool tc_ok = dtype == WIDE_BF16 && hidden % 64 == 0 && inner % 64 == 0 &&
+                       (group == 64 || group == 128 || group == 256 || group == 512);
+    if (!tc_ok) return PATH_NONE;
+    if (flags & WIDE_FLAG_FORCE_DECODE) return tokens <= WIDE_DECODE_MAX_TOKENS ? PATH_DECODE_TC : PATH_NONE;
+    if (flags & WIDE_FLAG_FORCE_PREFILL) return PATH_PREFILL_TC;
+    return tokens <= WIDE_DECODE_MAX_TOKENS ? PATH_DECODE_TC : PATH_PREFILL_TC;
+}
+
+size_t inner_scratch(int dtype, int tokens, int hidden, int inner) {
+    // hidden activation / masked attention output [tokens, inner] in dtype, or the decode scratch
+    size_t a = wide_align_up(static_cast<size_t>(tokens) * inner * wide_elem_bytes(dtype), 256);
+    size_t b = tokens <= WIDE_DECODE_MAX_TOKENS ? wide_decode_workspace(tokens, hidden, inner) : 0;
+    return a > b ? a : b;
+}
+
+}  // namespace
+
+extern "C" {
+
+int wide_version(void) { return WIDE_VERSION; }
+
+const char* wide_strerror(int code) {
+    switch (code) {
+        case WIDE_OK: return "ok";
+        case WIDE_ERR_INVALID_ARG: return "invalid argument";
+        case WIDE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape for the requested path";
+        case WIDE_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case WIDE_ERR_WORKSPACE: return "workspace missing or too small";
+        case WIDE_ERR_CUDA: return "CUDA runtime or driver error";
+        case WIDE_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown error code";
+    }
+}
+
+int wide_create(wide_ctx** out, int device) {
+    if (!out) return WIDE_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return WIDE_ERR_CUDA;
+    WIDE_CUDA_CHECK(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    WIDE_CUDA_CHECK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return WIDE_ERR_CUDA;  // built for sm_100a only
+    wide_ctx* ctx = new (std::nothrow) wide_ctx();
+    if (!ctx) return WIDE_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->wait_ns = 2000000000ull;
+    ctx->encode_tiled = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+        ctx->encode_tiled = fn;
+    if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) {
+        delete ctx;
+        return WIDE_ERR_CUDA;
+    }
+    if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
+        cudaFree(ctx->d_status);
+        delete ctx;
+        return WIDE_ERR_CUDA;
+    }
+    *out = ctx;
+    return WIDE_OK;
+}
+
+int wide_destroy(wide_ctx* ctx) {
+    if (!ctx) return WIDE_ERR_INVALID_ARG;
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return WIDE_OK;
+}
+
+int wide_status(wide_ctx* ctx, void* stream, int* status) {
+    if (!ctx || !status) return WIDE_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    WIDE_CUDA_CHECK(cudaMemcpyAsync(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
+    WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s));
+    WIDE_CUDA_CHECK(cudaStreamSynchronize(s));
+    *status = v;
+    return WIDE_OK;
+}
+
+int wide_set_wait_limit_ns(wide_ctx* ctx, uint64_t ns) {
+    if (!ctx || ns == 0) return WIDE_ERR_INVALID_ARG;
+    ctx->wait_ns = ns;
+    return WIDE_OK;
+}
+
+size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, int inner, int group, int n_groups) {
+    (void)group;
+    if (tokens < 0 || hidden < 0 || inner < 0 || n_groups < 0 || !valid_dtype(dtype)) return 0;
+    switch (op) {
+        case WIDE_OP_ROUTE: return wide_route_workspace(tokens, n_groups, 64);
+        case WIDE_OP_FFN:
+        case WIDE_OP_OPROJ: return inner_scratch(dtype, tokens, hidden, inner);
+        default: return 0;
+    }
+}
+
+int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens, int hidden,
+               const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
+               const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* workspace,
+               size_t workspace_bytes, unsigned flags) {
+    (void)flags;
+    if (!ctx || !x || !w_router || !mask_bits || !valid_dtype(dtype)) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || n_groups <= 0) return WIDE_ERR_INVALID_ARG;
+    if (mode == WIDE_ROUTE_TOPK) {
+        if (w2 || rank != 0) return WIDE_ERR_INVALID_ARG;
+        if (!k_per_token && (k < 0 || k > n_groups)) return WIDE_ERR_INVALID_ARG;
+    } else if (mode == WIDE_ROUTE_PAIR_ARGMAX) {
+        if (!w2 || rank <= 0 || rank > 64) return WIDE_ERR_INVALID_ARG;
+    } else {
+        return WIDE_ERR_INVALID_ARG;
+    }
+    if (n_groups > WIDE_MAX_GROUPS || hidden % 8 != 0) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(x) || !wide_aligned16(w_router) || (w2 && !wide_aligned16(w2)) || !wide_aligned16(workspace))
+        return WIDE_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < wide_route_workspace(tokens, n_groups, rank)) return WIDE_ERR_WORKSPACE;
+    return wide_launch_route(ctx, static_cast<cudaStream_t>(stream), x, dtype, tokens, hidden, w_router, w2, rank,
+                             n_groups, mode, k, k_per_token, mask_bits, scores, workspace);
+}
+
+int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
+                 int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map, int32_t* work_list,
+                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets) {
+    if (!ctx || !mask_bits || !perm || !counts || !tile_map || !work_list || !n_work || !union_list || !n_union ||
+        !offsets)
+        return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || n_groups <= 0 || !is_pow2(tile_m) || tile_m < 16) return WIDE_ERR_INVALID_ARG;
+    if (n_groups > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    return wide_launch_reorder(ctx, static_cast<cudaStream_t>(stream), mask_bits, tokens, n_groups, tile_m, perm,
+                               counts, tile_map, work_list, n_work, union_list, n_union, offsets);
+}
+
+int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
+             const void* w_down, int dtype, int tokens, int hidden, int d_ff, int group,
+             const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
+             const int32_t* work_list, const int32_t* n_work, void* y, int out_dtype,
+             void* workspace, size_t workspace_bytes, unsigned flags) {
+    if (!ctx || !x || !w_gate || !w_up || !w_down || !mask_bits || !y) return WIDE_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || !valid_dtype(out_dtype)) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || d_ff <= 0 || group <= 0 || d_ff % group != 0) return WIDE_ERR_INVALID_ARG;
+    if (d_ff / group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    const Path path = choose_path(dtype, tokens, hidden, d_ff, group, flags);
+    if (path == PATH_NONE) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (path == PATH_SIMT && (hidden % 4 != 0 || group % 4 != 0)) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (path == PATH_PREFILL_TC && (!perm || !counts || !work_list || !n_work)) return WIDE_ERR_INVALID_ARG;
+    if (!wide_aligned16(x) || !wide_aligned16(w_gate) || !wide_aligned16(w_up) || !wide_aligned16(w_down) ||
+        !wide_aligned16(y) || !wide_aligned16(workspace))
+        return WIDE_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, d_ff)) return WIDE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (path) {
+        case PATH_SIMT:
+            return wide_launch_ffn_simt(s, x, w_gate, w_up, w_down, dtype, tokens, hidden, d_ff, group, mask_bits, y,
+                                        out_dtype, workspace);
+        case PATH_PREFILL_TC:
+            return wide_launch_ffn_prefill_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
+                                              perm, counts, work_list, n_work, y, out_dtype, workspace);
+        default:
+            return wide_launch_ffn_decode_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
+                                             y, out_dtype, workspace);
+    }
+}
+
+int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
+               int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,
+               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
+               const int32_t* n_work, void* y, int out_dtype, void* workspace,
+               size_t workspace_bytes, unsigned flags) {
+    (void)perm; (void)counts; (void)work_list; (void)n_work;
+    if (!ctx || !attn_out || !w_o || !mask_bits || !y) return WIDE_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || !valid_dtype(out_dtype)) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || attn_dim <= 0 || group <= 0 || attn_dim % group != 0) return WIDE_ERR_INVALID_ARG;
+    if (attn_dim / group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    const Path path = choose_path(dtype, tokens, hidden, attn_dim, group, flags);
+    if (path == PATH_NONE) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (path == PATH_SIMT && (hidden % 4 != 0 || group % 4 != 0)) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(attn_out) || !wide_aligned16(w_o) || !wide_aligned16(y) || !wide_aligned16(workspace))
+        return WIDE_ERR_ALIGNMENT;
+    if (path != PATH_SIMT &&
+        (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, attn_dim)))
+        return WIDE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (path) {
+        case PATH_SIMT:
+            return wide_launch_oproj_simt(s, attn_out, w_o, dtype, tokens, hidden, attn_dim, group, mask_bits, y,
+                                          out_dtype);
+        case PATH_PREFILL_TC:
+            return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
+                                                out_dtype, workspace);
+        default:
+            return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
+                                               out_dtype, workspace);
+    }
+}
+
+int wide_unpermute(wide_ctx* ctx, void* stream, const void* src_packed, const int32_t* perm,
+                   const int32_t* counts, const int32_t* offsets, int tokens, int n_groups,
+                   int group, int elem_bytes, void* dst) {
+    if (!ctx || !src_packed || !perm || !counts || !offsets || !dst) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || n_groups <= 0 || group <= 0 || (elem_bytes != 2 && elem_bytes != 4)) return WIDE_ERR_INVALID_ARG;
+    if ((group * elem_bytes) % 16 != 0) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(src_packed) || !wide_aligned16(dst)) return WIDE_ERR_ALIGNMENT;
+    return wide_launch_unpermute(static_cast<cudaStream_t>(stream), src_packed, perm, counts, offsets, tokens,
+                                 n_groups, group, elem_bytes, dst);
+}
+
+}  // extern "C"

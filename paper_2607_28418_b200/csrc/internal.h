@@ -1,0 +1,82 @@
+// Internal declarations shared by the .cu files of libwide (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "wide.h"
+
+struct wide_ctx {
+    int device;
+    int sm_count;
+    int* d_status;          // device status word (WIDE_OK or WIDE_ERR_TIMEOUT)
+    unsigned long long wait_ns;  // bound of every device-side wait
+    void* encode_tiled;     // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+#define WIDE_CUDA_CHECK(expr)                         \
+    do {                                              \
+        cudaError_t err__ = (expr);                   \
+        if (err__ != cudaSuccess) return WIDE_ERR_CUDA; \
+    } while (0)
+
+static inline bool wide_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t wide_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int wide_elem_bytes(int dtype) { return dtype == WIDE_BF16 ? 2 : 4; }
+
+// ---- element conversion used by the CUDA-core kernels
+__device__ __forceinline__ float wide_to_float(float v) { return v; }
+__device__ __forceinline__ float wide_to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float wide_to_float(double v) { return static_cast<float>(v); }
+__device__ __forceinline__ double wide_to_double(float v) { return static_cast<double>(v); }
+__device__ __forceinline__ double wide_to_double(__nv_bfloat16 v) { return static_cast<double>(__bfloat162float(v)); }
+__device__ __forceinline__ double wide_to_double(double v) { return v; }
+__device__ __forceinline__ void wide_store(float* p, float v) { *p = v; }
+__device__ __forceinline__ void wide_store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ bool wide_mask_bit(const uint32_t* mask_bits, int words, int t, int g) {
+    return (mask_bits[static_cast<size_t>(t) * words + (g >> 5)] >> (g & 31)) & 1u;
+}
+
+// ---- launchers (each returns WIDE_OK or WIDE_ERR_CUDA; arguments already validated)
+int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
+                      const void* w_router, const void* w2, int rank, int NG, int mode, int k,
+                      const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws);
+size_t wide_route_workspace(int T, int NG, int rank);
+
+int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
+                        int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
+                        int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
+                        int32_t* offsets);
+
+int wide_launch_unpermute(cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
+                          const int32_t* offsets, int T, int NG, int G, int elem_bytes, void* dst);
+
+// CUDA-core FFN / O-proj (any shape, fp32 or bf16).  `h` is scratch [T, Dff] in `dtype`.
+int wide_launch_ffn_simt(cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd,
+                         int dtype, int T, int D, int Dff, int G, const uint32_t* mask_bits, void* y,
+                         int out_dtype, void* h);
+int wide_launch_oproj_simt(cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
+                           int K, int G, const uint32_t* mask_bits, void* y, int out_dtype);
+
+// tcgen05 prefill path (bf16).  `h` is scratch [T, Dff] bf16.
+int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg,
+                               const void* wu, const void* wd, int T, int D, int Dff, int G,
+                               const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
+                               const int32_t* work_list, const int32_t* n_work, void* y,
+                               int out_dtype, void* h);
+// `a_masked` is scratch [T, K] bf16.
+int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
+                                 int D, int K, int G, const uint32_t* mask_bits, void* y,
+                                 int out_dtype, void* a_masked);
+
+// tcgen05 decode path (bf16, T <= WIDE_DECODE_MAX_TOKENS).
+size_t wide_decode_workspace(int T, int D, int inner);
+int wide_launch_ffn_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg,
+                              const void* wu, const void* wd, int T, int D, int Dff, int G,
+                              const uint32_t* mask_bits, void* y, int out_dtype, void* ws);
+int wide_launch_oproj_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
+                                int D, int K, int G, const uint32_t* mask_bits, void* y,
+                                int out_dtype, void* ws);

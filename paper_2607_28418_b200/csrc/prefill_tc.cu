@@ -1,0 +1,548 @@
+// Prefill path of wide_ffn / wide_oproj on the 5th-generation tensor cores (tcgen05 + TMEM),
+// operands staged by TMA (weights, hidden activation) or gathered with cp.async (token rows
+// selected through the reorder permutation).
+//
+//   gateup_kernel  Algorithm 2 (GEMM-MN, N-axis): one work item = one active (token tile, group)
+//                  pair of the reordered mask.  A = 128 gathered rows of X, B = the group's rows of
+//                  W_gate and W_up side by side (one UMMA of N = 2*BN), fp32 accumulators in TMEM,
+//                  epilogue silu(gate)*up -> bf16, scattered through the permutation straight into
+//                  the token-major hidden activation H (rows past the group's count are dropped).
+//   down_kernel    Eq. 10 (K-axis) in owner-computes form: a CTA owns a 128-token x BN output tile
+//                  in original token order and walks the K-groups, skipping every group that no
+//                  token of the tile selected (block-level predicate on the unsorted mask);
+//                  inactive (token, group) pairs inside an active block are exact zeros of H.  No
+//                  atomics, deterministic, output written once.
+//
+// Both kernels are persistent (one CTA per SM) and warp-specialised: TMA producer, UMMA issuer,
+// (gather warps,) epilogue warps; a 4-stage shared-memory ring and two TMEM accumulator buffers
+// overlap loads, MMAs and epilogues.  Every mbarrier wait is bounded.
+#include <cuda.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace {
+
+using namespace wptx;
+
+constexpr int kStages = 4;
+constexpr int kBM = 128;              // rows per tile (UMMA M)
+constexpr int kBK = 64;               // bf16 elements per k-step = one 128-byte swizzle row
+constexpr int kABytes = kBM * kBK * 2;  // 16 KB
+constexpr int kAccCols = 256;         // TMEM columns per accumulator buffer
+constexpr int kMaskWords = WIDE_MAX_GROUPS / 32;
+
+struct SmemLayout {
+    uint8_t* stage_base;
+    uint32_t full, empty, tfull, tempty;  // shared-space addresses of barrier arrays
+    uint32_t* tmem_slot;
+    volatile int* abort_flag;
+};
+
+template <int kBBytes>
+__device__ __forceinline__ SmemLayout carve_smem(uint8_t* raw) {
+    SmemLayout L;
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    L.stage_base = base;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStages * (kABytes + kBBytes));
+    L.full = smem_u32(bars);
+    L.empty = smem_u32(bars + kStages);
+    L.tfull = smem_u32(bars + 2 * kStages);
+    L.tempty = smem_u32(bars + 2 * kStages + 2);
+    L.tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+    L.abort_flag = reinterpret_cast<volatile int*>(L.tmem_slot + 1);
+    return L;
+}
+
+template <int kBBytes>
+constexpr int smem_bytes() {
+    return kStages * (kABytes + kBBytes) + (2 * kStages + 4) * 8 + 16 + 1024;
+}
+
+// OR of the mask words of tokens [t0, t0 + 128) computed by one warp; every lane gets the result.
+__device__ __forceinline__ void tile_mask_or(const uint32_t* __restrict__ mask_bits, int words, int T, int t0,
+                                             int lane, uint32_t (&act)[kMaskWords]) {
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) act[w] = 0u;
+    if (mask_bits == nullptr) {
+#pragma unroll
+        for (int w = 0; w < kMaskWords; ++w) act[w] = 0xffffffffu;
+        return;
+    }
+    for (int i = lane; i < kBM; i += 32) {
+        const int t = t0 + i;
+        if (t < T) {
+#pragma unroll
+            for (int w = 0; w < kMaskWords; ++w)
+                if (w < words) act[w] |= mask_bits[static_cast<size_t>(t) * words + w];
+        }
+    }
+#pragma unroll
+    for (int w = 0; w < kMaskWords; ++w) act[w] = __reduce_or_sync(0xffffffffu, act[w]);
+}
+
+__device__ __forceinline__ void report_timeout(int* status) { atomicExch(status, WIDE_ERR_TIMEOUT); }
+
+// Give copies that are still in flight time to land before the CTA gives up its shared memory.
+__device__ __forceinline__ void abort_grace() {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ======================================================================================= down
+// Y[T, N] = A[T, K] * B[N, K]^T with K split into groups of G; group g is skipped for a token tile
+// when no token of the tile has bit g set (mask_bits == nullptr: nothing is skipped).
+template <int BN>
+__global__ void __launch_bounds__(192, 1)
+down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const uint32_t* __restrict__ mask_bits, int words, int T, int N, int K, int G, void* __restrict__ Y,
+            int out_bf16, int* __restrict__ status, unsigned long long wait_ns) {
+    constexpr int kBBytes = BN * kBK * 2;
+    constexpr int kStageBytes = kABytes + kBBytes;
+    extern __shared__ uint8_t smem_raw[];
+    SmemLayout L = carve_smem<kBBytes>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(L.full + 8 * s, 1);
+            mbar_init(L.empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(L.tfull + 8 * b, 1);
+            mbar_init(L.tempty + 8 * b, 4);
+        }
+        *L.abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(L.tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *L.tmem_slot;
+
+    const int n_m = (T + kBM - 1) / kBM, n_n = (N + BN - 1) / BN;
+    const int n_tiles = n_m * n_n;
+    const int NG = K / G, ksub = G / kBK;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const int m = tile % n_m, n = tile / n_m;
+            uint32_t act[kMaskWords];
+            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            if (lane == 0) {
+                for (int g = 0; g < NG && ok; ++g) {
+                    if (!((act[g >> 5] >> (g & 31)) & 1u)) continue;
+                    for (int kk = 0; kk < ksub; ++kk, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1;
+                        if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
+                        mbar_arrive_expect_tx(L.full + 8 * s, kStageBytes);
+                        const uint32_t a_dst = smem_u32(L.stage_base + s * kStageBytes);
+                        const int kcol = g * G + kk * kBK;
+                        tma_load_2d(a_dst, &tmA, kcol, m * kBM, L.full + 8 * s);
+                        tma_load_2d(a_dst + kABytes, &tmB, kcol, n * BN, L.full + 8 * s);
+                    }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        }
+        if (!ok && lane == 0) { report_timeout(status); abort_grace(); }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ UMMA issuer
+        constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN);
+        int it = 0, tc = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
+            const int m = tile % n_m;
+            uint32_t act[kMaskWords];
+            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            if (lane == 0) {
+                const int buf = tc & 1;
+                const uint32_t tph = (tc >> 1) & 1;
+                if (!mbar_wait(L.tempty + 8 * buf, tph ^ 1u, wait_ns, L.abort_flag)) ok = false;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * kAccCols;
+                uint32_t accumulate = 0;
+                for (int g = 0; g < NG && ok; ++g) {
+                    if (!((act[g >> 5] >> (g & 31)) & 1u)) continue;
+                    for (int kk = 0; kk < ksub; ++kk, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1;
+                        if (!mbar_wait(L.full + 8 * s, ph, wait_ns, L.abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = smem_u32(L.stage_base + s * kStageBytes);
+                        const uint64_t adesc = umma_desc_sw128(a_addr);
+                        const uint64_t bdesc = umma_desc_sw128(a_addr + kABytes);
+#pragma unroll
+                        for (int k4 = 0; k4 < kBK / 16; ++k4) {
+                            umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(L.empty + 8 * s);
+                    }
+                }
+                if (ok) {
+                    if (accumulate) umma_commit(L.tfull + 8 * buf);
+                    else mbar_arrive(L.tfull + 8 * buf);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        }
+        if (!ok && lane == 0) report_timeout(status);
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        int tc = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
+            const int m = tile % n_m, n = tile / n_m;
+            uint32_t act[kMaskWords];
+            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            bool any = false;
+            for (int g = 0; g < NG; ++g) any = any || ((act[g >> 5] >> (g & 31)) & 1u);
+            const int buf = tc & 1;
+            const uint32_t tph = (tc >> 1) & 1;
+            if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int row = m * kBM + q * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                if (any) {
+                    tmem_ld_32x32(taddr + c0, r);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                }
+                const int col = n * BN + c0;
+                if (row < T && col + 32 <= N) {
+                    if (out_bf16) {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(row) * N + col);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 o;
+                            o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+                            o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                            o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                            o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                            dst[v] = o;
+                        }
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(Y) + static_cast<size_t>(row) * N + col);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(L.tempty + 8 * buf);
+        }
+        if (!ok && lane == 0) report_timeout(status);
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ======================================================================================= gate/up
+// Work item j -> (pair = j / nsub, sub = j % nsub); pair = work_list[pair] = (tile m, group g);
+// channels [g*G + sub*BN, +BN) of W_gate and W_up; rows = perm[g][m*128 .. m*128+127].
+template <int BN>  // channels per item (UMMA N = 2*BN)
+__global__ void __launch_bounds__(320, 1)
+gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
+              const __nv_bfloat16* __restrict__ X, const int32_t* __restrict__ perm,
+              const int32_t* __restrict__ counts, const int32_t* __restrict__ work_list,
+              const int32_t* __restrict__ n_work, int T, int D, int Dff, int G, __nv_bfloat16* __restrict__ H,
+              int* __restrict__ status, unsigned long long wait_ns) {
+    constexpr int kBBytes = 2 * BN * kBK * 2;
+    constexpr int kStageBytes = kABytes + kBBytes;
+    constexpr int kLag = 2;  // gather warps signal stage (it - kLag) after issuing stage it
+    extern __shared__ uint8_t smem_raw[];
+    SmemLayout L = carve_smem<kBBytes>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(L.full + 8 * s, 1 + 4);  // TMA producer + 4 gather warps
+            mbar_init(L.empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(L.tfull + 8 * b, 1);
+            mbar_init(L.tempty + 8 * b, 4);
+        }
+        *L.abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmG);
+        prefetch_tmap(&tmU);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(L.tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *L.tmem_slot;
+
+    const int nsub = G / BN;
+    const int n_items = (*n_work) * nsub;
+    const int nk = D / kBK;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (weights)
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const int pair = item / nsub, sub = item - pair * nsub;
+                const int g = work_list[2 * pair + 1];
+                const int crow = g * G + sub * BN;
+                for (int k = 0; k < nk; ++k, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1;
+                    if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(L.full + 8 * s, kBBytes);
+                    const uint32_t b_dst = smem_u32(L.stage_base + s * kStageBytes) + kABytes;
+                    tma_load_2d(b_dst, &tmG, k * kBK, crow, L.full + 8 * s);
+                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, crow, L.full + 8 * s);
+                }
+            }
+            if (!ok) { report_timeout(status); abort_grace(); }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ UMMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, 2 * BN);
+            int it = 0, tc = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tc) {
+                const int buf = tc & 1;
+                const uint32_t tph = (tc >> 1) & 1;
+                if (!mbar_wait(L.tempty + 8 * buf, tph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * kAccCols;
+                for (int k = 0; k < nk; ++k, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1;
+                    if (!mbar_wait(L.full + 8 * s, ph, wait_ns, L.abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(L.stage_base + s * kStageBytes);
+                    const uint64_t adesc = umma_desc_sw128(a_addr);
+                    const uint64_t bdesc = umma_desc_sw128(a_addr + kABytes);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBK / 16; ++k4)
+                        umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (k > 0 || k4 > 0) ? 1u : 0u);
+                    umma_commit(L.empty + 8 * s);
+                }
+                if (ok) umma_commit(L.tfull + 8 * buf);
+            }
+            if (!ok) report_timeout(status);
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------------ A gather (warps 2..5)
+        const int r = (warp - 2) * 32 + lane;  // tile row owned by this thread
+        const uint32_t row_off = static_cast<uint32_t>(r) * 128u;
+        const uint32_t sw = static_cast<uint32_t>(r & 7);
+        int it = 0;        // stages issued
+        int signalled = 0; // stages whose arrival has been posted
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int pair = item / nsub;
+            const int m = work_list[2 * pair], g = work_list[2 * pair + 1];
+            int j = m * kBM + r;
+            if (j >= T) j = T - 1;
+            const int tok = perm[static_cast<size_t>(g) * T + j];
+            const uint8_t* src = reinterpret_cast<const uint8_t*>(X + static_cast<size_t>(tok) * D);
+            for (int k = 0; k < nk; ++k, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1;
+                if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
+                const uint32_t a_dst = smem_u32(L.stage_base + s * kStageBytes) + row_off;
+                const uint8_t* p = src + static_cast<size_t>(k) * (kBK * 2);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) cp_async_16(a_dst + ((static_cast<uint32_t>(c) ^ sw) << 4), p + 16 * c);
+                cp_async_commit();
+                if (it - signalled >= kLag) {
+                    cp_async_wait<kLag>();
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(L.full + 8 * (signalled % kStages));
+                    ++signalled;
+                }
+            }
+        }
+        // drain: everything issued has landed; post the remaining arrivals
+        cp_async_wait<0>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (ok) {
+            for (; signalled < it; ++signalled)
+                if (lane == 0) mbar_arrive(L.full + 8 * (signalled % kStages));
+        } else if (lane == 0) {
+            report_timeout(status);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 6..9)
+        const int q = warp & 3;
+        int tc = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tc) {
+            const int pair = item / nsub, sub = item - pair * nsub;
+            const int m = work_list[2 * pair], g = work_list[2 * pair + 1];
+            const int j = m * kBM + q * 32 + lane;
+            const bool live = j < counts[g];
+            const int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
+            __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN;
+            const int buf = tc & 1;
+            const uint32_t tph = (tc >> 1) & 1;
+            if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t gr[32], ur[32];
+                tmem_ld_32x32(taddr + c0, gr);
+                tmem_ld_32x32(taddr + BN + c0, ur);
+                tmem_ld_wait();
+                if (live) {
+                    uint4* dst = reinterpret_cast<uint4*>(hrow + c0);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int i = 8 * v + 2 * e;
+                            o[e] = pack_bf16(silu_mul(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
+                                             silu_mul(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
+                        }
+                        dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(L.tempty + 8 * buf);
+        }
+        if (!ok && lane == 0) report_timeout(status);
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// H~[t, c] = M[t, c/G] ? a[t, c] : 0   (16-byte pieces; G*2 bytes is a multiple of 16)
+__global__ void __launch_bounds__(256) mask_rows_kernel(const uint4* __restrict__ a, const uint32_t* __restrict__ mask_bits,
+                                                        int words, int T, int K, int G, uint4* __restrict__ out) {
+    const int vec_per_row = K / 8, vec_per_group = G / 8;
+    const long long total = static_cast<long long>(T) * vec_per_row;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int t = static_cast<int>(i / vec_per_row);
+        const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
+        out[i] = wide_mask_bit(mask_bits, words, t, g) ? a[i] : make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// --------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 row-major [rows, cols] tensor, box = [box_rows, 64 columns], 128-byte swizzle.
+bool make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
+                    uint32_t box_rows) {
+    if (!ctx->encode_tiled) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int BN>
+int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
+                int N, int K, int G, void* Y, int out_dtype) {
+    CUtensorMap tmA, tmB;
+    if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, N, K, BN)) return WIDE_ERR_CUDA;
+    constexpr int smem = smem_bytes<BN * kBK * 2>();
+    WIDE_CUDA_CHECK(cudaFuncSetAttribute(down_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int n_tiles = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+    const int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
+    const int words = (K / G + 31) / 32;
+    down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
+                                            ctx->d_status, ctx->wait_ns);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+}
+
+template <int BN>
+int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, int T, int D,
+                  int Dff, int G, const int32_t* perm, const int32_t* counts, const int32_t* work_list,
+                  const int32_t* n_work, void* h) {
+    CUtensorMap tmG, tmU;
+    if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
+    constexpr int smem = smem_bytes<2 * BN * kBK * 2>();
+    WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    gateup_kernel<BN><<<ctx->sm_count, 320, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm, counts,
+                                                       work_list, n_work, T, D, Dff, G,
+                                                       static_cast<__nv_bfloat16*>(h), ctx->d_status, ctx->wait_ns);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+}
+
+}  // namespace
+
+int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
+                               const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
+                               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
+                               const int32_t* n_work, void* y, int out_dtype, void* h) {
+    if (T == 0) return WIDE_OK;
+    // inactive (token, group) pairs of H must read as zero in the down projection
+    WIDE_CUDA_CHECK(cudaMemsetAsync(h, 0, static_cast<size_t>(T) * Dff * 2, s));
+    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h)
+                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h);
+    if (rc != WIDE_OK) return rc;
+    return launch_down<256>(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype);
+}
+
+int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T, int D,
+                                 int K, int G, const uint32_t* mask_bits, void* y, int out_dtype,
+                                 void* a_masked) {
+    if (T == 0) return WIDE_OK;
+    const int words = (K / G + 31) / 32;
+    const long long total = static_cast<long long>(T) * (K / 8);
+    long long blocks = (total + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    mask_rows_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(a), mask_bits, words, T, K, G,
+                                                              static_cast<uint4*>(a_masked));
+    if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
+    return launch_down<256>(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype);
+}

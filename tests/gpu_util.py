@@ -1,0 +1,46 @@
+"""Helpers shared by the GPU parity tests: upload of the seeded host buffers, tolerance check."""
+import numpy as np
+import torch
+
+from paper_2607_28418_b200 import synth
+
+REL_TOL = 2e-2  # max |err| <= REL_TOL * max |ref|  (bf16 inputs, fp32 accumulation)
+
+
+def to_dev(a: np.ndarray, dtype: str) -> torch.Tensor:
+    """float32 host array -> CUDA tensor of the workload dtype (exact for bf16-rounded inputs)."""
+    if dtype == "bf16":
+        bits = synth.to_bf16_bits(a)
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+
+
+def bits_to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int32)).cuda()
+
+
+def bits_to_host(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32)
+
+
+def assert_close(y_gpu: torch.Tensor, y_ref: np.ndarray, what: str = "", rel: float = REL_TOL):
+    got = y_gpu.float().cpu().numpy().astype(np.float64)
+    scale = float(np.abs(y_ref).max())
+    err = float(np.abs(got - y_ref).max()) if got.size else 0.0
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    assert err <= rel * scale + 1e-30, f"{what}: max|err| {err:.4e} > {rel} * max|ref| {scale:.4e}"
+    return err / scale if scale > 0 else 0.0
+
+
+def meta_to_dev(meta: dict) -> dict:
+    """Oracle reorder output -> device tensors in the layout wide_ffn expects."""
+    n_tiles, NG = meta["tile_map"].shape
+    wl = np.full((max(n_tiles * NG, 1), 2), -1, dtype=np.int32)
+    wl[: meta["n_work"]] = meta["work_list"]
+    return {
+        "perm": torch.from_numpy(meta["perm"]).cuda(),
+        "counts": torch.from_numpy(meta["counts"]).cuda(),
+        "work_list": torch.from_numpy(wl).cuda(),
+        "n_work": torch.tensor([meta["n_work"]], dtype=torch.int32).cuda(),
+        "offsets": torch.from_numpy(meta["offsets"]).cuda(),
+    }

@@ -1,0 +1,170 @@
+"""GPU parity: wide_ffn / wide_oproj (CUDA-core, tcgen05 prefill and decode paths) vs the oracle.
+
+Stage-wise: each stage gets the oracle's mask / metadata as input, so a routing difference
+cannot hide as an FFN error.  Float bar: max|err| <= 2e-2 * max|ref|.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import wide_oracle as wo
+from paper_2607_28418_b200 import synth
+from tests.gpu_util import assert_close, bits_to_dev, meta_to_dev, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2607_28418_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.status() == 0
+    c.close()
+
+
+def _ffn_inputs(cfg, seed, mask=None):
+    case = synth.make_ffn_case(cfg, seed)
+    if mask is None:
+        mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router"]), cfg.k)
+    dev = {k: to_dev(case[k], cfg.dtype) for k in ("x", "w_gate", "w_up", "w_down")}
+    return case, mask, dev
+
+
+def _run_ffn(ctx, cfg, seed, flags, mask=None, out_dtype=None, with_meta=True):
+    from paper_2607_28418_b200 import binding
+    case, mask, dev = _ffn_inputs(cfg, seed, mask)
+    ref = wo.ffn(case["x"], case["w_gate"], case["w_up"], case["w_down"], mask, cfg.group)
+    bits = bits_to_dev(wo.pack_mask_bits(mask))
+    meta = meta_to_dev(wo.reorder(mask, 128)) if with_meta else None
+    y = binding.wide_ffn(ctx, dev["x"], dev["w_gate"], dev["w_up"], dev["w_down"], cfg.group, bits, meta,
+                         out_dtype=out_dtype, flags=flags)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    return y, ref, mask
+
+
+# ----------------------------------------------------------------------------- CUDA-core path
+def test_tiny_config_fp32_simt(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.CONFIGS["tiny"]
+    y, ref, _ = _run_ffn(ctx, cfg, 0, binding.FLAG_SIMT, with_meta=False)
+    assert_close(y, ref, "tiny fp32", rel=1e-4)
+
+
+@pytest.mark.parametrize("T,D,Dff,G,k,dtype", [(70, 96, 320, 32, 5, "fp32"), (130, 128, 512, 16, 9, "bf16"),
+                                               (33, 64, 256, 64, 0, "bf16"), (33, 64, 256, 64, 4, "bf16")])
+def test_simt_odd_shapes(ctx, T, D, Dff, G, k, dtype):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=T, hidden=D, d_ff=Dff, group=G, k=k, dtype=dtype)
+    y, ref, _ = _run_ffn(ctx, cfg, 1, binding.FLAG_SIMT, with_meta=False)
+    if k == 0:
+        assert (y.float().cpu().numpy() == 0).all()
+    else:
+        assert_close(y, ref, f"simt {T}x{D}x{Dff}")
+
+
+# ----------------------------------------------------------------------------- tcgen05 prefill
+@pytest.mark.parametrize("T,D,Dff,G,k", [(128, 256, 512, 128, 2), (300, 512, 1024, 128, 4),
+                                         (257, 512, 1024, 64, 8), (200, 256, 1024, 256, 2),
+                                         (640, 1024, 2048, 128, 8)])
+def test_prefill_tc_matches_oracle(ctx, T, D, Dff, G, k):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=T, hidden=D, d_ff=Dff, group=G, k=k)
+    y, ref, _ = _run_ffn(ctx, cfg, 2, binding.FLAG_FORCE_PREFILL)
+    assert_close(y, ref, f"prefill tc {T}x{D}x{Dff} G{G}")
+
+
+def test_prefill_tc_fp32_output_and_variable_budget(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=384, hidden=512, d_ff=1024, group=128, k=4)
+    mask = synth.bernoulli_mask(3, 384, 8, 0.4)     # variable active groups per token
+    mask[5] = False                                  # a token with nothing active -> zero row
+    mask[:, 6] = False                               # a group nobody selects -> skipped block column
+    y, ref, _ = _run_ffn(ctx, cfg, 3, binding.FLAG_FORCE_PREFILL, mask=mask, out_dtype=torch.float32)
+    assert_close(y, ref, "prefill tc fp32 out")
+    assert (y[5] == 0).all()
+
+
+def test_prefill_tc_closed_cases(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=256, hidden=256, d_ff=512, group=128, k=4)
+    ones = np.ones((256, 4), dtype=bool)
+    y, ref, _ = _run_ffn(ctx, cfg, 4, binding.FLAG_FORCE_PREFILL, mask=ones)        # dense SwiGLU
+    assert_close(y, ref, "all-ones")
+    y, _, _ = _run_ffn(ctx, cfg, 4, binding.FLAG_FORCE_PREFILL, mask=~ones)         # exact zero
+    assert (y.float().cpu().numpy() == 0).all()
+    # clustered: first half of the tokens uses groups {0,1}, second half {2,3}: whole blocks skipped
+    m = np.zeros((256, 4), dtype=bool)
+    m[:128, :2] = True
+    m[128:, 2:] = True
+    y, ref, _ = _run_ffn(ctx, cfg, 4, binding.FLAG_FORCE_PREFILL, mask=m)
+    assert_close(y, ref, "block-clustered")
+
+
+def test_prefill_tc_agrees_with_simt_and_is_deterministic(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=300, hidden=512, d_ff=1024, group=128, k=4)
+    y1, ref, mask = _run_ffn(ctx, cfg, 6, binding.FLAG_FORCE_PREFILL)
+    y2, _, _ = _run_ffn(ctx, cfg, 6, binding.FLAG_FORCE_PREFILL)
+    assert torch.equal(y1, y2)
+    y3, _, _ = _run_ffn(ctx, cfg, 6, binding.FLAG_SIMT, with_meta=False)
+    assert_close(y1, y3.float().cpu().numpy().astype(np.float64), "tc vs simt")
+
+
+# ----------------------------------------------------------------------------- decode
+@pytest.mark.parametrize("B", [1, 8, 33, 64])
+@pytest.mark.parametrize("G", [64, 128, 256])
+def test_decode_matches_oracle(ctx, B, G):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=B, hidden=512, d_ff=2048, group=G, k=2048 // G // 2)
+    y, ref, _ = _run_ffn(ctx, cfg, 7 + B, binding.FLAG_NONE, with_meta=False)
+    assert_close(y, ref, f"decode B{B} G{G}")
+
+
+def test_decode_clustered_union_and_zero_cases(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=16, hidden=512, d_ff=2048, group=128, k=8, router="clustered")
+    y, ref, mask = _run_ffn(ctx, cfg, 11, binding.FLAG_NONE, with_meta=False)
+    assert len({r.tobytes() for r in mask}) <= 4
+    assert_close(y, ref, "decode clustered")
+    zero = np.zeros((16, 16), dtype=bool)
+    y, _, _ = _run_ffn(ctx, cfg, 11, binding.FLAG_NONE, mask=zero, with_meta=False)
+    assert (y.float().cpu().numpy() == 0).all()
+    y1, ref, _ = _run_ffn(ctx, cfg, 11, binding.FLAG_NONE, mask=~zero, with_meta=False, out_dtype=torch.float32)
+    assert_close(y1, ref, "decode dense fp32 out")
+
+
+# ----------------------------------------------------------------------------- O-projection
+def _run_oproj(ctx, T, D, K, G, k, flags, dtype="bf16", seed=0):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=T, hidden=D, d_ff=D, group=64, k=1, dtype=dtype, attn_dim=K, attn_group=G,
+                           attn_k=k)
+    case = synth.make_oproj_case(cfg, seed)
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router_attn"]), k)
+    ref = wo.oproj(case["attn_out"], case["w_o"], mask, G)
+    y = binding.wide_oproj(ctx, to_dev(case["attn_out"], dtype), to_dev(case["w_o"], dtype), G,
+                           bits_to_dev(wo.pack_mask_bits(mask)), meta_to_dev(wo.reorder(mask, 128)), flags=flags)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    return y, ref
+
+
+def test_oproj_simt_fp32(ctx):
+    from paper_2607_28418_b200 import binding
+    y, ref = _run_oproj(ctx, 100, 96, 160, 32, 2, binding.FLAG_SIMT, dtype="fp32")
+    assert_close(y, ref, "oproj simt fp32", rel=1e-4)
+
+
+@pytest.mark.parametrize("T,D,K,G,k", [(300, 512, 1024, 512, 1), (256, 256, 1024, 128, 3), (130, 512, 512, 64, 4)])
+def test_oproj_prefill_tc(ctx, T, D, K, G, k):
+    from paper_2607_28418_b200 import binding
+    y, ref = _run_oproj(ctx, T, D, K, G, k, binding.FLAG_FORCE_PREFILL)
+    assert_close(y, ref, f"oproj prefill {T}x{D}x{K} G{G}")
+
+
+@pytest.mark.parametrize("B", [1, 32])
+def test_oproj_decode(ctx, B):
+    from paper_2607_28418_b200 import binding
+    y, ref = _run_oproj(ctx, B, 512, 1024, 512, 1, binding.FLAG_NONE)
+    assert_close(y, ref, f"oproj decode B{B}")
