@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the WIDE hot path (route -> reorder -> masked SwiGLU FFN) on synthetic
+Llama-shaped layers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload llama7b_prefill|llama8b_prefill|llama13b_layer|llama8b_decode]
+                    [--batch B] [--router random|clustered|clustered_corr] [--k K] [--group G]
+
+One step = one pass of the whole path over one batch of tokens.  Rank 0 prints one JSON line.
+With N > 1 (torchrun) every rank runs its own token shard with replicated weights and no
+data-path collective (weak scaling); the timed region is bracketed by a barrier and the elapsed
+time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_28418_b200 import synth  # noqa: E402
+
+METRIC = "masked-layer tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
+# (profiles/), keyed by (kernel, workload); None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return dict(FALLBACK_PEAKS)
+
+
+# ------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------- workload
+def make_config(args) -> synth.WideConfig:
+    cfg = synth.CONFIGS[args.workload]
+    kw = {}
+    if args.batch:
+        kw["tokens"] = args.batch
+    if args.router:
+        kw["router"] = args.router
+    if args.group:
+        kw["group"] = args.group
+        kw["k"] = (cfg.d_ff // args.group) * cfg.k // cfg.n_groups
+    if args.k is not None:
+        kw["k"] = args.k
+    return cfg.with_(**kw) if kw else cfg
+
+
+def aggregate(units_per_rank: float, steps: int, elapsed_ms_max: float, world: int) -> float:
+    """Whole-job throughput: units processed by all ranks / (max-over-ranks time)."""
+    return units_per_rank * world * steps / (elapsed_ms_max * 1e-3)
+
+
+def reduce_max_ms(ms: float, world: int, device=None) -> float:
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def flops_ffn_active(cfg) -> float:
+    return 6.0 * cfg.tokens * cfg.k * cfg.group * cfg.hidden
+
+
+# ------------------------------------------------------------------------------- reference arm
+def oracle_sample_step(case, cfg, sample_tokens):
+    from oracle import wide_oracle as wo
+    return wo.layer_ffn(case["x"][:sample_tokens], case["w_router"], case["w_gate"], case["w_up"], case["w_down"],
+                        cfg.group, cfg.k, cfg.tile_m)
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(case, cfg, sample_tokens, steps, warmup):
+    for _ in range(warmup):
+        oracle_sample_step(case, cfg, sample_tokens)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(case, cfg, sample_tokens)
+    dt = time.perf_counter() - t0
+    return sample_tokens * steps / dt, dt / steps * 1e3
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = make_config(args)
+    case = synth.make_ffn_case(cfg, 0, tokens=min(cfg.tokens, args.oracle_tokens))
+    sample = min(cfg.tokens, args.oracle_tokens)
+    steps = max(1, args.steps)
+    value, ms = time_oracle(case, cfg, sample, steps, min(args.warmup, 1))
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "tokens": cfg.tokens, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
+                   "group": cfg.group, "k": cfg.k, "router": cfg.router},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": f"each step = the first {sample} of {cfg.tokens} tokens through route, top-k, "
+                                   "reorder and the masked FFN in fp64 numpy"},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_28418_b200 import binding
+    to_dev = binding.upload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    cfg = make_config(args)
+    peaks = load_peaks()
+    ctx = binding.Context(local)
+    case = synth.make_ffn_case(cfg, 1000 * rank)       # every rank its own token shard
+    d = {k: to_dev(v, cfg.dtype) for k, v in case.items()}
+    T, NG = cfg.tokens, cfg.n_groups
+    W = (NG + 31) // 32
+    bits = torch.empty((T, W), dtype=torch.int32, device=dev)
+    y = torch.empty((T, cfg.hidden), dtype=torch.bfloat16, device=dev)
+    meta = None
+    decode = T <= binding.DECODE_MAX_TOKENS
+
+    def step(k=cfg.k):
+        nonlocal meta
+        binding.wide_route(ctx, d["x"], d["w_router"], NG, k, mask_bits=bits)
+        if not decode:
+            meta = binding.wide_reorder(ctx, bits, NG, 128, out=meta)
+        binding.wide_ffn(ctx, d["x"], d["w_gate"], d["w_up"], d["w_down"], cfg.group, bits, meta, y=y)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync_all()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        sync_all()
+        return reduce_max_ms(e0.elapsed_time(e1), world, dev)
+
+    flush = None
+    if decode or args.flush_l2:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during warm-up")
+
+    # ---- timed region: K steps, kernels bracketed by the library's own event pairs
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ctx.profile_begin(64 * args.steps + 64)
+    if flush is None:
+        ms_total = timed(step, args.steps)
+    else:
+        # weights of a decode step fit in L2 only partly; flush between steps, time each step
+        ms_total = 0.0
+        for _ in range(args.steps):
+            flush.zero_()
+            ms_total += timed(step, 1)
+    prof = ctx.profile_end()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during the timed region")
+    value = aggregate(T, args.steps, ms_total, world)
+
+    # ---- end to end: pinned host input -> device, whole path, result -> host, every step
+    x_host = torch.from_numpy(synth.to_bf16_bits(case["x"]).view(np.int16)).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty((T, cfg.hidden), dtype=torch.bfloat16).pin_memory()
+
+    def step_e2e():
+        d["x"].copy_(x_host, non_blocking=True)
+        step()
+        y_host.copy_(y, non_blocking=True)
+
+    for _ in range(2):
+        step_e2e()
+    e2e_steps = max(3, min(args.steps, 10))
+    ms_e2e = timed(step_e2e, e2e_steps)
+    e2e_value = aggregate(T, e2e_steps, ms_e2e, world)
+
+    # ---- the same kernels run dense (k = N_G)
+    dense_ms = None
+    if not args.no_dense:
+        for _ in range(2):
+            step(NG)
+        dense_steps = max(3, min(args.steps, 10))
+        dense_ms = timed(lambda: step(NG), dense_steps) / dense_steps
+        step()
+
+    # ---- roofline of the dominant kernel (largest share of the timed region)
+    kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
+                   "share": round(v["total_ms"] / max(sum(p["total_ms"] for p in prof.values()), 1e-9), 4)}
+               for n, v in prof.items()}
+    dom = max(prof, key=lambda n: prof[n]["total_ms"]) if prof else None
+    roofline = None
+    if dom:
+        avg_s = prof[dom]["total_ms"] / prof[dom]["launches"] * 1e-3
+        tkgd = float(T) * cfg.k * cfg.group * cfg.hidden
+        if decode:
+            # union of active groups x (gate + up + down) weight bytes, bf16
+            union_words = np.bitwise_or.reduce(bits.cpu().numpy().view(np.uint32), axis=0)
+            n_union = sum(bin(int(w)).count("1") for w in union_words)
+            per_group = cfg.group * cfg.hidden * 2
+            bytes_alg = {"decode_stream_gateup": 2.0 * n_union * per_group,
+                         "decode_stream_down": 1.0 * n_union * per_group}.get(dom, 3.0 * n_union * per_group)
+            ach = bytes_alg / avg_s / 1e9
+            roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.name)),
+                        "peak_source": peaks["source"], "n_union": n_union}
+        else:
+            flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd}.get(dom, 6.0 * tkgd)
+            ach = flops_alg / avg_s / 1e12
+            roofline = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                        "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                        "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.name)), "peak_source": peaks["source"]}
+
+    line = None
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        ffn_ms = sum(v["total_ms"] for n, v in prof.items() if n.startswith(("prefill_", "decode_"))) / args.steps
+        line = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "tokens_per_gpu": T, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
+                       "group": cfg.group, "n_groups": NG, "k": cfg.k, "router": cfg.router,
+                       "parallelism": f"token-sharded x{world}, weights replicated, no collective",
+                       "l2": "flushed between steps" if flush is not None else
+                             "inputs larger than L2 (weights %.0f MB)" % (3 * cfg.d_ff * cfg.hidden * 2 / 1e6)},
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": x_host.numel() * 2,
+                    "d2h_bytes_per_step": y_host.numel() * 2,
+                    "note": "activations cross PCIe every step; weights are parameters and stay resident"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roofline,
+            "kernels": kernels,
+            "ffn": {"ms": ffn_ms, "active_tflops": flops_ffn_active(cfg) / (ffn_ms * 1e-3) / 1e12 if ffn_ms else None,
+                    "frac_of_bf16_peak": (flops_ffn_active(cfg) / (ffn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"])
+                    if ffn_ms else None},
+            "dense": {"ms_per_step": dense_ms, "speedup_vs_dense": (dense_ms / ms_step) if dense_ms else None,
+                      "ideal": NG / cfg.k if cfg.k else None},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            sample = min(T, args.oracle_tokens)
+            v, ms = time_oracle(case, cfg, sample, 1, 0)
+            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"first {sample} of {T} tokens, one pass of route, top-k, reorder and "
+                                              f"masked FFN in fp64 numpy ({ms / 1e3:.1f} s)"}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_prefill", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--batch", type=int, default=0, help="override the token count (decode batch)")
+    ap.add_argument("--router", default="", choices=["", "random", "clustered", "clustered_corr"])
+    ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--group", type=int, default=0)
+    ap.add_argument("--flush-l2", action="store_true")
+    ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--oracle-tokens", type=int, default=512)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

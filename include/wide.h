@@ -91,6 +91,16 @@ WIDE_API int wide_status(wide_ctx* ctx, void* stream, int* status);
 /* Override the bound of every device-side wait (nanoseconds; default 2e9). */
 WIDE_API int wide_set_wait_limit_ns(wide_ctx* ctx, uint64_t ns);
 
+/* Per-kernel timing (tracing aid).  wide_profile_begin creates `max_records` CUDA event pairs;
+ * until wide_profile_end every kernel the library launches is bracketed by one pair on its
+ * stream.  wide_profile_end synchronises `stream` and writes one text line per kernel name,
+ * "name,launches,total_ms\n", into buf (NUL-terminated), then frees the events.  Not for use
+ * during stream capture.  wide_launch_count returns the number of kernels launched through this
+ * context since it was created. */
+WIDE_API int wide_profile_begin(wide_ctx* ctx, int max_records);
+WIDE_API int wide_profile_end(wide_ctx* ctx, void* stream, char* buf, size_t buf_bytes);
+WIDE_API int wide_launch_count(wide_ctx* ctx, unsigned long long* count);
+
 WIDE_API const char* wide_strerror(int code);
 WIDE_API int wide_version(void);
 

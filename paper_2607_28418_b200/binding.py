@@ -24,7 +24,8 @@ DECODE_MAX_TOKENS = 64
 MAX_GROUPS = 256
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 
-EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_strerror",
+EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
+           "wide_profile_end", "wide_launch_count", "wide_strerror",
            "wide_version", "wide_workspace_bytes", "wide_route", "wide_reorder", "wide_ffn",
            "wide_oproj", "wide_unpermute"]
 
@@ -53,6 +54,9 @@ def load_library() -> ctypes.CDLL:
     lib.wide_destroy.argtypes = [_c_void_p]
     lib.wide_status.argtypes = [_c_void_p, _c_void_p, ctypes.POINTER(_c_int)]
     lib.wide_set_wait_limit_ns.argtypes = [_c_void_p, ctypes.c_uint64]
+    lib.wide_profile_begin.argtypes = [_c_void_p, _c_int]
+    lib.wide_profile_end.argtypes = [_c_void_p, _c_void_p, ctypes.c_char_p, _c_size_t]
+    lib.wide_launch_count.argtypes = [_c_void_p, ctypes.POINTER(ctypes.c_ulonglong)]
     lib.wide_strerror.argtypes = [_c_int]
     lib.wide_strerror.restype = ctypes.c_char_p
     lib.wide_version.argtypes = []
@@ -145,8 +149,39 @@ class Context:
         _check(self.lib.wide_status(self.handle, _stream(), ctypes.byref(v)), "wide_status")
         return v.value
 
+    def profile_begin(self, max_records: int = 4096):
+        _check(self.lib.wide_profile_begin(self.handle, max_records), "wide_profile_begin")
+
+    def profile_end(self) -> Dict[str, Dict[str, float]]:
+        """{kernel name: {"launches": n, "total_ms": t}} for everything launched since profile_begin."""
+        buf = ctypes.create_string_buffer(8192)
+        _check(self.lib.wide_profile_end(self.handle, _stream(), buf, len(buf)), "wide_profile_end")
+        out = {}
+        for line in buf.value.decode().splitlines():
+            name, n, ms = line.split(",")
+            out[name] = {"launches": int(n), "total_ms": float(ms)}
+        return out
+
+    def launch_count(self) -> int:
+        v = ctypes.c_ulonglong(0)
+        _check(self.lib.wide_launch_count(self.handle, ctypes.byref(v)), "wide_launch_count")
+        return int(v.value)
+
     def set_wait_limit_ns(self, ns: int):
         _check(self.lib.wide_set_wait_limit_ns(self.handle, ns), "wide_set_wait_limit_ns")
+
+
+def upload(a, dtype: str, device: Optional[torch.device] = None) -> torch.Tensor:
+    """Host float32 array -> CUDA tensor of the workload dtype ("bf16": the values must already be
+    bf16-representable, the upload is then exact; "fp32": as is)."""
+    import numpy as np
+
+    from . import synth
+    device = device or torch.device("cuda", torch.cuda.current_device())
+    if dtype == "bf16":
+        bits = synth.to_bf16_bits(a)
+        return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
 
 
 def workspace_bytes(op: int, dtype: int, tokens: int, hidden: int, inner: int, group: int, n_groups: int) -> int:

@@ -1,4 +1,5 @@
 // C ABI of libwide: argument validation, workspace sizing and dispatch.  See include/wide.h.
+#include <cstdio>
 #include <new>
 
 #include "internal.h"
@@ -62,6 +63,9 @@ int wide_create(wide_ctx** out, int device) {
     ctx->sm_count = prop.multiProcessorCount;
     ctx->wait_ns = 2000000000ull;
     ctx->encode_tiled = nullptr;
+    ctx->launches = 0;
+    ctx->prof = nullptr;
+    ctx->prof_cap = ctx->prof_used = 0;
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -80,8 +84,72 @@ int wide_create(wide_ctx** out, int device) {
     return WIDE_OK;
 }
 
+static void free_profile(wide_ctx* ctx) {
+    if (!ctx->prof) return;
+    for (int i = 0; i < ctx->prof_cap; ++i) {
+        cudaEventDestroy(ctx->prof[i].begin);
+        cudaEventDestroy(ctx->prof[i].end);
+    }
+    delete[] ctx->prof;
+    ctx->prof = nullptr;
+    ctx->prof_cap = ctx->prof_used = 0;
+}
+
+int wide_profile_begin(wide_ctx* ctx, int max_records) {
+    if (!ctx || max_records <= 0 || max_records > (1 << 20)) return WIDE_ERR_INVALID_ARG;
+    free_profile(ctx);
+    ctx->prof = new (std::nothrow) wide_prof_rec[max_records];
+    if (!ctx->prof) return WIDE_ERR_CUDA;
+    for (int i = 0; i < max_records; ++i) {
+        if (cudaEventCreate(&ctx->prof[i].begin) != cudaSuccess || cudaEventCreate(&ctx->prof[i].end) != cudaSuccess)
+            return WIDE_ERR_CUDA;
+        ctx->prof_cap = i + 1;
+    }
+    ctx->prof_used = 0;
+    return WIDE_OK;
+}
+
+int wide_profile_end(wide_ctx* ctx, void* stream, char* buf, size_t buf_bytes) {
+    if (!ctx || !buf || buf_bytes == 0) return WIDE_ERR_INVALID_ARG;
+    buf[0] = 0;
+    if (!ctx->prof) return WIDE_ERR_INVALID_ARG;
+    WIDE_CUDA_CHECK(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    // aggregate by kernel name (names are string literals: compare by pointer, then by text)
+    struct Agg { const char* name; int launches; double ms; };
+    Agg agg[64];
+    int n_agg = 0;
+    for (int i = 0; i < ctx->prof_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ctx->prof[i].begin, ctx->prof[i].end) != cudaSuccess) continue;
+        int j = 0;
+        for (; j < n_agg; ++j)
+            if (agg[j].name == ctx->prof[i].name) break;
+        if (j == n_agg) {
+            if (n_agg == 64) continue;
+            agg[n_agg++] = Agg{ctx->prof[i].name, 0, 0.0};
+        }
+        agg[j].launches += 1;
+        agg[j].ms += ms;
+    }
+    size_t off = 0;
+    for (int j = 0; j < n_agg; ++j) {
+        int w = snprintf(buf + off, buf_bytes - off, "%s,%d,%.6f\n", agg[j].name, agg[j].launches, agg[j].ms);
+        if (w < 0 || static_cast<size_t>(w) >= buf_bytes - off) break;
+        off += static_cast<size_t>(w);
+    }
+    free_profile(ctx);
+    return WIDE_OK;
+}
+
+int wide_launch_count(wide_ctx* ctx, unsigned long long* count) {
+    if (!ctx || !count) return WIDE_ERR_INVALID_ARG;
+    *count = ctx->launches;
+    return WIDE_OK;
+}
+
 int wide_destroy(wide_ctx* ctx) {
     if (!ctx) return WIDE_ERR_INVALID_ARG;
+    free_profile(ctx);
     cudaFree(ctx->d_status);
     delete ctx;
     return WIDE_OK;
@@ -170,7 +238,7 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (path) {
         case PATH_SIMT:
-            return wide_launch_ffn_simt(s, x, w_gate, w_up, w_down, dtype, tokens, hidden, d_ff, group, mask_bits, y,
+            return wide_launch_ffn_simt(ctx, s, x, w_gate, w_up, w_down, dtype, tokens, hidden, d_ff, group, mask_bits, y,
                                         out_dtype, workspace);
         case PATH_PREFILL_TC:
             return wide_launch_ffn_prefill_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
@@ -202,7 +270,7 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (path) {
         case PATH_SIMT:
-            return wide_launch_oproj_simt(s, attn_out, w_o, dtype, tokens, hidden, attn_dim, group, mask_bits, y,
+            return wide_launch_oproj_simt(ctx, s, attn_out, w_o, dtype, tokens, hidden, attn_dim, group, mask_bits, y,
                                           out_dtype);
         case PATH_PREFILL_TC:
             return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
@@ -220,7 +288,7 @@ int wide_unpermute(wide_ctx* ctx, void* stream, const void* src_packed, const in
     if (tokens < 0 || n_groups <= 0 || group <= 0 || (elem_bytes != 2 && elem_bytes != 4)) return WIDE_ERR_INVALID_ARG;
     if ((group * elem_bytes) % 16 != 0) return WIDE_ERR_UNSUPPORTED_SHAPE;
     if (!wide_aligned16(src_packed) || !wide_aligned16(dst)) return WIDE_ERR_ALIGNMENT;
-    return wide_launch_unpermute(static_cast<cudaStream_t>(stream), src_packed, perm, counts, offsets, tokens,
+    return wide_launch_unpermute(ctx, static_cast<cudaStream_t>(stream), src_packed, perm, counts, offsets, tokens,
                                  n_groups, group, elem_bytes, dst);
 }
 

@@ -344,7 +344,10 @@ DecodeWs carve_ws(void* ws, int D, int inner) {
 int launch_stream(wide_ctx* ctx, cudaStream_t s, const CUtensorMap& w0, const CUtensorMap& w1, const CUtensorMap& act,
                   const DecodeMeta* meta, const StreamArgs& a) {
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemD));
-    stream_kernel<<<ctx->sm_count, 192, kSmemD, s>>>(w0, w1, act, meta, a, ctx->d_status, ctx->wait_ns);
+    {
+        WideLaunch l(ctx, s, a.mode == MODE_GATEUP ? "decode_stream_gateup" : "decode_stream_down");
+        stream_kernel<<<ctx->sm_count, 192, kSmemD, s>>>(w0, w1, act, meta, a, ctx->d_status, ctx->wait_ns);
+    }
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -366,8 +369,11 @@ int run_down(wide_ctx* ctx, cudaStream_t s, const DecodeWs& w, const void* act_p
     int rc = launch_stream(ctx, s, tmW, tmW, tmAct, w.meta, a);
     if (rc != WIDE_OK) return rc;
     const long long n = static_cast<long long>(B) * D;
-    finish_kernel<<<static_cast<int>((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, s>>>(
-        w.yacc, n, y, out_dtype == WIDE_BF16 ? 1 : 0);
+    {
+        WideLaunch l(ctx, s, "decode_finish");
+        finish_kernel<<<static_cast<int>((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184), 256, 0, s>>>(
+            w.yacc, n, y, out_dtype == WIDE_BF16 ? 1 : 0);
+    }
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -387,8 +393,11 @@ int wide_launch_ffn_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* x, cons
     DecodeWs w = carve_ws(ws, D, Dff);
     // zero only the accumulator rows that are used: gate/up rows [0,B) and y rows [0,B) -- they are
     // laid out [64, inner] so rows 0..B-1 of each are contiguous; zero the three prefixes.
-    prep_kernel<<<ctx->sm_count, 256, 0, s>>>(mask_bits, B, NG, words, w.meta, reinterpret_cast<float4*>(w.gate),
-                                              static_cast<long long>(w.zero_floats / 4));
+    {
+        WideLaunch l(ctx, s, "decode_prep");
+        prep_kernel<<<ctx->sm_count, 256, 0, s>>>(mask_bits, B, NG, words, w.meta, reinterpret_cast<float4*>(w.gate),
+                                                  static_cast<long long>(w.zero_floats / 4));
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
 
     CUtensorMap tmG, tmU, tmX;
@@ -403,7 +412,10 @@ int wide_launch_ffn_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* x, cons
     int rc = launch_stream(ctx, s, tmG, tmU, tmX, w.meta, a);
     if (rc != WIDE_OK) return rc;
 
-    act_kernel<<<ctx->sm_count * 2, 256, 0, s>>>(w.meta, w.gate, w.up, mask_bits, words, B, Dff, G, w.h);
+    {
+        WideLaunch l(ctx, s, "decode_act");
+        act_kernel<<<ctx->sm_count * 2, 256, 0, s>>>(w.meta, w.gate, w.up, mask_bits, words, B, Dff, G, w.h);
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     return run_down(ctx, s, w, w.h, wd, B, NT, D, Dff, G, y, out_dtype);
 }
@@ -413,12 +425,18 @@ int wide_launch_oproj_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* a_in,
     if (T == 0) return WIDE_OK;
     const int B = T, NT = (B + 15) / 16 * 16, NG = K / G, words = (NG + 31) / 32;
     DecodeWs w = carve_ws(ws, D, K);
-    prep_kernel<<<ctx->sm_count, 256, 0, s>>>(mask_bits, B, NG, words, w.meta, reinterpret_cast<float4*>(w.gate),
-                                              static_cast<long long>(w.zero_floats / 4));
+    {
+        WideLaunch l(ctx, s, "decode_prep");
+        prep_kernel<<<ctx->sm_count, 256, 0, s>>>(mask_bits, B, NG, words, w.meta, reinterpret_cast<float4*>(w.gate),
+                                                  static_cast<long long>(w.zero_floats / 4));
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     const long long total = static_cast<long long>(B) * (K / 8);
-    mask_rows_small_kernel<<<static_cast<int>((total + 255) / 256), 256, 0, s>>>(
-        static_cast<const uint4*>(a_in), mask_bits, words, B, K, G, reinterpret_cast<uint4*>(w.h));
+    {
+        WideLaunch l(ctx, s, "decode_mask_rows");
+        mask_rows_small_kernel<<<static_cast<int>((total + 255) / 256), 256, 0, s>>>(
+            static_cast<const uint4*>(a_in), mask_bits, words, B, K, G, reinterpret_cast<uint4*>(w.h));
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     return run_down(ctx, s, w, w.h, wo, B, NT, D, K, G, y, out_dtype);
 }

@@ -146,10 +146,11 @@ __global__ void __launch_bounds__(256) gemm_nt_kernel(const TIn* __restrict__ A,
 }
 
 template <typename TIn>
-int run_gemm_nt(cudaStream_t s, const TIn* A, const TIn* B, void* C, int out_dtype, int M, int N, int K,
+int run_gemm_nt(wide_ctx* ctx, cudaStream_t s, const TIn* A, const TIn* B, void* C, int out_dtype, int M, int N, int K,
                 const uint32_t* mask_bits, int words, int G) {
     if (M == 0) return WIDE_OK;
     dim3 grid((N + BC - 1) / BC, (M + BT - 1) / BT);
+    WideLaunch l(ctx, s, "simt_gemm_nt");
     if (out_dtype == WIDE_BF16)
         gemm_nt_kernel<TIn, __nv_bfloat16><<<grid, 256, 0, s>>>(A, B, static_cast<__nv_bfloat16*>(C), M, N, K,
                                                                mask_bits, words, G);
@@ -159,35 +160,38 @@ int run_gemm_nt(cudaStream_t s, const TIn* A, const TIn* B, void* C, int out_dty
 }
 
 template <typename TIn>
-int run_ffn(cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd, int T, int D,
+int run_ffn(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd, int T, int D,
             int Dff, int G, const uint32_t* mask_bits, void* y, int out_dtype, void* h) {
     if (T == 0) return WIDE_OK;
     const int words = (Dff / G + 31) / 32;
     dim3 grid((Dff + BC - 1) / BC, (T + BT - 1) / BT);
-    gateup_kernel<TIn><<<grid, 256, 0, s>>>(static_cast<const TIn*>(x), static_cast<const TIn*>(wg),
-                                            static_cast<const TIn*>(wu), T, D, Dff, G, mask_bits, words,
-                                            static_cast<TIn*>(h));
+    {
+        WideLaunch l(ctx, s, "simt_gateup");
+        gateup_kernel<TIn><<<grid, 256, 0, s>>>(static_cast<const TIn*>(x), static_cast<const TIn*>(wg),
+                                                static_cast<const TIn*>(wu), T, D, Dff, G, mask_bits, words,
+                                                static_cast<TIn*>(h));
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
-    return run_gemm_nt<TIn>(s, static_cast<const TIn*>(h), static_cast<const TIn*>(wd), y, out_dtype, T, D, Dff,
+    return run_gemm_nt<TIn>(ctx, s, static_cast<const TIn*>(h), static_cast<const TIn*>(wd), y, out_dtype, T, D, Dff,
                             nullptr, 0, 1);
 }
 
 }  // namespace
 
-int wide_launch_ffn_simt(cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd,
+int wide_launch_ffn_simt(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd,
                          int dtype, int T, int D, int Dff, int G, const uint32_t* mask_bits, void* y,
                          int out_dtype, void* h) {
-    if (dtype == WIDE_BF16) return run_ffn<__nv_bfloat16>(s, x, wg, wu, wd, T, D, Dff, G, mask_bits, y, out_dtype, h);
-    return run_ffn<float>(s, x, wg, wu, wd, T, D, Dff, G, mask_bits, y, out_dtype, h);
+    if (dtype == WIDE_BF16) return run_ffn<__nv_bfloat16>(ctx, s, x, wg, wu, wd, T, D, Dff, G, mask_bits, y, out_dtype, h);
+    return run_ffn<float>(ctx, s, x, wg, wu, wd, T, D, Dff, G, mask_bits, y, out_dtype, h);
 }
 
-int wide_launch_oproj_simt(cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
+int wide_launch_oproj_simt(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
                            int K, int G, const uint32_t* mask_bits, void* y, int out_dtype) {
     const int words = (K / G + 31) / 32;
     if (dtype == WIDE_BF16)
-        return run_gemm_nt<__nv_bfloat16>(s, static_cast<const __nv_bfloat16*>(a),
+        return run_gemm_nt<__nv_bfloat16>(ctx, s, static_cast<const __nv_bfloat16*>(a),
                                           static_cast<const __nv_bfloat16*>(wo), y, out_dtype, T, D, K, mask_bits,
                                           words, G);
-    return run_gemm_nt<float>(s, static_cast<const float*>(a), static_cast<const float*>(wo), y, out_dtype, T, D, K,
+    return run_gemm_nt<float>(ctx, s, static_cast<const float*>(a), static_cast<const float*>(wo), y, out_dtype, T, D, K,
                               mask_bits, words, G);
 }

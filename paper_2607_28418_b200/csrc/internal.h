@@ -8,12 +8,40 @@
 
 #include "wide.h"
 
+struct wide_prof_rec {
+    const char* name;
+    cudaEvent_t begin, end;
+};
+
 struct wide_ctx {
     int device;
     int sm_count;
     int* d_status;          // device status word (WIDE_OK or WIDE_ERR_TIMEOUT)
     unsigned long long wait_ns;  // bound of every device-side wait
     void* encode_tiled;     // cuTensorMapEncodeTiled, resolved through the runtime
+    unsigned long long launches;  // kernels launched by the library so far
+    // optional per-launch timing: a pool of event pairs created by wide_profile_begin
+    wide_prof_rec* prof;
+    int prof_cap, prof_used;
+};
+
+// Counts one kernel launch and, when profiling is on, brackets it with a pair of CUDA events on
+// the launching stream.  Usage: { WideLaunch l(ctx, s, "name"); kernel<<<..., s>>>(...); }
+struct WideLaunch {
+    wide_ctx* ctx;
+    cudaStream_t s;
+    int idx;
+    WideLaunch(wide_ctx* c, cudaStream_t st, const char* name) : ctx(c), s(st), idx(-1) {
+        ++ctx->launches;
+        if (ctx->prof && ctx->prof_used < ctx->prof_cap) {
+            idx = ctx->prof_used++;
+            ctx->prof[idx].name = name;
+            cudaEventRecord(ctx->prof[idx].begin, s);
+        }
+    }
+    ~WideLaunch() {
+        if (idx >= 0) cudaEventRecord(ctx->prof[idx].end, s);
+    }
 };
 
 #define WIDE_CUDA_CHECK(expr)                         \
@@ -51,14 +79,14 @@ int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits
                         int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
                         int32_t* offsets);
 
-int wide_launch_unpermute(cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
+int wide_launch_unpermute(wide_ctx* ctx, cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
                           const int32_t* offsets, int T, int NG, int G, int elem_bytes, void* dst);
 
 // CUDA-core FFN / O-proj (any shape, fp32 or bf16).  `h` is scratch [T, Dff] in `dtype`.
-int wide_launch_ffn_simt(cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd,
+int wide_launch_ffn_simt(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, const void* wd,
                          int dtype, int T, int D, int Dff, int G, const uint32_t* mask_bits, void* y,
                          int out_dtype, void* h);
-int wide_launch_oproj_simt(cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
+int wide_launch_oproj_simt(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
                            int K, int G, const uint32_t* mask_bits, void* y, int out_dtype);
 
 // tcgen05 prefill path (bf16).  `h` is scratch [T, Dff] bf16.

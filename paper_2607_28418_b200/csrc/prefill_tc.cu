@@ -499,6 +499,7 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     const int n_tiles = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
     const int words = (K / G + 31) / 32;
+    WideLaunch l(ctx, s, "prefill_down");
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
@@ -512,6 +513,7 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
     if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
     constexpr int smem = smem_bytes<2 * BN * kBK * 2>();
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    WideLaunch l(ctx, s, "prefill_gateup");
     gateup_kernel<BN><<<ctx->sm_count, 320, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm, counts,
                                                        work_list, n_work, T, D, Dff, G,
                                                        static_cast<__nv_bfloat16*>(h), ctx->d_status, ctx->wait_ns);
@@ -526,7 +528,10 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const int32_t* n_work, void* y, int out_dtype, void* h) {
     if (T == 0) return WIDE_OK;
     // inactive (token, group) pairs of H must read as zero in the down projection
-    WIDE_CUDA_CHECK(cudaMemsetAsync(h, 0, static_cast<size_t>(T) * Dff * 2, s));
+    {
+        WideLaunch l(ctx, s, "prefill_zero_h");
+        WIDE_CUDA_CHECK(cudaMemsetAsync(h, 0, static_cast<size_t>(T) * Dff * 2, s));
+    }
     int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h)
                        : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h);
     if (rc != WIDE_OK) return rc;
@@ -541,8 +546,11 @@ int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, c
     const long long total = static_cast<long long>(T) * (K / 8);
     long long blocks = (total + 255) / 256;
     if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    {
+    WideLaunch l(ctx, s, "prefill_mask_rows");
     mask_rows_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(a), mask_bits, words, T, K, G,
                                                               static_cast<uint4*>(a_masked));
+    }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     return launch_down<256>(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype);
 }

@@ -131,22 +131,26 @@ int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits
                         int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
                         int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
                         int32_t* offsets) {
-    (void)ctx;
     const int words = (NG + 31) / 32;
     const int n_tiles = (T + tile_m - 1) / tile_m;
-    partition_kernel<<<NG, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts);
+    {
+        WideLaunch l(ctx, s, "reorder_partition");
+        partition_kernel<<<NG, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts);
+    }
+    WideLaunch l(ctx, s, "reorder_metadata");
     metadata_kernel<<<1, 256, 0, s>>>(counts, T, NG, tile_m, n_tiles, tile_map, work_list, n_work,
                                       union_list, n_union, offsets);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
-int wide_launch_unpermute(cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
+int wide_launch_unpermute(wide_ctx* ctx, cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
                           const int32_t* offsets, int T, int NG, int G, int elem_bytes, void* dst) {
     const int vec_per_group = G * elem_bytes / 16;
     const long long total = static_cast<long long>(NG) * T * vec_per_group;
     if (total == 0) return WIDE_OK;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
+    WideLaunch l(ctx, s, "unpermute");
     unpermute_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(src), perm, counts, offsets,
                                                               T, NG, vec_per_group, static_cast<uint4*>(dst));
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;

@@ -105,9 +105,10 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 }
 
 template <typename TA, typename TB>
-void launch_gemm_f64(cudaStream_t s, const TA* A, const TB* B, double* C, int M, int N, int K,
+void launch_gemm_f64(wide_ctx* ctx, cudaStream_t s, const TA* A, const TB* B, double* C, int M, int N, int K,
                      long long sbk, long long sbn) {
     dim3 grid((N + kTile - 1) / kTile, (M + kTile - 1) / kTile);
+    WideLaunch l(ctx, s, "route_scores_f64");
     gemm_f64_kernel<TA, TB><<<grid, 256, 0, s>>>(A, B, C, M, N, K, sbk, sbn);
 }
 
@@ -122,7 +123,6 @@ size_t wide_route_workspace(int T, int NG, int rank) {
 int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
                       const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws) {
-    (void)ctx;
     if (T == 0) return WIDE_OK;
     double* sc = static_cast<double*>(ws);
     double* u = reinterpret_cast<double*>(static_cast<char*>(ws) +
@@ -130,25 +130,27 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
     const int sel_blocks = (T + 7) / 8;
     if (mode == WIDE_ROUTE_TOPK) {
         if (dtype == WIDE_BF16)
-            launch_gemm_f64(s, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
+            launch_gemm_f64(ctx, s, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
                             sc, T, NG, D, 1LL, static_cast<long long>(D));
         else
-            launch_gemm_f64(s, static_cast<const float*>(x), static_cast<const float*>(w_router), sc, T, NG,
+            launch_gemm_f64(ctx, s, static_cast<const float*>(x), static_cast<const float*>(w_router), sc, T, NG,
                             D, 1LL, static_cast<long long>(D));
+        WideLaunch l(ctx, s, "route_topk_select");
         topk_select_kernel<<<sel_blocks, 256, 0, s>>>(sc, T, NG, k, k_per_token, mask_bits, scores);
     } else {
         // u = x W1 (W1 [D, rank]),  l = u W2 (W2 [rank, 2NG])
         if (dtype == WIDE_BF16) {
-            launch_gemm_f64(s, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
+            launch_gemm_f64(ctx, s, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
                             u, T, rank, D, static_cast<long long>(rank), 1LL);
-            launch_gemm_f64(s, u, static_cast<const __nv_bfloat16*>(w2), sc, T, 2 * NG, rank,
+            launch_gemm_f64(ctx, s, u, static_cast<const __nv_bfloat16*>(w2), sc, T, 2 * NG, rank,
                             static_cast<long long>(2 * NG), 1LL);
         } else {
-            launch_gemm_f64(s, static_cast<const float*>(x), static_cast<const float*>(w_router), u, T, rank,
+            launch_gemm_f64(ctx, s, static_cast<const float*>(x), static_cast<const float*>(w_router), u, T, rank,
                             D, static_cast<long long>(rank), 1LL);
-            launch_gemm_f64(s, u, static_cast<const float*>(w2), sc, T, 2 * NG, rank,
+            launch_gemm_f64(ctx, s, u, static_cast<const float*>(w2), sc, T, 2 * NG, rank,
                             static_cast<long long>(2 * NG), 1LL);
         }
+        WideLaunch l(ctx, s, "route_pair_select");
         pair_select_kernel<<<sel_blocks, 256, 0, s>>>(sc, T, NG, mask_bits, scores);
     }
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;

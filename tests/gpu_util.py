@@ -9,10 +9,8 @@ REL_TOL = 2e-2  # max |err| <= REL_TOL * max |ref|  (bf16 inputs, fp32 accumulat
 
 def to_dev(a: np.ndarray, dtype: str) -> torch.Tensor:
     """float32 host array -> CUDA tensor of the workload dtype (exact for bf16-rounded inputs)."""
-    if dtype == "bf16":
-        bits = synth.to_bf16_bits(a)
-        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    from paper_2607_28418_b200 import binding
+    return binding.upload(a, dtype)
 
 
 def bits_to_dev(bits: np.ndarray) -> torch.Tensor:

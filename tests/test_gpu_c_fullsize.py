@@ -1,0 +1,101 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+Integer stages (mask, permutation, tile map) are compared in full and bit-exact.  Float outputs
+are compared on sampled token rows: an output row depends only on its own token and mask row
+(Eq. 3 / Eq. 2), so the oracle can compute any row by itself.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import wide_oracle as wo
+from paper_2607_28418_b200 import synth
+from tests.gpu_util import REL_TOL, bits_to_host, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2607_28418_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.status() == 0
+    c.close()
+
+
+def _chain(ctx, cfg, seed, n_sample=48):
+    from paper_2607_28418_b200 import binding
+    case = synth.make_ffn_case(cfg, seed)
+    d = {k: to_dev(v, cfg.dtype) for k, v in case.items()}
+    NG, T = cfg.n_groups, cfg.tokens
+    bits, _ = binding.wide_route(ctx, d["x"], d["w_router"], NG, cfg.k)
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router"]), cfg.k)
+    assert (bits_to_host(bits) == wo.pack_mask_bits(mask)).all(), "mask bits differ"
+    meta = None
+    if T > 64:
+        meta = binding.wide_reorder(ctx, bits, NG, 128)
+        ref = wo.reorder(mask, 128)
+        assert (meta["perm"].cpu().numpy() == ref["perm"]).all()
+        assert (meta["counts"].cpu().numpy() == ref["counts"]).all()
+        assert (meta["tile_map"].cpu().numpy() == ref["tile_map"]).all()
+        nw = int(meta["n_work"].item())
+        assert nw == ref["n_work"] and (meta["work_list"].cpu().numpy()[:nw] == ref["work_list"]).all()
+        assert (meta["offsets"].cpu().numpy() == ref["offsets"]).all()
+    y = binding.wide_ffn(ctx, d["x"], d["w_gate"], d["w_up"], d["w_down"], cfg.group, bits, meta)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    rows = np.unique(np.concatenate([np.array([0, T - 1]),
+                                     np.random.default_rng(seed).integers(0, T, size=min(n_sample, T))]))
+    y_ref = wo.ffn(case["x"][rows], case["w_gate"], case["w_up"], case["w_down"], mask[rows], cfg.group)
+    got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    scale = np.abs(y_ref).max()
+    err = np.abs(got - y_ref).max()
+    assert np.isfinite(y.float()).all().item()
+    assert err <= REL_TOL * scale, f"{cfg.name}: max|err| {err:.3e} vs {REL_TOL} * {scale:.3e}"
+    return err / scale
+
+
+def test_llama7b_prefill_chain(ctx):
+    rel = _chain(ctx, synth.CONFIGS["llama7b_prefill"], 0)
+    print("llama7b_prefill rel err", rel)
+
+
+@pytest.mark.parametrize("B,seed", [(1, 0), (8, 1), (32, 2), (64, 3)])
+def test_llama8b_decode_chain(ctx, B, seed):
+    cfg = synth.CONFIGS["llama8b_decode"].with_(tokens=B, router="clustered" if seed % 2 else "random")
+    _chain(ctx, cfg, seed)
+
+
+@pytest.mark.parametrize("G,p,router", [(64, 0.25, "random"), (256, 0.75, "clustered"), (128, 0.5, "clustered_corr")])
+def test_sweep_points_prefill(ctx, G, p, router):
+    _chain(ctx, synth.sweep_point(4096, G, p, router), 4, n_sample=32)
+
+
+def test_sweep_point_decode_batch16(ctx):
+    _chain(ctx, synth.sweep_point(16, 128, 0.25, "clustered"), 5)
+
+
+def test_llama13b_layer_oproj_and_ffn(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.CONFIGS["llama13b_layer"]
+    case = synth.make_oproj_case(cfg, 0)
+    NG, G, T = cfg.attn_n_groups, cfg.attn_group, cfg.tokens
+    d = {k: to_dev(v, cfg.dtype) for k, v in case.items()}
+    bits, _ = binding.wide_route(ctx, d["x"], d["w_router_attn"], NG, cfg.attn_k)
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router_attn"]), cfg.attn_k)
+    assert (bits_to_host(bits) == wo.pack_mask_bits(mask)).all()
+    meta = binding.wide_reorder(ctx, bits, NG, 128)
+    assert (meta["perm"].cpu().numpy() == wo.reorder(mask, 128)["perm"]).all()
+    y = binding.wide_oproj(ctx, d["attn_out"], d["w_o"], G, bits, meta)
+    rows = np.random.default_rng(0).integers(0, T, size=64)
+    y_ref = wo.oproj(case["attn_out"][rows], case["w_o"], mask[rows], G)
+    got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert np.abs(got - y_ref).max() <= REL_TOL * np.abs(y_ref).max()
+    # decode batch 32 of the same layer
+    y32 = binding.wide_oproj(ctx, d["attn_out"][:32].contiguous(), d["w_o"], G, bits[:32].contiguous(), None)
+    y_ref = wo.oproj(case["attn_out"][:32], case["w_o"], mask[:32], G)
+    assert np.abs(y32.float().cpu().numpy() - y_ref).max() <= REL_TOL * np.abs(y_ref).max()
+    assert ctx.status() == 0
+    # FFN half of the layer, prefill
+    _chain(ctx, cfg, 1, n_sample=32)
