@@ -51,7 +51,7 @@ def _chain(ctx, cfg, seed, n_sample=48):
     got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
     scale = np.abs(y_ref).max()
     err = np.abs(got - y_ref).max()
-    assert np.isfinite(y.float()).all().item()
+    assert torch.isfinite(y.float()).all().item()
     assert err <= REL_TOL * scale, f"{cfg.name}: max|err| {err:.3e} vs {REL_TOL} * {scale:.3e}"
     return err / scale
 
