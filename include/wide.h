@@ -135,6 +135,30 @@ WIDE_API int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, i
                size_t workspace_bytes, unsigned flags);
 
 /*
+ * wide_route_static -- (no counterpart in the paper; a deployment variant of wide_route.)
+ * Same arguments, results and errors as wide_route, minus the workspace: the fp64 score buffer is
+ * a fixed array inside the library's device image.  It exists for hosts that may not allocate
+ * device memory where they route -- a serving process whose own pool owns the whole heap, a
+ * plugin called under another framework's allocator lock, a deployment that forbids cudaMalloc
+ * after start-up.  The call itself allocates nothing on host or device.
+ *   - Limit: wide_workspace_bytes(WIDE_OP_ROUTE, ...) for a rank-64 router, i.e.
+ *     tokens * (2 * n_groups + 64) * 8 bytes rounded up to 256-byte pieces, must not exceed
+ *     WIDE_ROUTE_STATIC_BYTES (2 MiB: e.g. 1100 tokens x 86 groups, 450 x 256); larger problems
+ *     return WIDE_ERR_WORKSPACE and launch nothing.  Every GPU on which the library is loaded
+ *     holds those 2 MiB until the process exits.
+ *   - The first call on a device looks up the array's device address; it must be made with
+ *     ctx's device current (else WIDE_ERR_INVALID_ARG) and should come before any stream
+ *     capture.  Later calls reuse the cached address.
+ *   - All calls on a device share the one array.  Nothing in it needs clearing between calls
+ *     (each call overwrites what it reads), but two calls that overlap on the GPU -- different
+ *     streams, or different contexts of the same device -- race on it: serialise them.
+ */
+#define WIDE_ROUTE_STATIC_BYTES (2u << 20)
+WIDE_API int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens, int hidden,
+                               const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
+                               const int32_t* k_per_token, uint32_t* mask_bits, float* scores, unsigned flags);
+
+/*
  * wide_reorder -- mask reordering, Eq. 6 / Algorithm 1, and the level-0 predicate of Eq. 7-8.
  * For each group g the rows are sorted by mask value, descending and STABLE (active rows in
  * ascending token order, then inactive rows in ascending token order).

@@ -26,7 +26,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, 
 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
            "wide_profile_end", "wide_launch_count", "wide_strerror",
-           "wide_version", "wide_workspace_bytes", "wide_route", "wide_reorder", "wide_ffn",
+           "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_ffn",
            "wide_oproj", "wide_unpermute"]
 
 _c_void_p, _c_int, _c_size_t, _c_uint = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
@@ -65,6 +65,7 @@ def load_library() -> ctypes.CDLL:
     lib.wide_route.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p,
                                _c_int, _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                                _c_size_t, _c_uint]
+    lib.wide_route_static.argtypes = lib.wide_route.argtypes[:15] + [_c_uint]
     lib.wide_reorder.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int] + [_c_void_p] * 8
     lib.wide_ffn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int,
                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
@@ -205,6 +206,26 @@ def wide_route(ctx: Context, x: torch.Tensor, w_router: torch.Tensor, n_groups: 
                             n_groups, mode, k, _ptr(k_per_token), _ptr(mask_bits), _ptr(scores), _ptr(ws),
                             ws.numel(), flags)
     _check(rc, "wide_route")
+    return mask_bits, scores
+
+
+ROUTE_STATIC_BYTES = 2 << 20
+
+
+def wide_route_static(ctx: Context, x: torch.Tensor, w_router: torch.Tensor, n_groups: int, k: int = 0,
+                      mode: int = ROUTE_TOPK, w2: Optional[torch.Tensor] = None, rank: int = 0,
+                      k_per_token: Optional[torch.Tensor] = None, scores: Optional[torch.Tensor] = None,
+                      mask_bits: Optional[torch.Tensor] = None, flags: int = 0):
+    """wide_route for callers that may not allocate: scratch is the library's fixed device array
+    (problems beyond ROUTE_STATIC_BYTES of scratch are refused with ERR_WORKSPACE).  Pass
+    preallocated ``mask_bits`` (and ``scores``) to keep the whole call allocation-free; calls that
+    overlap on the GPU share the array and must be serialised by the caller."""
+    T, D = x.shape
+    if mask_bits is None:
+        mask_bits = torch.empty((T, (n_groups + 31) // 32), dtype=torch.int32, device=x.device)
+    rc = ctx.lib.wide_route_static(ctx.handle, _stream(), _ptr(x), _dtype_code(x), T, D, _ptr(w_router), _ptr(w2),
+                                   rank, n_groups, mode, k, _ptr(k_per_token), _ptr(mask_bits), _ptr(scores), flags)
+    _check(rc, "wide_route_static")
     return mask_bits, scores
 
 

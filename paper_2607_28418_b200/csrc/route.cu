@@ -155,3 +155,67 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
     }
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------------------------------------
+// wide_route_static: the same routing as wide_route, for callers that cannot provide scratch.
+//
+// Some hosts of this library are not allowed to allocate device memory at the point where they
+// route: a serving loop that has handed the whole device heap to its own pool, a plugin that runs
+// inside another framework's allocator lock, or code running under a policy that forbids
+// cudaMalloc after start-up.  For them the fp64 score buffer lives in a file-scope device array of
+// fixed size instead of a caller-supplied workspace.  Every GPU that loads the library holds these
+// WIDE_ROUTE_STATIC_BYTES until the process exits.
+//
+// In host code the array's name is only a handle for the runtime, not a device address, so the
+// address is resolved once per device with cudaGetSymbolAddress while that device is current and
+// cached; kernels only ever see the resolved pointer.
+static __device__ __align__(256) unsigned char g_route_static_scratch[WIDE_ROUTE_STATIC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Returns the device address of the static scratch for `device`, resolving it on first use.
+// The first use must happen with `device` current and outside stream capture.
+int static_scratch_for(int device, void** out) {
+    if (device < 0 || device >= kMaxDevices) return WIDE_ERR_INVALID_ARG;
+    if (!g_static_ptr[device]) {
+        int cur = -1;
+        if (cudaGetDevice(&cur) != cudaSuccess) return WIDE_ERR_CUDA;
+        if (cur != device) return WIDE_ERR_INVALID_ARG;
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_route_static_scratch) != cudaSuccess || !p) return WIDE_ERR_CUDA;
+        g_static_ptr[device] = p;
+    }
+    *out = g_static_ptr[device];
+    return WIDE_OK;
+}
+}  // namespace
+
+extern "C" int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens, int hidden,
+                                 const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
+                                 const int32_t* k_per_token, uint32_t* mask_bits, float* scores, unsigned flags) {
+    (void)flags;
+    if (!ctx || !x || !w_router || !mask_bits || (dtype != WIDE_BF16 && dtype != WIDE_F32)) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || n_groups <= 0) return WIDE_ERR_INVALID_ARG;
+    if (mode == WIDE_ROUTE_TOPK) {
+        if (w2 || rank != 0) return WIDE_ERR_INVALID_ARG;
+        if (!k_per_token && (k < 0 || k > n_groups)) return WIDE_ERR_INVALID_ARG;
+    } else if (mode == WIDE_ROUTE_PAIR_ARGMAX) {
+        if (!w2 || rank <= 0 || rank > 64) return WIDE_ERR_INVALID_ARG;
+    } else {
+        return WIDE_ERR_INVALID_ARG;
+    }
+    if (n_groups > WIDE_MAX_GROUPS || hidden % 8 != 0) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(x) || !wide_aligned16(w_router) || (w2 && !wide_aligned16(w2))) return WIDE_ERR_ALIGNMENT;
+    // the fixed array bounds the problem size: say so instead of overrunning it
+    if (wide_route_workspace(tokens, n_groups, rank) > static_cast<size_t>(WIDE_ROUTE_STATIC_BYTES))
+        return WIDE_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const int rc = static_scratch_for(ctx->device, &scratch);
+    if (rc != WIDE_OK) return rc;
+    // every byte of the scratch that a call reads is written by that call first, so nothing has to
+    // be cleared between calls
+    return wide_launch_route(ctx, static_cast<cudaStream_t>(stream), x, dtype, tokens, hidden, w_router, w2, rank,
+                             n_groups, mode, k, k_per_token, mask_bits, scores, scratch);
+}
