@@ -121,8 +121,10 @@ WIDE_API size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, 
  *                                w2 = W2 [rank, 2*n_groups]; token t executes group g iff
  *                                l[t,2g] >= l[t,2g+1] (class 0 = execute, first index wins ties).
  *
- * The selection is decided on fp64 sums of the exact input products, so it does not depend on
- * summation order.
+ * The selection equals the one taken on fp64 sums of the exact input products, so it does not
+ * depend on summation order.  (bf16, TOPK, hidden % 64 == 0: scores come from the tensor cores in
+ * fp32 and every group closer to the selection boundary than a proven error bound is re-scored
+ * exactly in fp64; other cases, and WIDE_FLAG_SIMT, compute all scores in fp64.)
  *   x          [tokens, hidden]  dtype
  *   mask_bits  out uint32 [tokens, W]
  *   scores     out fp32 [tokens, n_groups] (TOPK) or [tokens, 2*n_groups] (PAIR), may be NULL
@@ -141,9 +143,9 @@ WIDE_API int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, i
  * device memory where they route -- a serving process whose own pool owns the whole heap, a
  * plugin called under another framework's allocator lock, a deployment that forbids cudaMalloc
  * after start-up.  The call itself allocates nothing on host or device.
- *   - Limit: wide_workspace_bytes(WIDE_OP_ROUTE, ...) for a rank-64 router, i.e.
- *     tokens * (2 * n_groups + 64) * 8 bytes rounded up to 256-byte pieces, must not exceed
- *     WIDE_ROUTE_STATIC_BYTES (2 MiB: e.g. 1100 tokens x 86 groups, 450 x 256); larger problems
+ *   - Limit: the scratch the call needs, about tokens * (16 * n_groups + 8 * max(rank, 1) + 128)
+ *     bytes plus 1 KiB (wide_workspace_bytes(WIDE_OP_ROUTE, ...) is an upper bound), must not
+ *     exceed WIDE_ROUTE_STATIC_BYTES (2 MiB: e.g. 1300 tokens x 86 groups, 490 x 256); larger problems
  *     return WIDE_ERR_WORKSPACE and launch nothing.  Every GPU on which the library is loaded
  *     holds those 2 MiB until the process exits.
  *   - The first call on a device looks up the array's device address; it must be made with

@@ -187,7 +187,6 @@ int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens
                const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
                const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* workspace,
                size_t workspace_bytes, unsigned flags) {
-    (void)flags;
     if (!ctx || !x || !w_router || !mask_bits || !valid_dtype(dtype)) return WIDE_ERR_INVALID_ARG;
     if (tokens < 0 || hidden <= 0 || n_groups <= 0) return WIDE_ERR_INVALID_ARG;
     if (mode == WIDE_ROUTE_TOPK) {
@@ -203,7 +202,7 @@ int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens
         return WIDE_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < wide_route_workspace(tokens, n_groups, rank)) return WIDE_ERR_WORKSPACE;
     return wide_launch_route(ctx, static_cast<cudaStream_t>(stream), x, dtype, tokens, hidden, w_router, w2, rank,
-                             n_groups, mode, k, k_per_token, mask_bits, scores, workspace);
+                             n_groups, mode, k, k_per_token, mask_bits, scores, workspace, flags);
 }
 
 int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,

@@ -71,7 +71,7 @@ __device__ __forceinline__ bool wide_mask_bit(const uint32_t* mask_bits, int wor
 // ---- launchers (each returns WIDE_OK or WIDE_ERR_CUDA; arguments already validated)
 int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
-                      const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws);
+                      const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws, unsigned flags);
 size_t wide_route_workspace(int T, int NG, int rank);
 
 int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
@@ -95,6 +95,8 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
                                const int32_t* work_list, const int32_t* n_work, void* y,
                                int out_dtype, void* h);
+int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
+                          int ld, int D, float* scores);
 // `a_masked` is scratch [T, K] bf16.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                  int D, int K, int G, const uint32_t* mask_bits, void* y,

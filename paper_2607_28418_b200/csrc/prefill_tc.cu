@@ -278,14 +278,13 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
               int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = 2 * BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
-    constexpr int kLag = 2;  // gather warps signal stage (it - kLag) after issuing stage it
     extern __shared__ uint8_t smem_raw[];
     SmemLayout L = carve_smem<kBBytes>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(L.full + 8 * s, 1 + 4);  // TMA producer + 4 gather warps
+            mbar_init(L.full + 8 * s, 1 + 128);  // TMA producer + one arrival per gather thread
             mbar_init(L.empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -347,6 +346,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
                     if (!mbar_wait(L.full + 8 * s, ph, wait_ns, L.abort_flag)) { ok = false; break; }
+                    fence_proxy_async_smem();  // the A rows were written through the generic proxy (cp.async)
                     tc_fence_after_sync();
                     const uint32_t a_addr = smem_u32(L.stage_base + s * kStageBytes);
                     const uint64_t adesc = umma_desc_sw128(a_addr);
@@ -362,11 +362,13 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ A gather (warps 2..5)
+        // Each thread copies its row's 128 bytes with eight 16-byte cp.async and lets the stage's
+        // mbarrier count an arrival when they have landed; nothing waits on the issuing side, so
+        // the gather runs as far ahead as the ring allows.
         const int r = (warp - 2) * 32 + lane;  // tile row owned by this thread
         const uint32_t row_off = static_cast<uint32_t>(r) * 128u;
         const uint32_t sw = static_cast<uint32_t>(r & 7);
-        int it = 0;        // stages issued
-        int signalled = 0; // stages whose arrival has been posted
+        int it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int pair = item / nsub;
@@ -383,26 +385,11 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                 const uint8_t* p = src + static_cast<size_t>(k) * (kBK * 2);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) cp_async_16(a_dst + ((static_cast<uint32_t>(c) ^ sw) << 4), p + 16 * c);
-                cp_async_commit();
-                if (it - signalled >= kLag) {
-                    cp_async_wait<kLag>();
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(L.full + 8 * (signalled % kStages));
-                    ++signalled;
-                }
+                cp_async_mbar_arrive_noinc(L.full + 8 * s);
             }
         }
-        // drain: everything issued has landed; post the remaining arrivals
-        cp_async_wait<0>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (ok) {
-            for (; signalled < it; ++signalled)
-                if (lane == 0) mbar_arrive(L.full + 8 * (signalled % kStages));
-        } else if (lane == 0) {
-            report_timeout(status);
-        }
+        cp_async_wait_all();
+        if (!ok && lane == 0) report_timeout(status);
     } else {
         // ------------------------------------------------------------------ epilogue (warps 6..9)
         const int q = warp & 3;
@@ -491,15 +478,16 @@ bool make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uin
 
 template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
-                int N, int K, int G, void* Y, int out_dtype) {
+                int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down") {
     CUtensorMap tmA, tmB;
-    if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, N, K, BN)) return WIDE_ERR_CUDA;
+    if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
+    if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
     constexpr int smem = smem_bytes<BN * kBK * 2>();
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int n_tiles = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
     const int words = (K / G + 31) / 32;
-    WideLaunch l(ctx, s, "prefill_down");
+    WideLaunch l(ctx, s, name);
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
@@ -553,4 +541,14 @@ int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, c
     }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     return launch_down<256>(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype);
+}
+
+// scores[T, ld] (fp32) = x[T, D] * w_router[NG, D]^T on the tensor cores; ld = NG rounded up to 32,
+// columns >= NG are written as zeros (weight rows past NG are zero-filled by the TMA).
+int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
+                          int ld, int D, float* scores) {
+    if (T == 0) return WIDE_OK;
+    if (ld <= 128)
+        return launch_down<128>(ctx, s, x, w_router, nullptr, T, ld, D, D, scores, WIDE_F32, NG, "route_scores_tc");
+    return launch_down<256>(ctx, s, x, w_router, nullptr, T, ld, D, D, scores, WIDE_F32, NG, "route_scores_tc");
 }

@@ -104,6 +104,189 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
     }
 }
 
+
+// ---------------------------------------------------------------------------- fast path (bf16)
+// Scores come from the tensor cores in fp32 (exact products, fp32 accumulation).  Their error is
+// bounded by eps_t = kAccumErr * D * ||x_t|| * max_g ||w_g|| (Cauchy-Schwarz on the sum of absolute
+// products times a per-step accumulation error).  A group whose fp32 score is further than
+// 2*eps_t from the selection boundary keeps its fp32 decision; the few groups inside that band
+// get their score recomputed exactly in fp64, and the band is re-ranked on those exact values.
+// The result equals the fp64 decision of the slow path.
+constexpr float kAccumErr = 5.9604645e-8f;  // 2^-24 per accumulated element
+
+// ||w_g||_2 for every group, one warp per group.
+__global__ void __launch_bounds__(256) wnorm_kernel(const __nv_bfloat16* __restrict__ w, int NG, int D,
+                                                    float* __restrict__ wnorm) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.x * 8 + warp;
+    if (g >= NG) return;
+    const uint4* row = reinterpret_cast<const uint4*>(w + static_cast<size_t>(g) * D);
+    float acc = 0.f;
+    for (int i = lane; i < D / 8; i += 32) {
+        const uint4 v = row[i];
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) wnorm[g] = sqrtf(acc) * 1.0001f;  // rounded up a little: it feeds a bound
+}
+
+// Exact x_t . w_g in fp64 by one warp (bf16 products are exact in fp64).
+__device__ __forceinline__ double warp_dot_f64(const __nv_bfloat16* __restrict__ xrow,
+                                               const __nv_bfloat16* __restrict__ wrow, int D, int lane) {
+    const uint4* xv = reinterpret_cast<const uint4*>(xrow);
+    const uint4* wv = reinterpret_cast<const uint4*>(wrow);
+    double acc = 0.0;
+    for (int i = lane; i < D / 8; i += 32) {
+        const uint4 a = xv[i], b = wv[i];
+        const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+        const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 fa = __bfloat1622float2(ah[e]), fb = __bfloat1622float2(bh[e]);
+            acc = fma(static_cast<double>(fa.x), static_cast<double>(fb.x), acc);
+            acc = fma(static_cast<double>(fa.y), static_cast<double>(fb.y), acc);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
+
+// One warp per token.
+__global__ void __launch_bounds__(256) select_band_kernel(const float* __restrict__ scores, int ld,
+                                                          const __nv_bfloat16* __restrict__ x,
+                                                          const __nv_bfloat16* __restrict__ w,
+                                                          const float* __restrict__ wnorm, int T, int NG, int D,
+                                                          int k, const int32_t* __restrict__ k_per_token,
+                                                          uint32_t* __restrict__ mask_bits,
+                                                          float* __restrict__ scores_out) {
+    __shared__ float sh_s[8][WIDE_MAX_GROUPS];
+    __shared__ double sh_e[8][WIDE_MAX_GROUPS];
+    __shared__ float sh_b[8][2];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 8 + warp;
+    if (t >= T) return;
+    float* s = sh_s[warp];
+    double* ex = sh_e[warp];
+    const int words = (NG + 31) >> 5;
+    float wmax = 0.f;
+    for (int g = lane; g < NG; g += 32) {
+        const float v = scores[static_cast<size_t>(t) * ld + g];
+        s[g] = v;
+        wmax = fmaxf(wmax, wnorm[g]);
+        if (scores_out) scores_out[static_cast<size_t>(t) * NG + g] = v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+    __syncwarp();
+    const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
+    const __nv_bfloat16* xrow = x + static_cast<size_t>(t) * D;
+
+    // fp32 ranks; remember the k-th and (k+1)-th largest
+    int rank[WIDE_MAX_GROUPS / 32];
+    if (lane == 0) { sh_b[warp][0] = 0.f; sh_b[warp][1] = 0.f; }
+    __syncwarp();
+#pragma unroll
+    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
+        rank[w8] = NG;
+        const int g = w8 * 32 + lane;
+        if (w8 < words && g < NG) {
+            const float v = s[g];
+            int beats = 0;
+            for (int h = 0; h < NG; ++h) {
+                const float u = s[h];
+                beats += (u > v) || (u == v && h < g);
+            }
+            rank[w8] = beats;
+            if (beats == kt - 1) sh_b[warp][0] = v;
+            if (beats == kt) sh_b[warp][1] = v;
+        }
+    }
+    __syncwarp();
+    const bool boundary = kt > 0 && kt < NG;
+    const float v_k = sh_b[warp][0], v_k1 = sh_b[warp][1];
+
+    float tau = 0.f;
+    if (boundary) {
+        // ||x_t||, then the band half-width 2*eps
+        float acc = 0.f;
+        const uint4* xv = reinterpret_cast<const uint4*>(xrow);
+        for (int i = lane; i < D / 8; i += 32) {
+            const uint4 a = xv[i];
+            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(ah[e]);
+                acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        tau = 2.f * kAccumErr * static_cast<float>(D) * sqrtf(acc) * 1.0001f * wmax;
+    }
+
+    // band membership, exact scores of the band
+    unsigned in_band[WIDE_MAX_GROUPS / 32];
+    int m_hi = 0;  // band members currently ranked inside the top k
+#pragma unroll
+    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
+        in_band[w8] = 0u;
+        if (w8 >= words) continue;
+        const int g = w8 * 32 + lane;
+        bool u = false, hi = false;
+        if (boundary && g < NG) {
+            hi = rank[w8] < kt;
+            u = hi ? (s[g] - v_k1 <= tau) : (v_k - s[g] <= tau);
+        }
+        unsigned vote = __ballot_sync(0xffffffffu, u);
+        in_band[w8] = vote;
+        m_hi += __popc(__ballot_sync(0xffffffffu, u && hi));
+        while (vote) {
+            const int b = __ffs(vote) - 1;
+            vote &= vote - 1;
+            const int gg = w8 * 32 + b;
+            const double e = warp_dot_f64(xrow, w + static_cast<size_t>(gg) * D, D, lane);
+            if (lane == 0) ex[gg] = e;
+        }
+    }
+    __syncwarp();
+
+    // final decision
+#pragma unroll
+    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
+        if (w8 >= words) continue;
+        const int g = w8 * 32 + lane;
+        bool sel = false;
+        if (g < NG) {
+            if ((in_band[w8] >> lane) & 1u) {
+                const double v = ex[g];
+                int beats = 0;
+                for (int w2 = 0; w2 < words; ++w2) {
+                    unsigned bits = in_band[w2];
+                    while (bits) {
+                        const int b = __ffs(bits) - 1;
+                        bits &= bits - 1;
+                        const int h = w2 * 32 + b;
+                        const double u = ex[h];
+                        beats += (u > v) || (u == v && h < g);
+                    }
+                }
+                sel = beats < m_hi;
+            } else {
+                sel = rank[w8] < kt;
+            }
+        }
+        const unsigned word = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) mask_bits[static_cast<size_t>(t) * words + w8] = word;
+    }
+}
+
 template <typename TA, typename TB>
 void launch_gemm_f64(wide_ctx* ctx, cudaStream_t s, const TA* A, const TB* B, double* C, int M, int N, int K,
                      long long sbk, long long sbn) {
@@ -115,15 +298,35 @@ void launch_gemm_f64(wide_ctx* ctx, cudaStream_t s, const TA* A, const TB* B, do
 }  // namespace
 
 size_t wide_route_workspace(int T, int NG, int rank) {
-    // fp64 scores [T, NG] (TOPK) or logits [T, 2NG] plus bottleneck activations [T, rank] (PAIR)
+    // fp64 scores [T, NG] (TOPK) or logits [T, 2NG] plus bottleneck activations [T, rank] (PAIR);
+    // the tensor-core path reuses the first part for fp32 scores [T, roundup(NG, 32)] and keeps
+    // the group norms in the tail
     return wide_align_up(static_cast<size_t>(T) * 2 * NG * sizeof(double), 256) +
-           wide_align_up(static_cast<size_t>(T) * (rank > 0 ? rank : 1) * sizeof(double), 256);
+           wide_align_up(static_cast<size_t>(T) * (rank > 0 ? rank : 1) * sizeof(double), 256) +
+           wide_align_up(static_cast<size_t>(T) * 128, 256) + 1024;
 }
 
 int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
-                      const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws) {
+                      const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws, unsigned flags) {
     if (T == 0) return WIDE_OK;
+    if (mode == WIDE_ROUTE_TOPK && dtype == WIDE_BF16 && D % 64 == 0 && ctx->encode_tiled &&
+        !(flags & WIDE_FLAG_SIMT)) {
+        const int ld = (NG + 31) / 32 * 32;
+        float* sc32 = static_cast<float*>(ws);
+        float* wn = reinterpret_cast<float*>(static_cast<char*>(ws) + wide_route_workspace(T, NG, rank) - 1024);
+        {
+            WideLaunch l(ctx, s, "route_wnorm");
+            wnorm_kernel<<<(NG + 7) / 8, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(w_router), NG, D, wn);
+        }
+        const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32);
+        if (rc != WIDE_OK) return rc;
+        WideLaunch l(ctx, s, "route_select_band");
+        select_band_kernel<<<(T + 7) / 8, 256, 0, s>>>(sc32, ld, static_cast<const __nv_bfloat16*>(x),
+                                                       static_cast<const __nv_bfloat16*>(w_router), wn, T, NG, D, k,
+                                                       k_per_token, mask_bits, scores);
+        return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+    }
     double* sc = static_cast<double*>(ws);
     double* u = reinterpret_cast<double*>(static_cast<char*>(ws) +
                                           wide_align_up(static_cast<size_t>(T) * 2 * NG * sizeof(double), 256));
@@ -195,7 +398,6 @@ int static_scratch_for(int device, void** out) {
 extern "C" int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens, int hidden,
                                  const void* w_router, const void* w2, int rank, int n_groups, int mode, int k,
                                  const int32_t* k_per_token, uint32_t* mask_bits, float* scores, unsigned flags) {
-    (void)flags;
     if (!ctx || !x || !w_router || !mask_bits || (dtype != WIDE_BF16 && dtype != WIDE_F32)) return WIDE_ERR_INVALID_ARG;
     if (tokens < 0 || hidden <= 0 || n_groups <= 0) return WIDE_ERR_INVALID_ARG;
     if (mode == WIDE_ROUTE_TOPK) {
@@ -217,5 +419,5 @@ extern "C" int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int
     // every byte of the scratch that a call reads is written by that call first, so nothing has to
     // be cleared between calls
     return wide_launch_route(ctx, static_cast<cudaStream_t>(stream), x, dtype, tokens, hidden, w_router, w2, rank,
-                             n_groups, mode, k, k_per_token, mask_bits, scores, scratch);
+                             n_groups, mode, k, k_per_token, mask_bits, scores, scratch, flags);
 }
