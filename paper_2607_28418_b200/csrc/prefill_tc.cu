@@ -365,26 +365,38 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         // Each thread copies its row's 128 bytes with eight 16-byte cp.async and lets the stage's
         // mbarrier count an arrival when they have landed; nothing waits on the issuing side, so
         // the gather runs as far ahead as the ring allows.
-        const int r = (warp - 2) * 32 + lane;  // tile row owned by this thread
-        const uint32_t row_off = static_cast<uint32_t>(r) * 128u;
-        const uint32_t sw = static_cast<uint32_t>(r & 7);
+        // Coalesced mapping: 8 consecutive lanes copy the 8 chunks of one row, a warp instruction
+        // covers 4 whole rows (4 x 128 contiguous bytes); instruction i of warp w handles tile rows
+        // w*32 + 4*i + lane/8.
+        const int chunk = lane & 7;
+        const int row0 = (warp - 2) * 32 + (lane >> 3);
+        uint32_t dst_off[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = row0 + 4 * i;
+            dst_off[i] = static_cast<uint32_t>(r) * 128u + ((static_cast<uint32_t>(chunk) ^ static_cast<uint32_t>(r & 7)) << 4);
+        }
         int it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int pair = item / nsub;
             const int m = work_list[2 * pair], g = work_list[2 * pair + 1];
-            int j = m * kBM + r;
-            if (j >= T) j = T - 1;
-            const int tok = perm[static_cast<size_t>(g) * T + j];
-            const uint8_t* src = reinterpret_cast<const uint8_t*>(X + static_cast<size_t>(tok) * D);
+            const uint8_t* src[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                int j = m * kBM + row0 + 4 * i;
+                if (j >= T) j = T - 1;
+                const int tok = perm[static_cast<size_t>(g) * T + j];
+                src[i] = reinterpret_cast<const uint8_t*>(X + static_cast<size_t>(tok) * D) + 16 * chunk;
+            }
             for (int k = 0; k < nk; ++k, ++it) {
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1;
                 if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
-                const uint32_t a_dst = smem_u32(L.stage_base + s * kStageBytes) + row_off;
-                const uint8_t* p = src + static_cast<size_t>(k) * (kBK * 2);
+                const uint32_t a_dst = smem_u32(L.stage_base + s * kStageBytes);
+                const size_t koff = static_cast<size_t>(k) * (kBK * 2);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) cp_async_16(a_dst + ((static_cast<uint32_t>(c) ^ sw) << 4), p + 16 * c);
+                for (int i = 0; i < 8; ++i) cp_async_16(a_dst + dst_off[i], src[i] + koff);
                 cp_async_mbar_arrive_noinc(L.full + 8 * s);
             }
         }
