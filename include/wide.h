@@ -143,9 +143,9 @@ WIDE_API int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, i
  * device memory where they route -- a serving process whose own pool owns the whole heap, a
  * plugin called under another framework's allocator lock, a deployment that forbids cudaMalloc
  * after start-up.  The call itself allocates nothing on host or device.
- *   - Limit: the scratch the call needs, about tokens * (16 * n_groups + 8 * max(rank, 1) + 128)
+ *   - Limit: the scratch the call needs, about tokens * (16 * n_groups + 8 * max(rank, 1) + 2176)
  *     bytes plus 1 KiB (wide_workspace_bytes(WIDE_OP_ROUTE, ...) is an upper bound), must not
- *     exceed WIDE_ROUTE_STATIC_BYTES (2 MiB: e.g. 1300 tokens x 86 groups, 490 x 256); larger problems
+ *     exceed WIDE_ROUTE_STATIC_BYTES (2 MiB: e.g. 580 tokens x 86 groups, 330 x 256); larger problems
  *     return WIDE_ERR_WORKSPACE and launch nothing.  Every GPU on which the library is loaded
  *     holds those 2 MiB until the process exits.
  *   - The first call on a device looks up the array's device address; it must be made with

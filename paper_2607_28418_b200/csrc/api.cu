@@ -71,11 +71,11 @@ int wide_create(wide_ctx** out, int device) {
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
         ctx->encode_tiled = fn;
-    if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) {
+    if (cudaMalloc(&ctx->d_status, 4 * sizeof(int)) != cudaSuccess) {
         delete ctx;
         return WIDE_ERR_CUDA;
     }
-    if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
+    if (cudaMemset(ctx->d_status, 0, 4 * sizeof(int)) != cudaSuccess) {
         cudaFree(ctx->d_status);
         delete ctx;
         return WIDE_ERR_CUDA;

@@ -16,7 +16,7 @@ struct wide_prof_rec {
 struct wide_ctx {
     int device;
     int sm_count;
-    int* d_status;          // device status word (WIDE_OK or WIDE_ERR_TIMEOUT)
+    int* d_status;          // [0] device status word (WIDE_OK or WIDE_ERR_TIMEOUT), [1] reorder ticket
     unsigned long long wait_ns;  // bound of every device-side wait
     void* encode_tiled;     // cuTensorMapEncodeTiled, resolved through the runtime
     unsigned long long launches;  // kernels launched by the library so far
@@ -96,7 +96,7 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const int32_t* work_list, const int32_t* n_work, void* y,
                                int out_dtype, void* h);
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
-                          int ld, int D, float* scores);
+                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out);
 // `a_masked` is scratch [T, K] bf16.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                  int D, int K, int G, const uint32_t* mask_bits, void* y,

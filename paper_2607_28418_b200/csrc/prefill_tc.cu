@@ -102,7 +102,8 @@ template <int BN>
 __global__ void __launch_bounds__(192, 1)
 down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const uint32_t* __restrict__ mask_bits, int words, int T, int N, int K, int G, void* __restrict__ Y,
-            int out_bf16, int* __restrict__ status, unsigned long long wait_ns) {
+            int out_bf16, int ksplit, const __nv_bfloat16* __restrict__ aux_w, int aux_rows,
+            float* __restrict__ aux_norm, int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -132,8 +133,11 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tc_fence_after_sync();
     const uint32_t tmem_base = *L.tmem_slot;
 
+    // ksplit > 1: the K-groups (exactly ksplit of them) are spread over separate CTAs and each
+    // writes its partial product into its own [T, N] slab of Y; nothing is masked in that mode.
     const int n_m = (T + kBM - 1) / kBM, n_n = (N + BN - 1) / BN;
-    const int n_tiles = n_m * n_n;
+    const int n_mn = n_m * n_n;
+    const int n_tiles = n_mn * ksplit;
     const int NG = K / G, ksub = G / kBK;
 
     if (warp == 0) {
@@ -141,12 +145,13 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int m = tile % n_m, n = tile / n_m;
+            const int mn = tile % n_mn, only = ksplit > 1 ? tile / n_mn : -1;
+            const int m = mn % n_m, n = mn / n_m;
             uint32_t act[kMaskWords];
             tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
             if (lane == 0) {
                 for (int g = 0; g < NG && ok; ++g) {
-                    if (!((act[g >> 5] >> (g & 31)) & 1u)) continue;
+                    if (!((act[g >> 5] >> (g & 31)) & 1u) || (only >= 0 && g != only)) continue;
                     for (int kk = 0; kk < ksub; ++kk, ++it) {
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1;
@@ -168,7 +173,8 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int it = 0, tc = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
-            const int m = tile % n_m;
+            const int mn = tile % n_mn, only = ksplit > 1 ? tile / n_mn : -1;
+            const int m = mn % n_m;
             uint32_t act[kMaskWords];
             tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
             if (lane == 0) {
@@ -179,7 +185,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t d_tmem = tmem_base + buf * kAccCols;
                 uint32_t accumulate = 0;
                 for (int g = 0; g < NG && ok; ++g) {
-                    if (!((act[g >> 5] >> (g & 31)) & 1u)) continue;
+                    if (!((act[g >> 5] >> (g & 31)) & 1u) || (only >= 0 && g != only)) continue;
                     for (int kk = 0; kk < ksub; ++kk, ++it) {
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1;
@@ -210,7 +216,8 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int tc = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
-            const int m = tile % n_m, n = tile / n_m;
+            const int mn = tile % n_mn, slab = ksplit > 1 ? tile / n_mn : 0;
+            const int m = mn % n_m, n = mn / n_m;
             uint32_t act[kMaskWords];
             tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
             bool any = false;
@@ -245,7 +252,8 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             dst[v] = o;
                         }
                     } else {
-                        uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(Y) + static_cast<size_t>(row) * N + col);
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(Y) + static_cast<size_t>(slab) * T * N +
+                                                              static_cast<size_t>(row) * N + col);
 #pragma unroll
                         for (int v = 0; v < 8; ++v) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                     }
@@ -256,6 +264,29 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (lane == 0) mbar_arrive(L.tempty + 8 * buf);
         }
         if (!ok && lane == 0) report_timeout(status);
+    }
+
+    // Spare CTAs (blockIdx.x >= n_tiles) carry a side job: the Euclidean norm of every row of
+    // aux_w, slightly rounded up, one warp per row (the router's error bound needs it).
+    if (aux_norm != nullptr && static_cast<int>(blockIdx.x) >= n_tiles) {
+        const int first = (static_cast<int>(blockIdx.x) - n_tiles) * 6;
+        const int r = first + warp;
+        if (r < aux_rows) {
+            const uint4* rowp = reinterpret_cast<const uint4*>(aux_w + static_cast<size_t>(r) * K);
+            float acc = 0.f;
+            for (int i = lane; i < K / 8; i += 32) {
+                const uint4 v = rowp[i];
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __bfloat1622float2(h[e]);
+                    acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) aux_norm[r] = sqrtf(acc) * 1.0001f;
+        }
     }
 
     tc_fence_before_sync();
@@ -490,17 +521,20 @@ bool make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uin
 
 template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
-                int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down") {
+                int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down",
+                int ksplit = 1, float* aux_norm = nullptr) {
     CUtensorMap tmA, tmB;
     if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
     constexpr int smem = smem_bytes<BN * kBK * 2>();
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    const int n_tiles = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
-    const int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
+    const int n_tiles = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN) * ksplit;
+    int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
+    if (aux_norm) grid = n_tiles + (b_rows + 5) / 6;  // spare CTAs for the row norms of B
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, name);
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
+                                            ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm,
                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
@@ -555,12 +589,23 @@ int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, c
     return launch_down<256>(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype);
 }
 
-// scores[T, ld] (fp32) = x[T, D] * w_router[NG, D]^T on the tensor cores; ld = NG rounded up to 32,
-// columns >= NG are written as zeros (weight rows past NG are zero-filled by the TMA).
+// scores (fp32) = x[T, D] * w_router[NG, D]^T on the tensor cores, K split `ksplit` ways: slab ks
+// [T, ld] holds the partial sum over columns [ks*D/ksplit, (ks+1)*D/ksplit); ld = NG rounded up to
+// 32, columns >= NG are zeros (weight rows past NG are zero-filled by the TMA).  The same launch
+// writes ||w_g|| (rounded up) to wnorm[0..NG).  Returns the ksplit it used through *ksplit_out.
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
-                          int ld, int D, float* scores) {
+                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out) {
+    const int n_m = (T + kBM - 1) / kBM;
+    int ksplit = 1;
+    // more CTAs while each keeps >= 8 k-steps, the slabs fit, and everything is co-resident
+    while (ksplit * 2 <= max_split && D % (ksplit * 2 * kBK) == 0 && D / (ksplit * 2 * kBK) >= 8 &&
+           n_m * ksplit * 2 + (NG + 5) / 6 <= ctx->sm_count)
+        ksplit *= 2;
+    *ksplit_out = ksplit;
     if (T == 0) return WIDE_OK;
     if (ld <= 128)
-        return launch_down<128>(ctx, s, x, w_router, nullptr, T, ld, D, D, scores, WIDE_F32, NG, "route_scores_tc");
-    return launch_down<256>(ctx, s, x, w_router, nullptr, T, ld, D, D, scores, WIDE_F32, NG, "route_scores_tc");
+        return launch_down<128>(ctx, s, x, w_router, nullptr, T, ld, D, D / ksplit, scores, WIDE_F32, NG,
+                                "route_scores_tc", ksplit, wnorm);
+    return launch_down<256>(ctx, s, x, w_router, nullptr, T, ld, D, D / ksplit, scores, WIDE_F32, NG,
+                            "route_scores_tc", ksplit, wnorm);
 }

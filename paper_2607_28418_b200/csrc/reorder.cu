@@ -7,12 +7,24 @@ namespace {
 
 constexpr int kPartThreads = 512;
 
+__device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_tiles, uint8_t* __restrict__ tile_map,
+                               int32_t* __restrict__ work_list, int32_t* __restrict__ n_work,
+                               int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
+                               int32_t* __restrict__ offsets);
+
 // One CTA per group: pass 1 counts the active rows, pass 2 places every row.
 __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t* __restrict__ mask_bits, int T,
                                                                  int NG, int words, int32_t* __restrict__ perm,
-                                                                 int32_t* __restrict__ counts) {
+                                                                 int32_t* counts, int tile_m, int n_tiles,
+                                                                 uint8_t* __restrict__ tile_map,
+                                                                 int32_t* __restrict__ work_list,
+                                                                 int32_t* __restrict__ n_work,
+                                                                 int32_t* __restrict__ union_list,
+                                                                 int32_t* __restrict__ n_union,
+                                                                 int32_t* __restrict__ offsets, int* ticket) {
     __shared__ int warp_cnt[kPartThreads / 32];
     __shared__ int s_total;
+    __shared__ int s_last;
     const int g = blockIdx.x;
     const int w = g >> 5, b = g & 31;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -54,19 +66,32 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t*
         }
         base += chunk;
     }
+
+    // The CTA that finishes last has every group's count in view and builds the rest.
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const int done = atomicAdd(ticket, 1);
+        s_last = (done == NG - 1) ? 1 : 0;
+        if (s_last) *ticket = 0;  // ready for the next call on this context
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        build_metadata(counts, NG, tile_m, n_tiles, tile_map, work_list, n_work, union_list, n_union, offsets);
+    }
 }
 
-// One CTA: offsets, tile map, work list, union list.
-__global__ void __launch_bounds__(256) metadata_kernel(const int32_t* __restrict__ counts, int T, int NG,
-                                                       int tile_m, int n_tiles, uint8_t* __restrict__ tile_map,
-                                                       int32_t* __restrict__ work_list, int32_t* __restrict__ n_work,
-                                                       int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
-                                                       int32_t* __restrict__ offsets) {
+// Run by one whole CTA: offsets, tile map, work list, union list.
+__device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_tiles, uint8_t* __restrict__ tile_map,
+                               int32_t* __restrict__ work_list, int32_t* __restrict__ n_work,
+                               int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
+                               int32_t* __restrict__ offsets) {
     __shared__ int s_tiles[WIDE_MAX_GROUPS];      // active tiles of each group
     __shared__ int s_work_off[WIDE_MAX_GROUPS + 1];
     __shared__ int s_union_pos[WIDE_MAX_GROUPS + 1];
     const int tid = threadIdx.x;
-    for (int g = tid; g < NG; g += blockDim.x) s_tiles[g] = (counts[g] + tile_m - 1) / tile_m;
+    for (int g = tid; g < NG; g += blockDim.x) s_tiles[g] = (__ldcg(counts + g) + tile_m - 1) / tile_m;
     __syncthreads();
     if (tid == 0) {
         int woff = 0, uoff = 0, roff = 0;
@@ -75,7 +100,7 @@ __global__ void __launch_bounds__(256) metadata_kernel(const int32_t* __restrict
             s_union_pos[g] = uoff;
             offsets[g] = roff;
             woff += s_tiles[g];
-            uoff += counts[g] > 0 ? 1 : 0;
+            uoff += __ldcg(counts + g) > 0 ? 1 : 0;
             roff += s_tiles[g] * tile_m;
         }
         s_work_off[NG] = woff;
@@ -100,7 +125,7 @@ __global__ void __launch_bounds__(256) metadata_kernel(const int32_t* __restrict
             work_list[2 * (wo + m)] = m;
             work_list[2 * (wo + m) + 1] = g;
         }
-        if (counts[g] > 0) union_list[s_union_pos[g]] = g;
+        if (__ldcg(counts + g) > 0) union_list[s_union_pos[g]] = g;
         if (g >= total_union) union_list[g] = -1;
     }
 }
@@ -133,13 +158,9 @@ int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits
                         int32_t* offsets) {
     const int words = (NG + 31) / 32;
     const int n_tiles = (T + tile_m - 1) / tile_m;
-    {
-        WideLaunch l(ctx, s, "reorder_partition");
-        partition_kernel<<<NG, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts);
-    }
-    WideLaunch l(ctx, s, "reorder_metadata");
-    metadata_kernel<<<1, 256, 0, s>>>(counts, T, NG, tile_m, n_tiles, tile_map, work_list, n_work,
-                                      union_list, n_union, offsets);
+    WideLaunch l(ctx, s, "reorder_partition");
+    partition_kernel<<<NG, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts, tile_m, n_tiles, tile_map,
+                                                 work_list, n_work, union_list, n_union, offsets, ctx->d_status + 1);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 

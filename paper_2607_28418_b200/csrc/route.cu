@@ -114,43 +114,36 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 // The result equals the fp64 decision of the slow path.
 constexpr float kAccumErr = 5.9604645e-8f;  // 2^-24 per accumulated element
 
-// ||w_g||_2 for every group, one warp per group.
-__global__ void __launch_bounds__(256) wnorm_kernel(const __nv_bfloat16* __restrict__ w, int NG, int D,
-                                                    float* __restrict__ wnorm) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = blockIdx.x * 8 + warp;
-    if (g >= NG) return;
-    const uint4* row = reinterpret_cast<const uint4*>(w + static_cast<size_t>(g) * D);
-    float acc = 0.f;
-    for (int i = lane; i < D / 8; i += 32) {
-        const uint4 v = row[i];
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(h[e]);
-            acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) wnorm[g] = sqrtf(acc) * 1.0001f;  // rounded up a little: it feeds a bound
-}
+constexpr int kSelWarps = 4;   // tokens (warps) per CTA in select_band_kernel
+constexpr int kBatch = 8;      // 16-byte loads in flight per lane
 
-// Exact x_t . w_g in fp64 by one warp (bf16 products are exact in fp64).
-__device__ __forceinline__ double warp_dot_f64(const __nv_bfloat16* __restrict__ xrow,
-                                               const __nv_bfloat16* __restrict__ wrow, int D, int lane) {
-    const uint4* xv = reinterpret_cast<const uint4*>(xrow);
+// Exact x_t . w_g in fp64 by one warp: x row in shared memory, w row streamed from L2 with
+// kBatch loads in flight per lane (bf16 products are exact in fp64).
+__device__ __forceinline__ double warp_dot_f64(const uint4* __restrict__ xs, const __nv_bfloat16* __restrict__ wrow,
+                                               int nch, int lane) {
     const uint4* wv = reinterpret_cast<const uint4*>(wrow);
     double acc = 0.0;
-    for (int i = lane; i < D / 8; i += 32) {
-        const uint4 a = xv[i], b = wv[i];
-        const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
-        const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b);
+    for (int base = 0; base < nch; base += 32 * kBatch) {
+        uint4 b[kBatch];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float2 fa = __bfloat1622float2(ah[e]), fb = __bfloat1622float2(bh[e]);
-            acc = fma(static_cast<double>(fa.x), static_cast<double>(fb.x), acc);
-            acc = fma(static_cast<double>(fa.y), static_cast<double>(fb.y), acc);
+        for (int j = 0; j < kBatch; ++j) {
+            const int i = base + lane + 32 * j;
+            b[j] = i < nch ? wv[i] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int i = base + lane + 32 * j;
+            if (i < nch) {
+                const uint4 a = xs[i];
+                const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+                const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b[j]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 fa = __bfloat1622float2(ah[e]), fb = __bfloat1622float2(bh[e]);
+                    acc = fma(static_cast<double>(fa.x), static_cast<double>(fb.x), acc);
+                    acc = fma(static_cast<double>(fa.y), static_cast<double>(fb.y), acc);
+                }
+            }
         }
     }
 #pragma unroll
@@ -158,132 +151,152 @@ __device__ __forceinline__ double warp_dot_f64(const __nv_bfloat16* __restrict__
     return acc;
 }
 
-// One warp per token.
-__global__ void __launch_bounds__(256) select_band_kernel(const float* __restrict__ scores, int ld,
-                                                          const __nv_bfloat16* __restrict__ x,
-                                                          const __nv_bfloat16* __restrict__ w,
-                                                          const float* __restrict__ wnorm, int T, int NG, int D,
-                                                          int k, const int32_t* __restrict__ k_per_token,
-                                                          uint32_t* __restrict__ mask_bits,
-                                                          float* __restrict__ scores_out) {
-    __shared__ float sh_s[8][WIDE_MAX_GROUPS];
-    __shared__ double sh_e[8][WIDE_MAX_GROUPS];
-    __shared__ float sh_b[8][2];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = blockIdx.x * 8 + warp;
-    if (t >= T) return;
-    float* s = sh_s[warp];
-    double* ex = sh_e[warp];
+// One CTA (4 warps) per token.  scores: nsplit partial slabs [nsplit][T, ld] that are summed on
+// load.  Thread g ranks group g (and g + 128); the exact re-scoring of the band is spread over
+// the four warps.
+__global__ void __launch_bounds__(32 * kSelWarps)
+select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
+                   const __nv_bfloat16* __restrict__ w, const float* __restrict__ wnorm, int T, int NG, int D, int k,
+                   const int32_t* __restrict__ k_per_token, uint32_t* __restrict__ mask_bits,
+                   float* __restrict__ scores_out) {
+    extern __shared__ uint4 sh_x[];  // [D / 8]
+    __shared__ float s[WIDE_MAX_GROUPS];
+    __shared__ double ex[WIDE_MAX_GROUPS];
+    __shared__ int band[WIDE_MAX_GROUPS];
+    __shared__ float red[2 * kSelWarps];
+    __shared__ float sh_b[2];
+    __shared__ int n_band, n_band_hi;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int t = blockIdx.x;
+    const int nch = D / 8;
     const int words = (NG + 31) >> 5;
+    const size_t slab = static_cast<size_t>(T) * ld;
+    constexpr int kThreads = 32 * kSelWarps;
+    constexpr int kPer = WIDE_MAX_GROUPS / kThreads;  // groups per thread (2)
+
     float wmax = 0.f;
-    for (int g = lane; g < NG; g += 32) {
-        const float v = scores[static_cast<size_t>(t) * ld + g];
-        s[g] = v;
-        wmax = fmaxf(wmax, wnorm[g]);
-        if (scores_out) scores_out[static_cast<size_t>(t) * NG + g] = v;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+        const int g = tid + q * kThreads;
+        if (g < NG) {
+            float v = 0.f;
+            for (int ks = 0; ks < nsplit; ++ks) v += scores[ks * slab + static_cast<size_t>(t) * ld + g];
+            s[g] = v;
+            wmax = fmaxf(wmax, wnorm[g]);
+            if (scores_out) scores_out[static_cast<size_t>(t) * NG + g] = v;
+        }
+    }
+    const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
+    const bool boundary = kt > 0 && kt < NG;
+
+    // x row -> shared memory, partial ||x_t||^2 on the way
+    float xsq = 0.f;
+    if (boundary) {
+        const uint4* xv = reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * D);
+        for (int base = 0; base < nch; base += kThreads * kBatch) {
+            uint4 a[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int i = base + tid + kThreads * j;
+                a[j] = i < nch ? xv[i] : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int i = base + tid + kThreads * j;
+                if (i < nch) {
+                    sh_x[i] = a[j];
+                    const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a[j]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __bfloat1622float2(ah[e]);
+                        xsq = fmaf(f.x, f.x, fmaf(f.y, f.y, xsq));
+                    }
+                }
+            }
+        }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
-    __syncwarp();
-    const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
-    const __nv_bfloat16* xrow = x + static_cast<size_t>(t) * D;
+    for (int o = 16; o > 0; o >>= 1) {
+        xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
+        wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
+    }
+    if (lane == 0) { red[warp] = xsq; red[kSelWarps + warp] = wmax; }
+    if (tid == 0) { sh_b[0] = 0.f; sh_b[1] = 0.f; n_band = 0; n_band_hi = 0; }
+    __syncthreads();
+    xsq = 0.f;
+    wmax = 0.f;
+#pragma unroll
+    for (int i = 0; i < kSelWarps; ++i) { xsq += red[i]; wmax = fmaxf(wmax, red[kSelWarps + i]); }
 
     // fp32 ranks; remember the k-th and (k+1)-th largest
-    int rank[WIDE_MAX_GROUPS / 32];
-    if (lane == 0) { sh_b[warp][0] = 0.f; sh_b[warp][1] = 0.f; }
-    __syncwarp();
+    int rank[kPer];
 #pragma unroll
-    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
-        rank[w8] = NG;
-        const int g = w8 * 32 + lane;
-        if (w8 < words && g < NG) {
+    for (int q = 0; q < kPer; ++q) {
+        rank[q] = NG;
+        const int g = tid + q * kThreads;
+        if (g < NG) {
             const float v = s[g];
             int beats = 0;
             for (int h = 0; h < NG; ++h) {
                 const float u = s[h];
                 beats += (u > v) || (u == v && h < g);
             }
-            rank[w8] = beats;
-            if (beats == kt - 1) sh_b[warp][0] = v;
-            if (beats == kt) sh_b[warp][1] = v;
+            rank[q] = beats;
+            if (beats == kt - 1) sh_b[0] = v;
+            if (beats == kt) sh_b[1] = v;
         }
     }
-    __syncwarp();
-    const bool boundary = kt > 0 && kt < NG;
-    const float v_k = sh_b[warp][0], v_k1 = sh_b[warp][1];
+    __syncthreads();
+    const float v_k = sh_b[0], v_k1 = sh_b[1];
+    // band half-width 2 * eps_t (a little slack for the fp32 evaluation of the bound itself)
+    const float tau = boundary ? 2.f * kAccumErr * static_cast<float>(D) * sqrtf(xsq) * 1.0001f * wmax : 0.f;
 
-    float tau = 0.f;
-    if (boundary) {
-        // ||x_t||, then the band half-width 2*eps
-        float acc = 0.f;
-        const uint4* xv = reinterpret_cast<const uint4*>(xrow);
-        for (int i = lane; i < D / 8; i += 32) {
-            const uint4 a = xv[i];
-            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+    bool in_band[kPer];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 f = __bfloat1622float2(ah[e]);
-                acc = fmaf(f.x, f.x, fmaf(f.y, f.y, acc));
+    for (int q = 0; q < kPer; ++q) {
+        in_band[q] = false;
+        const int g = tid + q * kThreads;
+        if (boundary && g < NG) {
+            const bool hi = rank[q] < kt;
+            const bool u = hi ? (s[g] - v_k1 <= tau) : (v_k - s[g] <= tau);
+            if (u) {
+                in_band[q] = true;
+                band[atomicAdd(&n_band, 1)] = g;
+                if (hi) atomicAdd(&n_band_hi, 1);
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        tau = 2.f * kAccumErr * static_cast<float>(D) * sqrtf(acc) * 1.0001f * wmax;
     }
-
-    // band membership, exact scores of the band
-    unsigned in_band[WIDE_MAX_GROUPS / 32];
-    int m_hi = 0;  // band members currently ranked inside the top k
-#pragma unroll
-    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
-        in_band[w8] = 0u;
-        if (w8 >= words) continue;
-        const int g = w8 * 32 + lane;
-        bool u = false, hi = false;
-        if (boundary && g < NG) {
-            hi = rank[w8] < kt;
-            u = hi ? (s[g] - v_k1 <= tau) : (v_k - s[g] <= tau);
-        }
-        unsigned vote = __ballot_sync(0xffffffffu, u);
-        in_band[w8] = vote;
-        m_hi += __popc(__ballot_sync(0xffffffffu, u && hi));
-        while (vote) {
-            const int b = __ffs(vote) - 1;
-            vote &= vote - 1;
-            const int gg = w8 * 32 + b;
-            const double e = warp_dot_f64(xrow, w + static_cast<size_t>(gg) * D, D, lane);
-            if (lane == 0) ex[gg] = e;
-        }
+    __syncthreads();
+    const int nb = n_band, m_hi = n_band_hi;
+    for (int i = warp; i < nb; i += kSelWarps) {
+        const int gg = band[i];
+        const double e = warp_dot_f64(sh_x, w + static_cast<size_t>(gg) * D, nch, lane);
+        if (lane == 0) ex[gg] = e;
     }
-    __syncwarp();
+    __syncthreads();
 
-    // final decision
+    // final decision: band members are re-ranked among themselves on the exact scores
 #pragma unroll
-    for (int w8 = 0; w8 < WIDE_MAX_GROUPS / 32; ++w8) {
-        if (w8 >= words) continue;
-        const int g = w8 * 32 + lane;
+    for (int q = 0; q < kPer; ++q) {
+        const int g = tid + q * kThreads;
         bool sel = false;
         if (g < NG) {
-            if ((in_band[w8] >> lane) & 1u) {
+            if (in_band[q]) {
                 const double v = ex[g];
                 int beats = 0;
-                for (int w2 = 0; w2 < words; ++w2) {
-                    unsigned bits = in_band[w2];
-                    while (bits) {
-                        const int b = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        const int h = w2 * 32 + b;
-                        const double u = ex[h];
-                        beats += (u > v) || (u == v && h < g);
-                    }
+                for (int i = 0; i < nb; ++i) {
+                    const int h = band[i];
+                    const double u = ex[h];
+                    beats += (u > v) || (u == v && h < g);
                 }
                 sel = beats < m_hi;
             } else {
-                sel = rank[w8] < kt;
+                sel = rank[q] < kt;
             }
         }
         const unsigned word = __ballot_sync(0xffffffffu, sel);
-        if (lane == 0) mask_bits[static_cast<size_t>(t) * words + w8] = word;
+        const int widx = warp + q * kSelWarps;
+        if (lane == 0 && widx < words) mask_bits[static_cast<size_t>(t) * words + widx] = word;
     }
 }
 
@@ -303,28 +316,32 @@ size_t wide_route_workspace(int T, int NG, int rank) {
     // the group norms in the tail
     return wide_align_up(static_cast<size_t>(T) * 2 * NG * sizeof(double), 256) +
            wide_align_up(static_cast<size_t>(T) * (rank > 0 ? rank : 1) * sizeof(double), 256) +
-           wide_align_up(static_cast<size_t>(T) * 128, 256) + 1024;
+           wide_align_up(static_cast<size_t>(T) * 128, 256) + wide_align_up(static_cast<size_t>(T) * 2048, 256) + 1024;
 }
 
 int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
                       const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws, unsigned flags) {
     if (T == 0) return WIDE_OK;
-    if (mode == WIDE_ROUTE_TOPK && dtype == WIDE_BF16 && D % 64 == 0 && ctx->encode_tiled &&
+    if (mode == WIDE_ROUTE_TOPK && dtype == WIDE_BF16 && D % 64 == 0 && D <= 16384 && ctx->encode_tiled &&
         !(flags & WIDE_FLAG_SIMT)) {
         const int ld = (NG + 31) / 32 * 32;
         float* sc32 = static_cast<float*>(ws);
         float* wn = reinterpret_cast<float*>(static_cast<char*>(ws) + wide_route_workspace(T, NG, rank) - 1024);
-        {
-            WideLaunch l(ctx, s, "route_wnorm");
-            wnorm_kernel<<<(NG + 7) / 8, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(w_router), NG, D, wn);
-        }
-        const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32);
+        // as many K-split slabs as the first part of the workspace holds (at most 8)
+        const size_t part0 = wide_route_workspace(T, NG, rank) - 1024;
+        int max_split = static_cast<int>(part0 / (static_cast<size_t>(T) * ld * sizeof(float)));
+        if (max_split > 8) max_split = 8;
+        if (max_split < 1) max_split = 1;
+        int ksplit = 1;
+        const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32, wn, max_split, &ksplit);
         if (rc != WIDE_OK) return rc;
+        const int sel_smem = (D / 8) * static_cast<int>(sizeof(uint4));
+        WIDE_CUDA_CHECK(cudaFuncSetAttribute(select_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sel_smem));
         WideLaunch l(ctx, s, "route_select_band");
-        select_band_kernel<<<(T + 7) / 8, 256, 0, s>>>(sc32, ld, static_cast<const __nv_bfloat16*>(x),
-                                                       static_cast<const __nv_bfloat16*>(w_router), wn, T, NG, D, k,
-                                                       k_per_token, mask_bits, scores);
+        select_band_kernel<<<T, 32 * kSelWarps, sel_smem, s>>>(
+            sc32, ksplit, ld, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router), wn, T,
+            NG, D, k, k_per_token, mask_bits, scores);
         return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
     }
     double* sc = static_cast<double*>(ws);
