@@ -307,8 +307,7 @@ def run_ours(args):
             union_words = np.bitwise_or.reduce(bits.cpu().numpy().view(np.uint32), axis=0)
             n_union = sum(bin(int(w)).count("1") for w in union_words)
             per_group = cfg.group * cfg.hidden * 2
-            bytes_alg = {"decode_stream_gateup": 2.0 * n_union * per_group,
-                         "decode_stream_down": 1.0 * n_union * per_group}.get(dom, 3.0 * n_union * per_group)
+            bytes_alg = 3.0 * n_union * per_group     # gate + up + down weights of the groups in the union
             ach = bytes_alg / avg_s / 1e9
             roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.name)),

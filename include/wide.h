@@ -80,12 +80,15 @@ extern "C" {
 typedef struct wide_ctx wide_ctx;
 
 /* Create / destroy a context bound to CUDA device `device` (ordinal).  The context holds the
- * device properties and a 4-byte device status word; nothing else.  Host-synchronous. */
+ * device properties, a few device status / barrier words and the fp32 accumulators of the decode
+ * path (21 MB, kept zero between calls).  Host-synchronous.  A context serves one stream at a
+ * time: calls issued through the same context must not overlap on the GPU. */
 WIDE_API int wide_create(wide_ctx** ctx, int device);
 WIDE_API int wide_destroy(wide_ctx* ctx);
 
 /* Synchronise `stream`, read the device status word into *status (WIDE_OK or
- * WIDE_ERR_TIMEOUT) and clear it.  The only call that blocks the host. */
+ * WIDE_ERR_TIMEOUT) and clear it; after a timeout the context's internal buffers are reset.
+ * The only call that blocks the host. */
 WIDE_API int wide_status(wide_ctx* ctx, void* stream, int* status);
 
 /* Override the bound of every device-side wait (nanoseconds; default 2e9). */

@@ -71,11 +71,17 @@ int wide_create(wide_ctx** out, int device) {
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
         ctx->encode_tiled = fn;
-    if (cudaMalloc(&ctx->d_status, 4 * sizeof(int)) != cudaSuccess) {
+    // decode accumulators: 64 tokens x (2 * inner + hidden) floats for inner <= 32768, hidden <= 16384
+    ctx->decode_acc = nullptr;
+    ctx->decode_acc_floats = static_cast<size_t>(WIDE_DECODE_MAX_TOKENS) * (2 * 32768 + 16384);
+    if (cudaMalloc(&ctx->d_status, 16 * sizeof(int)) != cudaSuccess) {
         delete ctx;
         return WIDE_ERR_CUDA;
     }
-    if (cudaMemset(ctx->d_status, 0, 4 * sizeof(int)) != cudaSuccess) {
+    if (cudaMalloc(&ctx->decode_acc, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess ||
+        cudaMemset(ctx->d_status, 0, 16 * sizeof(int)) != cudaSuccess ||
+        cudaMemset(ctx->decode_acc, 0, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess) {
+        cudaFree(ctx->decode_acc);
         cudaFree(ctx->d_status);
         delete ctx;
         return WIDE_ERR_CUDA;
@@ -150,6 +156,7 @@ int wide_launch_count(wide_ctx* ctx, unsigned long long* count) {
 int wide_destroy(wide_ctx* ctx) {
     if (!ctx) return WIDE_ERR_INVALID_ARG;
     free_profile(ctx);
+    cudaFree(ctx->decode_acc);
     cudaFree(ctx->d_status);
     delete ctx;
     return WIDE_OK;
@@ -162,6 +169,12 @@ int wide_status(wide_ctx* ctx, void* stream, int* status) {
     WIDE_CUDA_CHECK(cudaMemcpyAsync(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
     WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s));
     WIDE_CUDA_CHECK(cudaStreamSynchronize(s));
+    if (v != WIDE_OK) {
+        // a kernel gave up half-way: restore the invariants later calls rely on
+        WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->d_status, 0, 16 * sizeof(int), s));
+        WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->decode_acc, 0, ctx->decode_acc_floats * sizeof(float), s));
+        WIDE_CUDA_CHECK(cudaStreamSynchronize(s));
+    }
     *status = v;
     return WIDE_OK;
 }
