@@ -78,10 +78,14 @@ int wide_create(wide_ctx** out, int device) {
         delete ctx;
         return WIDE_ERR_CUDA;
     }
+    ctx->d_tickets = nullptr;
     if (cudaMalloc(&ctx->decode_acc, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&ctx->d_tickets, 2048 * sizeof(unsigned)) != cudaSuccess ||
+        cudaMemset(ctx->d_tickets, 0, 2048 * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->d_status, 0, 16 * sizeof(int)) != cudaSuccess ||
         cudaMemset(ctx->decode_acc, 0, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess) {
         cudaFree(ctx->decode_acc);
+        cudaFree(ctx->d_tickets);
         cudaFree(ctx->d_status);
         delete ctx;
         return WIDE_ERR_CUDA;
@@ -156,6 +160,7 @@ int wide_launch_count(wide_ctx* ctx, unsigned long long* count) {
 int wide_destroy(wide_ctx* ctx) {
     if (!ctx) return WIDE_ERR_INVALID_ARG;
     free_profile(ctx);
+    cudaFree(ctx->d_tickets);
     cudaFree(ctx->decode_acc);
     cudaFree(ctx->d_status);
     delete ctx;
@@ -173,6 +178,7 @@ int wide_status(wide_ctx* ctx, void* stream, int* status) {
         // a kernel gave up half-way: restore the invariants later calls rely on
         WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->d_status, 0, 16 * sizeof(int), s));
         WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->decode_acc, 0, ctx->decode_acc_floats * sizeof(float), s));
+        WIDE_CUDA_CHECK(cudaMemsetAsync(ctx->d_tickets, 0, 2048 * sizeof(unsigned), s));
         WIDE_CUDA_CHECK(cudaStreamSynchronize(s));
     }
     *status = v;

@@ -3,26 +3,26 @@
 //
 // Reordering is bypassed (the paper does the same for T_q = 1 and dispatches GEMV-style kernels
 // for tiny M); instead every CTA forms the union U of the groups selected by any token of the
-// batch, and only the weight rows / columns of groups in U are read, each exactly once:
+// batch, and only the weight rows / columns of groups in U are read, each exactly once.
 //
-//   phase 1 (FFN)   stream W_gate / W_up rows of groups in U:  C^T[128 rows, NT tokens] +=
-//                   W_tile * X_tile^T  (swap-AB: the weight tile is the 128-row UMMA operand, the
-//                   padded batch is N).  Weight tiles arrive by TMA through an 8-stage ring
-//                   (>= 128 KB in flight per SM), tcgen05 accumulates in TMEM, the epilogue adds
-//                   the partial tile into an L2-resident fp32 accumulator with coalesced red.add.
-//                   Items are ~128 KB of weights (K split), so every SM streams until the end.
-//       (O-proj)    instead: a_masked = M ? attn_out : 0
-//   grid barrier
-//   phase 2 (FFN)   h = M ? silu(gate) * up : 0 -> bf16, accumulators re-zeroed on the way
-//   grid barrier
-//   phase 3         stream W_down (or W_o): 128-row tiles x chunks of groups in U, same pipeline,
-//                   partial tiles added into the fp32 output accumulator
-//   grid barrier
-//   phase 4         accumulator -> output dtype, accumulator re-zeroed
+//   pass 1 (FFN)  W_gate / W_up rows of groups in U:  C^T[128 rows, NT tokens] += W_tile * X_tile^T
+//                 (swap-AB: the weight tile is the 128-row UMMA operand, the padded batch is N).
+//                 The k-steps of all row blocks form one long sequence that is cut into equal,
+//                 contiguous shares, one per CTA, so every SM streams the same number of bytes and
+//                 a row block is split between at most a few CTAs.  Weight tiles arrive by TMA
+//                 through an 8-stage ring (>= 128 KB in flight per SM), tcgen05 accumulates in
+//                 TMEM, the epilogue adds each partial tile into an L2-resident fp32 accumulator
+//                 with 16-byte red.add.  The CTA that adds the last partial of a 128-channel block
+//                 (a ticket counter tells) turns it into h = M ? silu(gate) * up : 0 (bf16) and
+//                 re-zeroes the accumulator.
+//       (O-proj)  instead: a_masked = M ? attn_out : 0
+//   grid barrier  -- while waiting, each CTA's ring is already filled with its first W_down tiles
+//   pass 2        W_down (or W_o): 128-row tiles x the columns of groups in U, same scheme; the CTA
+//                 that adds the last partial of a row tile converts it to the output dtype and
+//                 re-zeroes the accumulator.
 //
-// The fp32 accumulators belong to the context and are zero between calls; a call leaves them zero.
-// Grid barriers are counters in the context with bounded spins.  One context must not run two
-// decode calls concurrently.
+// The fp32 accumulators, ticket counters and barrier words belong to the context and are zero
+// between calls.  One context must not run two decode calls concurrently.
 #include <cuda.h>
 
 #include "internal.h"
@@ -50,18 +50,18 @@ struct DecodeArgs {
     int D, inner, G, NG, words;
     int rows_valid;        // gate/up weight rows fetched per tile: min(G, 128)
     int blocks_per_group;  // gate/up: max(1, G / 128)
-    int kchunk, ksplit;    // gate/up: k columns per item, items per row block
-    int row_tiles;         // down: ceil(D / 128)
-    int groups_per_item;   // down
+    int row_tiles;         // pass 2: ceil(D / 128)
     const uint32_t* mask_bits;
     const __nv_bfloat16* act_in;  // O-proj: attention output [B, inner]
-    float* gate;           // [64, inner] fp32, zero on entry and on exit
+    float* gate;           // [inner, NT] fp32 (token fastest), zero on entry and on exit
     float* up;
-    float* yacc;           // [64, D]
+    float* yacc;           // [D, NT]
     __nv_bfloat16* h;      // [64, inner] bf16 scratch (caller workspace)
     void* y;
     int out_bf16;
-    unsigned* bar;         // 3 grid-barrier counters
+    unsigned* bar;         // grid barrier: arrivals, departures
+    unsigned* tickets1;    // one per (union slot, 128-channel block)
+    unsigned* tickets2;    // one per output row tile
     int* status;
     unsigned long long wait_ns;
 };
@@ -75,8 +75,33 @@ struct Pipe {
     int tc;  // accumulator tiles so far (per role)
 };
 
-__device__ __forceinline__ void red_add_f32(float* p, float v) {
-    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+// One contiguous piece of a CTA's share: `nsteps` k-steps of work block `blk` starting at step k0.
+struct Segment { int blk, k0, nsteps; };
+
+// Share of CTA `cta`: global k-steps [cta*L, min((cta+1)*L, total)), cut at block boundaries.
+struct Share {
+    int cur, end, spb;
+    __device__ Share(int cta, int total, int L, int steps_per_block) : cur(cta * L), end(min((cta + 1) * L, total)), spb(steps_per_block) {
+        if (cur > end) cur = end;
+    }
+    __device__ bool next(Segment& s) {
+        if (cur >= end) return false;
+        s.blk = cur / spb;
+        s.k0 = cur - s.blk * spb;
+        s.nsteps = min(spb - s.k0, end - cur);
+        cur += s.nsteps;
+        return true;
+    }
+};
+
+// Number of CTAs whose share touches block `blk`.
+__device__ __forceinline__ int pieces_of_block(int blk, int spb, int L) {
+    const int first = blk * spb, last = first + spb - 1;
+    return last / L - first / L + 1;
+}
+
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     unsigned v;
@@ -84,157 +109,276 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     return v;
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// All CTAs of the (co-resident) grid meet here.  Returns false if the wait expired.
-__device__ bool grid_barrier(unsigned* counter, unsigned long long wait_ns, volatile int* abort_flag, int* status) {
+// All CTAs of the (co-resident) grid meet here; used once per launch.  bar[0] counts arrivals,
+// bar[1] departures: the CTA that leaves last puts both back to zero for the next launch, so the
+// kernel can be replayed from a CUDA graph without host-side state.  Returns false if the wait
+// expired.
+__device__ bool grid_barrier(unsigned* bar, unsigned long long wait_ns, volatile int* abort_flag, int* status) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(counter, 1u);
+        atomicAdd(bar, 1u);
+        bool passed = true;
         if (!*abort_flag) {
             const uint64_t start = globaltimer_ns();
-            while (ld_acquire_u32(counter) < gridDim.x) {
-                __nanosleep(32);
+            while (ld_acquire_u32(bar) < gridDim.x) {
+                __nanosleep(20);
                 if (globaltimer_ns() - start > wait_ns) {
                     *abort_flag = 1;
                     atomicExch(status, WIDE_ERR_TIMEOUT);
+                    passed = false;
                     break;
                 }
             }
+        } else {
+            passed = false;
         }
         __threadfence();
+        if (passed && atomicAdd(bar + 1, 1u) + 1u == gridDim.x) {
+            bar[0] = 0u;
+            bar[1] = 0u;
+        }
     }
     __syncthreads();
     return *abort_flag == 0;
 }
 
-// One streaming pass.  Every warp calls it; roles: warp 0 TMA producer, warp 1 UMMA issuer,
-// warps 2..5 epilogue.  s_union / n_union: groups in U (shared memory).
-__device__ void stream_phase(int mode, const DecodeArgs& a, const CUtensorMap* tmW0, const CUtensorMap* tmW1,
-                             const CUtensorMap* tmAct, Pipe& P, const int* s_union, int n_union) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ksub = a.G / kBKD;
-    int n_items;
+struct PassGeom {
+    int n_blocks, spb, total, L;
+};
+
+__device__ __forceinline__ PassGeom geom_of(int mode, const DecodeArgs& a, int n_union) {
+    PassGeom g;
     if (mode == MODE_GATEUP) {
-        n_items = n_union * a.blocks_per_group * 2 * a.ksplit;
+        g.n_blocks = n_union * a.blocks_per_group * 2;   // block index = (slot * bpg + blk) * 2 + mat
+        g.spb = a.D / kBKD;
     } else {
-        const int n_chunks = (n_union + a.groups_per_item - 1) / a.groups_per_item;
-        n_items = a.row_tiles * n_chunks;
+        g.n_blocks = a.row_tiles;
+        g.spb = n_union * (a.G / kBKD);
     }
+    g.total = g.n_blocks * g.spb;
+    g.L = (g.total + gridDim.x - 1) / gridDim.x;
+    if (g.L < 1) g.L = 1;
+    return g;
+}
+
+// Producer side of one pass (single thread).  `pre` stages of this pass may already hold their
+// weight tile (issued before the grid barrier); for those only the activation tile is loaded.
+__device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* tmW0, const CUtensorMap* tmW1,
+                             const CUtensorMap* tmAct, Pipe& P, const int* s_union, int n_union, int weights_only_steps,
+                             int skip_weight_steps) {
+    const PassGeom g = geom_of(mode, a, n_union);
+    const int ksub = a.G / kBKD;
     const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
     const uint32_t stage_tx = static_cast<uint32_t>(rows_valid * kBKD * 2 + a.NT * kBKD * 2);
-
-    struct Item { int mat, row0, nsteps, col0, u0; };
-    auto decode_item = [&](int item) {
-        Item it;
+    Share sh(blockIdx.x, g.total, g.L, g.spb);
+    Segment sg;
+    int step = 0;
+    int n = P.n;
+    while (sh.next(sg)) {
+        int row0, mat = 0;
         if (mode == MODE_GATEUP) {
-            const int ks = item % a.ksplit;
-            int r = item / a.ksplit;
-            it.mat = r & 1;
-            r >>= 1;
-            const int blk = r % a.blocks_per_group, u = r / a.blocks_per_group;
-            it.row0 = s_union[u] * a.G + blk * kRows;
-            it.nsteps = a.kchunk / kBKD;
-            it.col0 = ks * a.kchunk;
-            it.u0 = 0;
+            mat = sg.blk & 1;
+            const int r = sg.blk >> 1;
+            row0 = s_union[r / a.blocks_per_group] * a.G + (r % a.blocks_per_group) * kRows;
         } else {
-            const int rt = item % a.row_tiles, ch = item / a.row_tiles;
-            it.mat = 0;
-            it.row0 = rt * kRows;
-            it.u0 = ch * a.groups_per_item;
-            it.nsteps = min(a.groups_per_item, n_union - it.u0) * ksub;
-            it.col0 = 0;
+            row0 = sg.blk * kRows;
         }
-        return it;
-    };
-    auto step_col = [&](const Item& it, int i) {
-        if (mode == MODE_GATEUP) return it.col0 + i * kBKD;
-        return s_union[it.u0 + i / ksub] * a.G + (i % ksub) * kBKD;
-    };
-
-    if (warp == 0) {
-        if (lane == 0) {
-            fence_proxy_async_all();  // activations written by other CTAs before the last grid barrier
-            bool ok = *P.abort_flag == 0;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const Item it = decode_item(item);
-                const CUtensorMap* tw = it.mat ? tmW1 : tmW0;
-                for (int i = 0; i < it.nsteps; ++i, ++P.n) {
-                    const int s = P.n % kStagesD;
-                    const uint32_t ph = (P.n / kStagesD) & 1;
-                    if (!mbar_wait(P.empty + 8 * s, ph ^ 1u, a.wait_ns, P.abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(P.full + 8 * s, stage_tx);
-                    const uint32_t dst = smem_u32(P.base + s * kStageBytesD);
-                    const int col = step_col(it, i);
-                    tma_load_2d(dst, tw, col, it.row0, P.full + 8 * s);
-                    tma_load_2d(dst + kWBytes, tmAct, col, 0, P.full + 8 * s);
-                }
+        const CUtensorMap* tw = mat ? tmW1 : tmW0;
+        for (int i = 0; i < sg.nsteps; ++i, ++step, ++n) {
+            if (weights_only_steps >= 0 && step >= weights_only_steps) return true;  // pre-issue done
+            const int ks = sg.k0 + i;
+            const int col = mode == MODE_GATEUP ? ks * kBKD : s_union[ks / ksub] * a.G + (ks % ksub) * kBKD;
+            const int s = n % kStagesD;
+            const uint32_t dst = smem_u32(P.base + s * kStageBytesD);
+            if (step >= skip_weight_steps) {
+                const uint32_t ph = (n / kStagesD) & 1;
+                if (!mbar_wait(P.empty + 8 * s, ph ^ 1u, a.wait_ns, P.abort_flag)) return false;
+                mbar_arrive_expect_tx(P.full + 8 * s, stage_tx);
+                tma_load_2d(dst, tw, col, row0, P.full + 8 * s);
             }
-            if (!ok) {
-                atomicExch(a.status, WIDE_ERR_TIMEOUT);
-                for (int i = 0; i < 64; ++i) __nanosleep(1000);
-            }
+            if (weights_only_steps < 0) tma_load_2d(dst + kWBytes, tmAct, col, 0, P.full + 8 * s);
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(kRows, a.NT);
-            bool ok = *P.abort_flag == 0;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++P.tc) {
-                const Item it = decode_item(item);
-                const int buf = P.tc & 1;
-                const uint32_t tph = (P.tc >> 1) & 1;
-                if (!mbar_wait(P.tempty + 8 * buf, tph ^ 1u, a.wait_ns, P.abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d_tmem = P.tmem_base + buf * kAccColsD;
-                for (int i = 0; i < it.nsteps; ++i, ++P.n) {
-                    const int s = P.n % kStagesD;
-                    const uint32_t ph = (P.n / kStagesD) & 1;
-                    if (!mbar_wait(P.full + 8 * s, ph, a.wait_ns, P.abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t w_addr = smem_u32(P.base + s * kStageBytesD);
-                    const uint64_t adesc = umma_desc_sw128(w_addr);
-                    const uint64_t bdesc = umma_desc_sw128(w_addr + kWBytes);
-#pragma unroll
-                    for (int k4 = 0; k4 < kBKD / 16; ++k4)
-                        umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
-                    umma_commit(P.empty + 8 * s);
-                }
-                if (ok) umma_commit(P.tfull + 8 * buf);
-            }
-            if (!ok) atomicExch(a.status, WIDE_ERR_TIMEOUT);
-        }
-    } else {
-        const int q = warp & 3;
-        bool ok = *P.abort_flag == 0;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++P.tc) {
-            const Item it = decode_item(item);
-            const int rloc = q * 32 + lane;
-            const int row = it.row0 + rloc;
-            const int rows_total = mode == MODE_GATEUP ? a.inner : a.D;
-            const bool live = rloc < rows_valid && row < rows_total;
-            float* out = mode == MODE_GATEUP ? (it.mat ? a.up : a.gate) : a.yacc;
-            const long long ldo = mode == MODE_GATEUP ? a.inner : a.D;
-            const int buf = P.tc & 1;
-            const uint32_t tph = (P.tc >> 1) & 1;
-            if (!mbar_wait(P.tfull + 8 * buf, tph, a.wait_ns, P.abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            const uint32_t taddr = P.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccColsD;
-            for (int c0 = 0; c0 < a.NT; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld_32x16(taddr + c0, r);
-                tmem_ld_wait();
-                if (live) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c0 + i < a.B) red_add_f32(out + (c0 + i) * ldo + row, __uint_as_float(r[i]));
-                }
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(P.tempty + 8 * buf);
-        }
-        if (!ok && lane == 0) atomicExch(a.status, WIDE_ERR_TIMEOUT);
     }
+    if (weights_only_steps < 0) P.n = n;
+    return true;
+}
+
+__device__ bool mma_pass(int mode, const DecodeArgs& a, Pipe& P, int n_union) {
+    const PassGeom g = geom_of(mode, a, n_union);
+    const uint32_t idesc = umma_idesc_bf16(kRows, a.NT);
+    Share sh(blockIdx.x, g.total, g.L, g.spb);
+    Segment sg;
+    while (sh.next(sg)) {
+        const int buf = P.tc & 1;
+        const uint32_t tph = (P.tc >> 1) & 1;
+        if (!mbar_wait(P.tempty + 8 * buf, tph ^ 1u, a.wait_ns, P.abort_flag)) return false;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = P.tmem_base + buf * kAccColsD;
+        for (int i = 0; i < sg.nsteps; ++i, ++P.n) {
+            const int s = P.n % kStagesD;
+            const uint32_t ph = (P.n / kStagesD) & 1;
+            if (!mbar_wait(P.full + 8 * s, ph, a.wait_ns, P.abort_flag)) return false;
+            tc_fence_after_sync();
+            const uint32_t w_addr = smem_u32(P.base + s * kStageBytesD);
+            const uint64_t adesc = umma_desc_sw128(w_addr);
+            const uint64_t bdesc = umma_desc_sw128(w_addr + kWBytes);
+#pragma unroll
+            for (int k4 = 0; k4 < kBKD / 16; ++k4)
+                umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (i > 0 || k4 > 0) ? 1u : 0u);
+            umma_commit(P.empty + 8 * s);
+        }
+        umma_commit(P.tfull + 8 * buf);
+        ++P.tc;
+    }
+    return true;
+}
+
+// Epilogue warps (4 warps, 128 threads; thread e = row e of the tile).
+__device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int* s_union, int n_union, int* s_flag,
+                              unsigned* s_tokmask) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q = warp & 3;
+    const int e = (warp - 2) * 32 + lane;  // 0..127, unique per epilogue thread
+    const PassGeom g = geom_of(mode, a, n_union);
+    const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
+    const int nb4 = (a.B + 3) / 4;  // 16-byte pieces of a row that hold real tokens
+    Share sh(blockIdx.x, g.total, g.L, g.spb);
+    Segment sg;
+    while (sh.next(sg)) {
+        int row0, mat = 0, slot_blk = 0;
+        if (mode == MODE_GATEUP) {
+            mat = sg.blk & 1;
+            slot_blk = sg.blk >> 1;
+            row0 = s_union[slot_blk / a.blocks_per_group] * a.G + (slot_blk % a.blocks_per_group) * kRows;
+        } else {
+            row0 = sg.blk * kRows;
+        }
+        const int rloc = q * 32 + lane;
+        const int row = row0 + rloc;
+        const int rows_total = mode == MODE_GATEUP ? a.inner : a.D;
+        const bool live = rloc < rows_valid && row < rows_total;
+        float* out = (mode == MODE_GATEUP ? (mat ? a.up : a.gate) : a.yacc) + static_cast<size_t>(row) * a.NT;
+        const int buf = P.tc & 1;
+        const uint32_t tph = (P.tc >> 1) & 1;
+        if (!mbar_wait(P.tfull + 8 * buf, tph, a.wait_ns, P.abort_flag)) return false;
+        tc_fence_after_sync();
+        const uint32_t taddr = P.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccColsD;
+        for (int c0 = 0; c0 < a.NT; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld_32x16(taddr + c0, r);
+            tmem_ld_wait();
+            if (live) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    if (c0 / 4 + v < nb4)
+                        red_add_v4(out + c0 + 4 * v, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+            }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(P.tempty + 8 * buf);
+        ++P.tc;
+
+        // ticket: has every piece of this block been added?
+        __threadfence();
+        epilogue_bar_sync();
+        if (e == 0) {
+            unsigned* tk;
+            int expected;
+            if (mode == MODE_GATEUP) {
+                tk = a.tickets1 + slot_blk;
+                expected = pieces_of_block(2 * slot_blk, g.spb, g.L) + pieces_of_block(2 * slot_blk + 1, g.spb, g.L);
+            } else {
+                tk = a.tickets2 + sg.blk;
+                expected = pieces_of_block(sg.blk, g.spb, g.L);
+            }
+            const unsigned done = atomicAdd(tk, 1u) + 1u;
+            const int last = done == static_cast<unsigned>(expected);
+            if (last) *tk = 0u;
+            *s_flag = last;
+            __threadfence();
+        }
+        epilogue_bar_sync();
+        if (*s_flag) {
+            constexpr int kB4 = 4;  // 16-byte pieces per round: 2 * kB4 loads in flight per thread
+            if (mode == MODE_GATEUP) {
+                // h[b, ch] for the 128 (or G) channels of this block; re-zero gate / up
+                const int gidx = s_union[slot_blk / a.blocks_per_group];
+                // which tokens execute this group: thread e < 64 looks at token e
+                const bool tb = e < a.B && wide_mask_bit(a.mask_bits, a.words, e, gidx);
+                const unsigned vote = __ballot_sync(0xffffffffu, tb);
+                if (lane == 0 && e < 64) s_tokmask[e >> 5] = vote;
+                epilogue_bar_sync();
+                const unsigned long long tokmask =
+                    static_cast<unsigned long long>(s_tokmask[0]) | (static_cast<unsigned long long>(s_tokmask[1]) << 32);
+                const int ch = gidx * a.G + (slot_blk % a.blocks_per_group) * kRows + e;
+                if (e < rows_valid) {
+                    float4* gp = reinterpret_cast<float4*>(a.gate + static_cast<size_t>(ch) * a.NT);
+                    float4* up = reinterpret_cast<float4*>(a.up + static_cast<size_t>(ch) * a.NT);
+                    for (int b0 = 0; b0 < nb4; b0 += kB4) {
+                        float4 gv[kB4], uv[kB4];
+#pragma unroll
+                        for (int j = 0; j < kB4; ++j) {
+                            if (b0 + j < nb4) {
+                                gv[j] = __ldcg(gp + b0 + j);
+                                uv[j] = __ldcg(up + b0 + j);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < kB4; ++j) {
+                            if (b0 + j < nb4) {
+                                gp[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                up[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                const float gs[4] = {gv[j].x, gv[j].y, gv[j].z, gv[j].w};
+                                const float us[4] = {uv[j].x, uv[j].y, uv[j].z, uv[j].w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int b = 4 * (b0 + j) + i;
+                                    if (b < a.B) {
+                                        const float v = ((tokmask >> b) & 1ull) ? gs[i] / (1.f + __expf(-gs[i])) * us[i] : 0.f;
+                                        a.h[static_cast<size_t>(b) * a.inner + ch] = __float2bfloat16_rn(v);
+                                    }
+                                }
+                            }
+                        }
+                    }
+                }
+            } else {
+                const int orow = sg.blk * kRows + e;
+                if (orow < a.D) {
+                    float4* yp = reinterpret_cast<float4*>(a.yacc + static_cast<size_t>(orow) * a.NT);
+                    for (int b0 = 0; b0 < nb4; b0 += 2 * kB4) {
+                        float4 v[2 * kB4];
+#pragma unroll
+                        for (int j = 0; j < 2 * kB4; ++j)
+                            if (b0 + j < nb4) v[j] = __ldcg(yp + b0 + j);
+#pragma unroll
+                        for (int j = 0; j < 2 * kB4; ++j) {
+                            if (b0 + j < nb4) {
+                                yp[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                const float vs[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int b = 4 * (b0 + j) + i;
+                                    if (b < a.B) {
+                                        const size_t o = static_cast<size_t>(b) * a.D + orow;
+                                        if (a.out_bf16) static_cast<__nv_bfloat16*>(a.y)[o] = __float2bfloat16_rn(vs[i]);
+                                        else static_cast<float*>(a.y)[o] = vs[i];
+                                    }
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        epilogue_bar_sync();  // s_flag is rewritten by the next segment
+    }
+    return true;
 }
 
 __global__ void __launch_bounds__(kThreadsD, 1)
@@ -244,6 +388,8 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     __shared__ int s_union[WIDE_MAX_GROUPS];
     __shared__ int s_nunion;
+    __shared__ int s_flag;
+    __shared__ unsigned s_tokmask[2];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStagesD * kStageBytesD);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStagesD + 4);
@@ -274,7 +420,6 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
         prefetch_tmap(&tmX);
         prefetch_tmap(&tmWd);
         prefetch_tmap(&tmH);
-        if (blockIdx.x == 0) a.bar[2] = 0u;  // last barrier of the previous call; nobody is near it yet
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 2 * kAccColsD);
@@ -303,58 +448,62 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
     const long long gtid = static_cast<long long>(blockIdx.x) * kThreadsD + tid;
     const long long gthreads = static_cast<long long>(gridDim.x) * kThreadsD;
 
-    // ---- phase 1
-    if (a.is_ffn) {
-        stream_phase(MODE_GATEUP, a, &tmG, &tmU, &tmX, P, s_union, n_union);
-    } else {
-        const int vec_per_row = a.inner / 8, vec_per_group = a.G / 8;
-        const uint4* src = reinterpret_cast<const uint4*>(a.act_in);
-        uint4* dst = reinterpret_cast<uint4*>(a.h);
-        for (long long i = gtid; i < static_cast<long long>(a.B) * vec_per_row; i += gthreads) {
-            const int t = static_cast<int>(i / vec_per_row);
-            const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
-            dst[i] = wide_mask_bit(a.mask_bits, a.words, t, g) ? src[i] : make_uint4(0u, 0u, 0u, 0u);
-        }
-    }
-    grid_barrier(a.bar + 0, a.wait_ns, P.abort_flag, a.status);
-
-    // ---- phase 2: activation (FFN only); consumes and re-zeroes the gate/up accumulators
-    if (a.is_ffn) {
-        if (!*P.abort_flag) {
-            const int per_group = a.B * a.G;  // elements of one group: b-major, c fastest
-            const int total = n_union * per_group;
-            for (long long i = gtid; i < total; i += gthreads) {
-                const int u = static_cast<int>(i) / per_group;
-                const int rem = static_cast<int>(i) - u * per_group;
-                const int b = rem / a.G, c = rem - b * a.G;
-                const int g = s_union[u];
-                const size_t idx = static_cast<size_t>(b) * a.inner + static_cast<size_t>(g) * a.G + c;
-                const float gv = __ldcg(a.gate + idx), uv = __ldcg(a.up + idx);
-                a.gate[idx] = 0.f;
-                a.up[idx] = 0.f;
-                const float v = wide_mask_bit(a.mask_bits, a.words, b, g) ? gv / (1.f + __expf(-gv)) * uv : 0.f;
-                a.h[idx] = __float2bfloat16_rn(v);
-            }
-        }
-        grid_barrier(a.bar + 1, a.wait_ns, P.abort_flag, a.status);
-    }
-
-    // ---- phase 3: down / output projection
-    stream_phase(MODE_DOWN, a, &tmWd, &tmWd, &tmH, P, s_union, n_union);
-    grid_barrier(a.bar + 2, a.wait_ns, P.abort_flag, a.status);
-
-    // ---- phase 4: write the output, leave the accumulator zero
-    if (blockIdx.x == 0 && tid == 0) {
-        a.bar[0] = 0u;
-        a.bar[1] = 0u;
-    }
-    if (!*P.abort_flag) {
+    if (n_union == 0) {
+        // nothing is active: the output is exactly zero and no accumulator was touched
         const long long n = static_cast<long long>(a.B) * a.D;
         for (long long i = gtid; i < n; i += gthreads) {
-            const float v = __ldcg(a.yacc + i);
-            a.yacc[i] = 0.f;
-            if (a.out_bf16) static_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(v);
-            else static_cast<float*>(a.y)[i] = v;
+            if (a.out_bf16) static_cast<__nv_bfloat16*>(a.y)[i] = __float2bfloat16_rn(0.f);
+            else static_cast<float*>(a.y)[i] = 0.f;
+        }
+    } else {
+        bool ok = true;
+        int pre = 0;  // stages of pass 2 whose weight tile was issued before the barrier
+        // ---- pass 1
+        if (a.is_ffn) {
+            if (warp == 0) {
+                if (lane == 0) {
+                    ok = produce_pass(MODE_GATEUP, a, &tmG, &tmU, &tmX, P, s_union, n_union, -1, 0);
+                    if (ok) {
+                        // fill the ring with this CTA's first W_down tiles while the others finish
+                        const PassGeom g2 = geom_of(MODE_DOWN, a, n_union);
+                        const int mine = max(0, min((static_cast<int>(blockIdx.x) + 1) * g2.L, g2.total) -
+                                                    min(static_cast<int>(blockIdx.x) * g2.L, g2.total));
+                        pre = min(kStagesD, mine);
+                        ok = produce_pass(MODE_DOWN, a, &tmWd, &tmWd, &tmH, P, s_union, n_union, pre, 0);
+                    }
+                }
+            } else if (warp == 1) {
+                if (lane == 0) ok = mma_pass(MODE_GATEUP, a, P, n_union);
+            } else {
+                ok = epilogue_pass(MODE_GATEUP, a, P, s_union, n_union, &s_flag, s_tokmask);
+            }
+        } else {
+            const int vec_per_row = a.inner / 8, vec_per_group = a.G / 8;
+            const uint4* src = reinterpret_cast<const uint4*>(a.act_in);
+            uint4* dst = reinterpret_cast<uint4*>(a.h);
+            for (long long i = gtid; i < static_cast<long long>(a.B) * vec_per_row; i += gthreads) {
+                const int t = static_cast<int>(i / vec_per_row);
+                const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
+                dst[i] = wide_mask_bit(a.mask_bits, a.words, t, g) ? src[i] : make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        if (!ok && lane == 0) atomicExch(a.status, WIDE_ERR_TIMEOUT);
+        grid_barrier(a.bar, a.wait_ns, P.abort_flag, a.status);
+
+        // ---- pass 2
+        if (!*P.abort_flag) {
+            if (warp == 0) {
+                if (lane == 0) {
+                    fence_proxy_async_all();  // h was written through the generic proxy by other CTAs
+                    ok = produce_pass(MODE_DOWN, a, &tmWd, &tmWd, &tmH, P, s_union, n_union, -1, pre);
+                    if (!ok) for (int i = 0; i < 64; ++i) __nanosleep(1000);
+                }
+            } else if (warp == 1) {
+                if (lane == 0) ok = mma_pass(MODE_DOWN, a, P, n_union);
+            } else {
+                ok = epilogue_pass(MODE_DOWN, a, P, s_union, n_union, &s_flag, s_tokmask);
+            }
+            if (!ok && lane == 0) atomicExch(a.status, WIDE_ERR_TIMEOUT);
         }
     }
 
@@ -384,12 +533,6 @@ bool make_tmap(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t
 
 constexpr int kSmemD = kStagesD * kStageBytesD + (2 * kStagesD + 4) * 8 + 16 + 1024;
 
-int pick_kchunk(int D) {
-    for (int kc = 512; kc >= 64; kc >>= 1)
-        if (D % kc == 0) return kc;
-    return 64;
-}
-
 int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a, const void* wg, const void* wu,
                   const void* wd, int B, int D, int inner, int G, const uint32_t* mask_bits, void* y, int out_dtype,
                   void* ws) {
@@ -406,10 +549,7 @@ int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a
     a.words = (a.NG + 31) / 32;
     a.rows_valid = G < kRows ? G : kRows;
     a.blocks_per_group = G / kRows > 0 ? G / kRows : 1;
-    a.kchunk = pick_kchunk(D);
-    a.ksplit = D / a.kchunk;
     a.row_tiles = (D + kRows - 1) / kRows;
-    a.groups_per_item = 512 / G > 0 ? 512 / G : 1;
     a.mask_bits = mask_bits;
     a.act_in = static_cast<const __nv_bfloat16*>(x_or_a);
     a.gate = ctx->decode_acc;
@@ -418,7 +558,9 @@ int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a
     a.h = static_cast<__nv_bfloat16*>(ws);
     a.y = y;
     a.out_bf16 = out_dtype == WIDE_BF16 ? 1 : 0;
-    a.bar = reinterpret_cast<unsigned*>(ctx->d_status + 4);
+    a.bar = reinterpret_cast<unsigned*>(ctx->d_status) + 4;
+    a.tickets1 = ctx->d_tickets;
+    a.tickets2 = ctx->d_tickets + 1024;
     a.status = ctx->d_status;
     a.wait_ns = ctx->wait_ns;
 
@@ -436,7 +578,7 @@ int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemD));
     void* params[] = {&tmG, &tmU, &tmX, &tmWd, &tmH, &a};
     WideLaunch l(ctx, s, is_ffn ? "decode_ffn_fused" : "decode_oproj_fused");
-    // cooperative: the grid barriers need every CTA resident (one per SM)
+    // cooperative: the grid barrier needs every CTA resident (one per SM)
     WIDE_CUDA_CHECK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_fused_kernel), dim3(ctx->sm_count),
                                                 dim3(kThreadsD), params, kSmemD, s));
     return WIDE_OK;
