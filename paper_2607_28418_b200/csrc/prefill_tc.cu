@@ -6,7 +6,8 @@
 //                  pair of the reordered mask.  A = 128 gathered rows of X, B = the group's rows of
 //                  W_gate and W_up side by side (one UMMA of N = 2*BN), fp32 accumulators in TMEM,
 //                  epilogue silu(gate)*up -> bf16, scattered through the permutation straight into
-//                  the token-major hidden activation H (rows past the group's count are dropped).
+//                  the token-major hidden activation H (rows past the group's count are dropped);
+//                  the same warps zero the group's inactive rows of H.
 //   down_kernel    Eq. 10 (K-axis) in owner-computes form: a CTA owns a 128-token x BN output tile
 //                  in original token order and walks the K-groups, skipping every group that no
 //                  token of the tile selected (block-level predicate on the unsorted mask);
@@ -445,6 +446,23 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             const bool live = j < counts[g];
             const int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
             __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN;
+            {
+                // While the MMAs of this item run: zero this item's share of the group's INACTIVE
+                // rows of H (sorted positions [c, T) split evenly over the group's active tiles),
+                // so that the down projection reads exact zeros for every inactive (token, group)
+                // pair of a group that is active anywhere.  Groups nobody selected are never read.
+                const int c = counts[g];
+                const int nt = (c + kBM - 1) / kBM;
+                const int per = (T - c + nt - 1) / nt;
+                const int j0 = c + m * per;
+                const int j1 = min(T, j0 + per);
+                for (int jj = j0 + (warp - 6) * 32 + lane; jj < j1; jj += 128) {
+                    const int tz = perm[static_cast<size_t>(g) * T + jj];
+                    uint4* z = reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN);
+#pragma unroll
+                    for (int v = 0; v < BN / 8; ++v) z[v] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
             const int buf = tc & 1;
             const uint32_t tph = (tc >> 1) & 1;
             if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
@@ -561,11 +579,8 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const int32_t* perm, const int32_t* counts, const int32_t* work_list,
                                const int32_t* n_work, void* y, int out_dtype, void* h) {
     if (T == 0) return WIDE_OK;
-    // inactive (token, group) pairs of H must read as zero in the down projection
-    {
-        WideLaunch l(ctx, s, "prefill_zero_h");
-        WIDE_CUDA_CHECK(cudaMemsetAsync(h, 0, static_cast<size_t>(T) * Dff * 2, s));
-    }
+    // inactive (token, group) pairs of H must read as zero in the down projection: the gate/up
+    // kernel's epilogue warps write those zeros themselves
     int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h)
                        : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h);
     if (rc != WIDE_OK) return rc;

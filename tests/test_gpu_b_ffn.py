@@ -78,6 +78,7 @@ def test_prefill_tc_matches_oracle(ctx, T, D, Dff, G, k):
 def test_prefill_tc_fp32_output_and_variable_budget(ctx):
     from paper_2607_28418_b200 import binding
     cfg = synth.WideConfig("t", tokens=384, hidden=512, d_ff=1024, group=128, k=4)
+    ctx.workspace(1 << 20).fill_(0xFF)              # stale scratch (NaN patterns) must not leak into y
     mask = synth.bernoulli_mask(3, 384, 8, 0.4)     # variable active groups per token
     mask[5] = False                                  # a token with nothing active -> zero row
     mask[:, 6] = False                               # a group nobody selects -> skipped block column
