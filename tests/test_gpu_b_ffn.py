@@ -75,6 +75,18 @@ def test_prefill_tc_matches_oracle(ctx, T, D, Dff, G, k):
     assert_close(y, ref, f"prefill tc {T}x{D}x{Dff} G{G}")
 
 
+@pytest.mark.parametrize("T,D,Dff,G,k,out", [(1280, 4096, 256, 128, 1, None), (1100, 4096, 512, 64, 5, torch.float32)])
+def test_prefill_tc_more_tiles_than_sms(ctx, T, D, Dff, G, k, out):
+    """More output tiles than SMs with a ragged remainder (both tile heights of the down
+    projection get exercised across the parametrisations); run twice: same result."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=T, hidden=D, d_ff=Dff, group=G, k=k)
+    y1, ref, _ = _run_ffn(ctx, cfg, 8, binding.FLAG_FORCE_PREFILL, out_dtype=out)
+    assert_close(y1, ref, f"many tiles {T}x{D}x{Dff}")
+    y2, _, _ = _run_ffn(ctx, cfg, 8, binding.FLAG_FORCE_PREFILL, out_dtype=out)
+    assert_close(y2, ref, f"many tiles, second call {T}x{D}x{Dff}")
+
+
 def test_prefill_tc_fp32_output_and_variable_budget(ctx):
     from paper_2607_28418_b200 import binding
     cfg = synth.WideConfig("t", tokens=384, hidden=512, d_ff=1024, group=128, k=4)
