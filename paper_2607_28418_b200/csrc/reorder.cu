@@ -12,7 +12,25 @@ __device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_
                                int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
                                int32_t* __restrict__ offsets);
 
-// One CTA per group: pass 1 counts the active rows, pass 2 places every row.
+// One CTA per group.  Every thread owns kPerThread consecutive tokens of a chunk, so a token's
+// rank among the active rows is (active rows in earlier chunks) + (exclusive prefix over threads)
+// + (bits below it in the thread's own nibble): one warp scan and one 16-entry block scan per
+// chunk.  The group's total is needed before the inactive rows can be placed, so the counting
+// sweep runs first (its loads stay in L1 for the placing sweep).
+constexpr int kPerThread = 4;
+constexpr int kChunk = kPartThreads * kPerThread;
+
+__device__ __forceinline__ unsigned load_nibble(const uint32_t* __restrict__ mask_bits, int words, int w, int b,
+                                                int t0, int T) {
+    unsigned nib = 0;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+        const int t = t0 + i;
+        if (t < T) nib |= ((mask_bits[static_cast<size_t>(t) * words + w] >> b) & 1u) << i;
+    }
+    return nib;
+}
+
 __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t* __restrict__ mask_bits, int T,
                                                                  int NG, int words, int32_t* __restrict__ perm,
                                                                  int32_t* counts, int tile_m, int n_tiles,
@@ -30,8 +48,9 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t*
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int nwarps = kPartThreads / 32;
 
+    // sweep 1: total number of active rows
     int local = 0;
-    for (int t = tid; t < T; t += kPartThreads) local += (mask_bits[static_cast<size_t>(t) * words + w] >> b) & 1u;
+    for (int c0 = 0; c0 < T; c0 += kChunk) local += __popc(load_nibble(mask_bits, words, w, b, c0 + tid * kPerThread, T));
     local = __reduce_add_sync(0xffffffffu, local);
     if (lane == 0) warp_cnt[warp] = local;
     __syncthreads();
@@ -44,27 +63,39 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t*
     __syncthreads();
     const int total = s_total;
 
+    // sweep 2: place every row
     int32_t* out = perm + static_cast<size_t>(g) * T;
-    int base = 0;  // active rows before this chunk
-    for (int t0 = 0; t0 < T; t0 += kPartThreads) {
-        const int t = t0 + tid;
-        const unsigned bit = (t < T) ? ((mask_bits[static_cast<size_t>(t) * words + w] >> b) & 1u) : 0u;
-        const unsigned vote = __ballot_sync(0xffffffffu, bit);
-        __syncthreads();  // warp_cnt from the previous round has been consumed
-        if (lane == 0) warp_cnt[warp] = __popc(vote);
+    int base = 0;  // active rows in earlier chunks
+    for (int c0 = 0; c0 < T; c0 += kChunk) {
+        const int t0 = c0 + tid * kPerThread;
+        const unsigned nib = load_nibble(mask_bits, words, w, b, t0, T);
+        const int mine = __popc(nib);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        __syncthreads();  // warp_cnt of the previous round (or of sweep 1) has been consumed
+        if (lane == 31) warp_cnt[warp] = incl;
         __syncthreads();
-        int before = 0, chunk = 0;
+        int before = 0, chunk_total = 0;
+#pragma unroll
         for (int i = 0; i < nwarps; ++i) {
             const int c = warp_cnt[i];
             before += (i < warp) ? c : 0;
-            chunk += c;
+            chunk_total += c;
         }
-        const int rank = base + before + __popc(vote & ((1u << lane) - 1u));  // active rows before t
-        if (t < T) {
-            if (bit) out[rank] = t;
-            else out[total + (t - rank)] = t;
+        int rank = base + before + incl - mine;  // active rows before token t0
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            const int t = t0 + i;
+            if (t < T) {
+                if ((nib >> i) & 1u) out[rank++] = t;
+                else out[total + (t - rank)] = t;
+            }
         }
-        base += chunk;
+        base += chunk_total;
     }
 
     // The CTA that finishes last has every group's count in view and builds the rest.
@@ -93,21 +124,34 @@ __device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_
     const int tid = threadIdx.x;
     for (int g = tid; g < NG; g += blockDim.x) s_tiles[g] = (__ldcg(counts + g) + tile_m - 1) / tile_m;
     __syncthreads();
-    if (tid == 0) {
-        int woff = 0, uoff = 0, roff = 0;
-        for (int g = 0; g < NG; ++g) {
-            s_work_off[g] = woff;
-            s_union_pos[g] = uoff;
-            offsets[g] = roff;
-            woff += s_tiles[g];
-            uoff += __ldcg(counts + g) > 0 ? 1 : 0;
-            roff += s_tiles[g] * tile_m;
+    if (tid < 32) {
+        // exclusive prefix sums over the groups, 32 at a time
+        int woff = 0, uoff = 0;
+        for (int g0 = 0; g0 < NG; g0 += 32) {
+            const int g = g0 + tid;
+            const int tv = g < NG ? s_tiles[g] : 0;
+            const int uv = (g < NG && __ldcg(counts + g) > 0) ? 1 : 0;
+            int tp = tv, up = uv;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a = __shfl_up_sync(0xffffffffu, tp, o), c = __shfl_up_sync(0xffffffffu, up, o);
+                if (tid >= o) { tp += a; up += c; }
+            }
+            if (g < NG) {
+                s_work_off[g] = woff + tp - tv;
+                s_union_pos[g] = uoff + up - uv;
+                offsets[g] = (woff + tp - tv) * tile_m;
+            }
+            woff += __shfl_sync(0xffffffffu, tp, 31);
+            uoff += __shfl_sync(0xffffffffu, up, 31);
         }
-        s_work_off[NG] = woff;
-        s_union_pos[NG] = uoff;
-        offsets[NG] = roff;
-        *n_work = woff;
-        *n_union = uoff;
+        if (tid == 0) {
+            s_work_off[NG] = woff;
+            s_union_pos[NG] = uoff;
+            offsets[NG] = woff * tile_m;
+            *n_work = woff;
+            *n_union = uoff;
+        }
     }
     __syncthreads();
     const int total_work = s_work_off[NG], total_union = s_union_pos[NG];

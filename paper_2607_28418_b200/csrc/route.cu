@@ -161,6 +161,7 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
                    float* __restrict__ scores_out) {
     extern __shared__ uint4 sh_x[];  // [D / 8]
     __shared__ float s[WIDE_MAX_GROUPS];
+    __shared__ __align__(16) unsigned long long skey[WIDE_MAX_GROUPS + 2];  // (ordered score bits, NG - index)
     __shared__ double ex[WIDE_MAX_GROUPS];
     __shared__ int band[WIDE_MAX_GROUPS];
     __shared__ float red[2 * kSelWarps];
@@ -182,8 +183,14 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
             float v = 0.f;
             for (int ks = 0; ks < nsplit; ++ks) v += scores[ks * slab + static_cast<size_t>(t) * ld + g];
             s[g] = v;
+            // total order "score descending, index ascending" as one unsigned 64-bit compare
+            const uint32_t u = __float_as_uint(v + 0.0f);  // -0 -> +0
+            const uint32_t ord = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+            skey[g] = (static_cast<unsigned long long>(ord) << 32) | static_cast<uint32_t>(NG - g);
             wmax = fmaxf(wmax, wnorm[g]);
             if (scores_out) scores_out[static_cast<size_t>(t) * NG + g] = v;
+        } else if (g < NG + 2) {
+            skey[g] = 0ull;  // padding: beats nobody
         }
     }
     const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
@@ -236,10 +243,13 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
         const int g = tid + q * kThreads;
         if (g < NG) {
             const float v = s[g];
+            const unsigned long long mine = skey[g];
             int beats = 0;
-            for (int h = 0; h < NG; ++h) {
-                const float u = s[h];
-                beats += (u > v) || (u == v && h < g);
+            const ulonglong2* kp = reinterpret_cast<const ulonglong2*>(skey);
+#pragma unroll 4
+            for (int h = 0; h < (NG + 1) / 2; ++h) {
+                const ulonglong2 kk = kp[h];
+                beats += (kk.x > mine) + (kk.y > mine);
             }
             rank[q] = beats;
             if (beats == kt - 1) sh_b[0] = v;
