@@ -245,6 +245,29 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
     const PassGeom g = geom_of(mode, a, n_union);
     const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
     const int nb4 = (a.B + 3) / 4;  // 16-byte pieces of a row that hold real tokens
+    {
+        // Warm L2 with the accumulator rows this CTA will add to (they may have been evicted since
+        // the previous call zeroed them), so the red.adds at the end of the pass hit L2.
+        Share pre(blockIdx.x, g.total, g.L, g.spb);
+        Segment ps;
+        while (pre.next(ps)) {
+            int prow;
+            float* pbase;
+            if (mode == MODE_GATEUP) {
+                const int sb = ps.blk >> 1;
+                prow = s_union[sb / a.blocks_per_group] * a.G + (sb % a.blocks_per_group) * kRows + e;
+                pbase = (ps.blk & 1) ? a.up : a.gate;
+                if (e >= rows_valid || prow >= a.inner) continue;
+            } else {
+                prow = ps.blk * kRows + e;
+                pbase = a.yacc;
+                if (prow >= a.D) continue;
+            }
+            const char* p = reinterpret_cast<const char*>(pbase + static_cast<size_t>(prow) * a.NT);
+            for (int off = 0; off < nb4 * 16; off += 128)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p + off));
+        }
+    }
     Share sh(blockIdx.x, g.total, g.L, g.spb);
     Segment sg;
     while (sh.next(sg)) {

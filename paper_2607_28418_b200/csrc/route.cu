@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 constexpr float kAccumErr = 5.9604645e-8f;  // 2^-24 per accumulated element
 
 constexpr int kSelWarps = 4;   // tokens (warps) per CTA in select_band_kernel
-constexpr int kBatch = 8;      // 16-byte loads in flight per lane
+constexpr int kBatch = 4;      // 16-byte loads in flight per lane
 
 // Exact x_t . w_g in fp64 by one warp: x row in shared memory, w row streamed from L2 with
 // kBatch loads in flight per lane (bf16 products are exact in fp64).
@@ -154,7 +154,7 @@ __device__ __forceinline__ double warp_dot_f64(const uint4* __restrict__ xs, con
 // One CTA (4 warps) per token.  scores: nsplit partial slabs [nsplit][T, ld] that are summed on
 // load.  Thread g ranks group g (and g + 128); the exact re-scoring of the band is spread over
 // the four warps.
-__global__ void __launch_bounds__(32 * kSelWarps)
+__global__ void __launch_bounds__(32 * kSelWarps, 12)
 select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
                    const __nv_bfloat16* __restrict__ w, const float* __restrict__ wnorm, int T, int NG, int D, int k,
                    const int32_t* __restrict__ k_per_token, uint32_t* __restrict__ mask_bits,
