@@ -136,8 +136,8 @@ def reduce_max_ms(ms: float, world: int, device=None) -> float:
     return float(t.item())
 
 
-def flops_ffn_active(cfg) -> float:
-    return 6.0 * cfg.tokens * cfg.k * cfg.group * cfg.hidden
+def flops_ffn_active(cfg, oproj: bool = False) -> float:
+    return (2.0 if oproj else 6.0) * cfg.tokens * cfg.k * cfg.group * cfg.hidden
 
 
 # ------------------------------------------------------------------------------- reference arm
@@ -213,7 +213,13 @@ def run_ours(args):
     cfg = make_config(args)
     peaks = load_peaks()
     ctx = binding.Context(local)
-    case = synth.make_ffn_case(cfg, 1000 * rank)       # every rank its own token shard
+    oproj = args.op == "oproj"
+    if oproj:
+        case = synth.make_oproj_case(cfg, 1000 * rank)  # every rank its own token shard
+        case["w_router"] = case.pop("w_router_attn")
+        cfg = cfg.with_(d_ff=cfg.attn_dim, group=cfg.attn_group, k=cfg.attn_k)  # the op's inner dim / groups
+    else:
+        case = synth.make_ffn_case(cfg, 1000 * rank)
     d = {k: to_dev(v, cfg.dtype) for k, v in case.items()}
     T, NG = cfg.tokens, cfg.n_groups
     W = (NG + 31) // 32
@@ -230,11 +236,18 @@ def run_ours(args):
     # its weights from HBM although the launches run back to back without an L2 flush in between.
     n_copies = 1
     if decode and not args.flush_l2:
-        per_copy = 3 * cfg.d_ff * cfg.hidden * 2
+        per_copy = (1 if oproj else 3) * cfg.d_ff * cfg.hidden * 2
         n_copies = max(2, -(-(640 << 20) // per_copy))
-    wsets = [{k: d[k] for k in ("w_gate", "w_up", "w_down")}]
+    wkeys = ("w_o",) if oproj else ("w_gate", "w_up", "w_down")
+    wsets = [{k: d[k] for k in wkeys}]
     for _ in range(n_copies - 1):
-        wsets.append({k: d[k].clone() for k in ("w_gate", "w_up", "w_down")})
+        wsets.append({k: d[k].clone() for k in wkeys})
+
+    def main_op(x_in, w, y_out):
+        if oproj:
+            binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out)
+        else:
+            binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out)
     calls = {"n": 0}
 
     def step(k=cfg.k, slot=0, copy=None):
@@ -247,7 +260,7 @@ def run_ours(args):
         binding.wide_route(ctx, x_in, d["w_router"], NG, k, mask_bits=bits)
         if not decode:
             meta = binding.wide_reorder(ctx, bits, NG, 128, out=meta)
-        binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out)
+        main_op(x_in, w, y_out)
 
     def rotating(make):
         """One graph per weight copy; successive calls replay them in turn."""
@@ -319,8 +332,7 @@ def run_ours(args):
 
     # ---- the FFN call alone, replayed as a graph: at decode sizes the host cannot enqueue as fast
     # as the GPU runs, so event pairs recorded around direct launches would include idle time
-    run_ffn = rotating(lambda c: binding.wide_ffn(ctx, xbuf[0], wsets[c]["w_gate"], wsets[c]["w_up"],
-                                                  wsets[c]["w_down"], cfg.group, bits, meta, y=ybuf[0]))
+    run_ffn = rotating(lambda c: main_op(xbuf[0], wsets[c], ybuf[0]))
     for _ in range(n_copies):
         run_ffn()
     if flush is None:
@@ -414,7 +426,7 @@ def run_ours(args):
             union_words = np.bitwise_or.reduce(bits.cpu().numpy().view(np.uint32), axis=0)
             n_union = sum(bin(int(w)).count("1") for w in union_words)
             per_group = cfg.group * cfg.hidden * 2
-            bytes_alg = 3.0 * n_union * per_group     # gate + up + down weights of the groups in the union
+            bytes_alg = (1.0 if oproj else 3.0) * n_union * per_group   # weights of the groups in the union
             ach = bytes_alg / avg_s / 1e9
             roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": ach / peaks["hbm_gbs"],
@@ -422,7 +434,7 @@ def run_ours(args):
                                     if (dom, cfg.name) in NCU_TRAFFIC_BYTES else None),
                         "peak_source": peaks["source"], "n_union": n_union}
         else:
-            flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd}.get(dom, 6.0 * tkgd)
+            flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd}.get(dom, 2.0 * tkgd if oproj else 6.0 * tkgd)
             ach = flops_alg / avg_s / 1e12
             roofline = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
                         "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
@@ -436,7 +448,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "tokens_per_gpu": T, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
+            "config": {"workload": cfg.name, "op": args.op, "tokens_per_gpu": T, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
                        "group": cfg.group, "n_groups": NG, "k": cfg.k, "router": cfg.router,
                        "parallelism": f"token-sharded x{world}, weights replicated, no collective",
                        "l2": "flushed between steps" if flush is not None else
@@ -453,13 +465,13 @@ def run_ours(args):
             "clocks": clocks,
             "roofline": roofline,
             "kernels": kernels,
-            "ffn": {"ms": ffn_ms, "graph_ms": ffn_graph_ms, "active_tflops": flops_ffn_active(cfg) / (ffn_ms * 1e-3) / 1e12 if ffn_ms else None,
-                    "frac_of_bf16_peak": (flops_ffn_active(cfg) / (ffn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"])
+            "ffn": {"ms": ffn_ms, "graph_ms": ffn_graph_ms, "active_tflops": flops_ffn_active(cfg, oproj) / (ffn_ms * 1e-3) / 1e12 if ffn_ms else None,
+                    "frac_of_bf16_peak": (flops_ffn_active(cfg, oproj) / (ffn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"])
                     if ffn_ms else None},
             "dense": {"ms_per_step": dense_ms, "speedup_vs_dense": (dense_ms / ms_step) if dense_ms else None,
                       "ideal": NG / cfg.k if cfg.k else None},
         }
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not oproj:
             sample = min(T, args.oracle_tokens)
             v, ms = time_oracle(case, cfg, sample, 1, 0)
             line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
@@ -483,6 +495,7 @@ def main():
     ap.add_argument("--router", default="", choices=["", "random", "clustered", "clustered_corr"])
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--group", type=int, default=0)
+    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj"], help="oproj needs a workload with an attention half")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")

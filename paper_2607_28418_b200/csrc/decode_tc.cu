@@ -10,7 +10,7 @@
 //                 The k-steps of all row blocks form one long sequence that is cut into equal,
 //                 contiguous shares, one per CTA, so every SM streams the same number of bytes and
 //                 a row block is split between at most a few CTAs.  Weight tiles arrive by TMA
-//                 through an 8-stage ring (>= 128 KB in flight per SM), tcgen05 accumulates in
+//                 through a ring of 8 to 10 stages (>= 128 KB in flight per SM), tcgen05 accumulates in
 //                 TMEM, the epilogue adds each partial tile into an L2-resident fp32 accumulator
 //                 with 16-byte red.add.  The CTA that adds the last partial of a 128-channel block
 //                 (a ticket counter tells) turns it into h = M ? silu(gate) * up : 0 (bf16) and
@@ -32,13 +32,13 @@ namespace {
 
 using namespace wptx;
 
-constexpr int kStagesD = 8;
+constexpr int kMaxStagesD = 16;            // ring depth is chosen per launch: as many stages as fit
 constexpr int kRows = 128;                 // weight rows per tile (UMMA M)
 constexpr int kBKD = 64;
 constexpr int kWBytes = kRows * kBKD * 2;  // 16 KB
 constexpr int kMaxNT = WIDE_DECODE_MAX_TOKENS;
 constexpr int kActBytes = kMaxNT * kBKD * 2;  // 8 KB reserved per stage
-constexpr int kStageBytesD = kWBytes + kActBytes;
+constexpr int kRingBytesD = 8 * (kWBytes + kActBytes);  // 192 KB of shared memory for the ring
 constexpr int kAccColsD = 64;              // TMEM columns per accumulator buffer
 constexpr int kThreadsD = 192;
 
@@ -73,6 +73,8 @@ struct Pipe {
     uint32_t tmem_base;
     int n;   // k-steps issued / consumed so far (per role)
     int tc;  // accumulator tiles so far (per role)
+    int nstages;       // ring depth
+    int stage_bytes;   // 16 KB weight tile + NT x 128 B activation tile
 };
 
 // One contiguous piece of a CTA's share: `nsteps` k-steps of work block `blk` starting at step k0.
@@ -191,10 +193,10 @@ __device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* t
             if (weights_only_steps >= 0 && step >= weights_only_steps) return true;  // pre-issue done
             const int ks = sg.k0 + i;
             const int col = mode == MODE_GATEUP ? ks * kBKD : s_union[ks / ksub] * a.G + (ks % ksub) * kBKD;
-            const int s = n % kStagesD;
-            const uint32_t dst = smem_u32(P.base + s * kStageBytesD);
+            const int s = n % P.nstages;
+            const uint32_t dst = smem_u32(P.base + s * P.stage_bytes);
             if (step >= skip_weight_steps) {
-                const uint32_t ph = (n / kStagesD) & 1;
+                const uint32_t ph = (n / P.nstages) & 1;
                 if (!mbar_wait(P.empty + 8 * s, ph ^ 1u, a.wait_ns, P.abort_flag)) return false;
                 mbar_arrive_expect_tx(P.full + 8 * s, stage_tx);
                 tma_load_2d(dst, tw, col, row0, P.full + 8 * s);
@@ -218,11 +220,11 @@ __device__ bool mma_pass(int mode, const DecodeArgs& a, Pipe& P, int n_union) {
         tc_fence_after_sync();
         const uint32_t d_tmem = P.tmem_base + buf * kAccColsD;
         for (int i = 0; i < sg.nsteps; ++i, ++P.n) {
-            const int s = P.n % kStagesD;
-            const uint32_t ph = (P.n / kStagesD) & 1;
+            const int s = P.n % P.nstages;
+            const uint32_t ph = (P.n / P.nstages) & 1;
             if (!mbar_wait(P.full + 8 * s, ph, a.wait_ns, P.abort_flag)) return false;
             tc_fence_after_sync();
-            const uint32_t w_addr = smem_u32(P.base + s * kStageBytesD);
+            const uint32_t w_addr = smem_u32(P.base + s * P.stage_bytes);
             const uint64_t adesc = umma_desc_sw128(w_addr);
             const uint64_t bdesc = umma_desc_sw128(w_addr + kWBytes);
 #pragma unroll
@@ -327,7 +329,7 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
         }
         epilogue_bar_sync();
         if (*s_flag) {
-            constexpr int kB4 = 4;  // 16-byte pieces per round: 2 * kB4 loads in flight per thread
+            constexpr int kB4 = 8;  // 16-byte pieces per round: 2 * kB4 loads in flight per thread
             if (mode == MODE_GATEUP) {
                 // h[b, ch] for the 128 (or G) channels of this block; re-zero gate / up
                 const int gidx = s_union[slot_blk / a.blocks_per_group];
@@ -374,13 +376,13 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
                 const int orow = sg.blk * kRows + e;
                 if (orow < a.D) {
                     float4* yp = reinterpret_cast<float4*>(a.yacc + static_cast<size_t>(orow) * a.NT);
-                    for (int b0 = 0; b0 < nb4; b0 += 2 * kB4) {
-                        float4 v[2 * kB4];
+                    for (int b0 = 0; b0 < nb4; b0 += kB4) {
+                        float4 v[kB4];
 #pragma unroll
-                        for (int j = 0; j < 2 * kB4; ++j)
+                        for (int j = 0; j < kB4; ++j)
                             if (b0 + j < nb4) v[j] = __ldcg(yp + b0 + j);
 #pragma unroll
-                        for (int j = 0; j < 2 * kB4; ++j) {
+                        for (int j = 0; j < kB4; ++j) {
                             if (b0 + j < nb4) {
                                 yp[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 const float vs[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
@@ -414,21 +416,23 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
     __shared__ int s_flag;
     __shared__ unsigned s_tokmask[2];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStagesD * kStageBytesD);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStagesD + 4);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + kRingBytesD);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStagesD + 4);
     Pipe P;
     P.base = base;
     P.full = smem_u32(bars);
-    P.empty = smem_u32(bars + kStagesD);
-    P.tfull = smem_u32(bars + 2 * kStagesD);
-    P.tempty = smem_u32(bars + 2 * kStagesD + 2);
+    P.empty = smem_u32(bars + kMaxStagesD);
+    P.tfull = smem_u32(bars + 2 * kMaxStagesD);
+    P.tempty = smem_u32(bars + 2 * kMaxStagesD + 2);
+    P.stage_bytes = kWBytes + a.NT * kBKD * 2;
+    P.nstages = min(kMaxStagesD, kRingBytesD / P.stage_bytes);
     P.abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     P.n = 0;
     P.tc = 0;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < kStagesD; ++s) {
+        for (int s = 0; s < P.nstages; ++s) {
             mbar_init(P.full + 8 * s, 1);
             mbar_init(P.empty + 8 * s, 1);
         }
@@ -491,7 +495,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
                         const PassGeom g2 = geom_of(MODE_DOWN, a, n_union);
                         const int mine = max(0, min((static_cast<int>(blockIdx.x) + 1) * g2.L, g2.total) -
                                                     min(static_cast<int>(blockIdx.x) * g2.L, g2.total));
-                        pre = min(kStagesD, mine);
+                        pre = min(P.nstages, mine);
                         ok = produce_pass(MODE_DOWN, a, &tmWd, &tmWd, &tmH, P, s_union, n_union, pre, 0);
                     }
                 }
@@ -554,7 +558,7 @@ bool make_tmap(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kSmemD = kStagesD * kStageBytesD + (2 * kStagesD + 4) * 8 + 16 + 1024;
+constexpr int kSmemD = kRingBytesD + (2 * kMaxStagesD + 4) * 8 + 16 + 1024;
 
 int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a, const void* wg, const void* wu,
                   const void* wd, int B, int D, int inner, int G, const uint32_t* mask_bits, void* y, int out_dtype,
