@@ -89,8 +89,6 @@ __device__ __forceinline__ void abort_grace() {
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
 }
 
-__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
-
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -488,46 +486,144 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ======================================================================================= gate/up
-// Work item j -> (pair = j / nsub, sub = j % nsub); pair = work_list[pair] = (tile m, group g);
-// channels [g*G + sub*BN, +BN) of W_gate and W_up; rows = perm[g][m*128 .. m*128+127].
+// Items.  A group g with c_g active tokens has nt_g = ceil(c_g / 128) row tiles in its sorted
+// order.  Two consecutive tiles of the same (group, channel sub-block) form a DOUBLE item: 256
+// gathered rows, two M=128 UMMAs per 16-wide k-slice sharing the weight tile in shared memory
+// (1.5x fewer bytes per FLOP, the ring covers 1.5x more latency).  Doubles are dealt round-robin
+// for as many full rounds as there are; what is left of them is cut back into 128-row SINGLE items
+// and dealt together with the odd last tiles, so that every CTA ends within one single item of the
+// others.  Every CTA derives the same schedule from `counts` alone (prefix sums in shared memory).
+// The two accumulators of a double fill TMEM, so an item's epilogue does not overlap the next
+// item's MMAs; it is kept short instead (8 epilogue warps, fast SiLU).
+struct GuItem {
+    int gs;     // group * nsub + sub-block
+    int m;      // first 128-row tile
+    int rows;   // 128 or 256
+};
+
+struct GuSched {
+    const int* dbl_off;   // [n_gs + 1] prefix of doubles per (group, sub)
+    const int* sgl_off;   // [n_gs + 1] prefix of odd last tiles
+    int n_gs, nD, nS, grid, rfull, remD, nS2, pos;
+    __device__ GuSched(const int* d, const int* sg, int n) : dbl_off(d), sgl_off(sg), n_gs(n), grid(gridDim.x), pos(0) {
+        nD = d[n];
+        nS = sg[n];
+        rfull = nD / grid;
+        remD = nD - rfull * grid;
+        nS2 = 2 * remD + nS;
+    }
+    __device__ int find(const int* off, int idx) const {  // largest i with off[i] <= idx
+        int lo = 0, hi = n_gs;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (off[mid] <= idx) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+    __device__ bool next(GuItem& it) {
+        const int b = blockIdx.x;
+        if (pos < rfull) {
+            const int di = pos * grid + b;
+            it.gs = find(dbl_off, di);
+            it.m = 2 * (di - dbl_off[it.gs]);
+            it.rows = 256;
+            ++pos;
+            return true;
+        }
+        const int idx = (pos - rfull) * grid + b;
+        if (idx >= nS2) return false;
+        if (idx < 2 * remD) {
+            const int di = rfull * grid + (idx >> 1);
+            it.gs = find(dbl_off, di);
+            it.m = 2 * (di - dbl_off[it.gs]) + (idx & 1);
+        } else {
+            const int si = idx - 2 * remD;
+            it.gs = find(sgl_off, si);
+            it.m = 2 * (dbl_off[it.gs + 1] - dbl_off[it.gs]);   // the odd tile follows the group's doubles
+        }
+        it.rows = 128;
+        ++pos;
+        return true;
+    }
+};
+
+__device__ __forceinline__ float silu_mul_fast(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+
+constexpr int kGuThreads = 448;  // TMA, MMA, 4 gather warps, 8 epilogue warps
+
 template <int BN>  // channels per item (UMMA N = 2*BN)
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(kGuThreads, 1)
 gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
               const __nv_bfloat16* __restrict__ X, const int32_t* __restrict__ perm,
-              const int32_t* __restrict__ counts, const int32_t* __restrict__ work_list,
-              const int32_t* __restrict__ n_work, int T, int D, int Dff, int G, __nv_bfloat16* __restrict__ H,
+              const int32_t* __restrict__ counts, int NG, int T, int D, int Dff, int G, __nv_bfloat16* __restrict__ H,
               int* __restrict__ status, unsigned long long wait_ns) {
+    constexpr int kStagesG = BN == 128 ? 3 : 4;
+    constexpr int kAB = 2 * kABytes;              // 256 rows x 128 B
     constexpr int kBBytes = 2 * BN * kBK * 2;
-    constexpr int kStageBytes = kABytes + kBBytes;
+    constexpr int kStageBytes = kAB + kBBytes;
+    constexpr int kMaxGs = WIDE_MAX_GROUPS * 4;  // (group, sub-block) pairs: G <= 512, BN >= 128 there
     extern __shared__ uint8_t smem_raw[];
-    SmemLayout L = carve_smem<kBBytes>(smem_raw);
+    __shared__ int s_dbl[kMaxGs + 1];
+    __shared__ int s_sgl[kMaxGs + 1];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStagesG * kStageBytes);
+    const uint32_t full = smem_u32(bars), empty = smem_u32(bars + kStagesG);
+    const uint32_t tfull = smem_u32(bars + 2 * kStagesG), tempty = smem_u32(bars + 2 * kStagesG + 1);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStagesG + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nsub = G / BN;
+    const int n_gs = NG * nsub;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(L.full + 8 * s, 1 + 128);  // TMA producer + one arrival per gather thread
-            mbar_init(L.empty + 8 * s, 1);
+        for (int s = 0; s < kStagesG; ++s) {
+            mbar_init(full + 8 * s, 1 + 128);  // TMA producer + one arrival per gather thread
+            mbar_init(empty + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(L.tfull + 8 * b, 1);
-            mbar_init(L.tempty + 8 * b, 4);
-        }
-        *L.abort_flag = 0;
+        mbar_init(tfull, 1);
+        mbar_init(tempty, 8);
+        *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmG);
         prefetch_tmap(&tmU);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(L.tmem_slot), 512);
+        tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
+    }
+    if (warp == 2) {
+        // prefix sums of doubles and odd tiles per (group, sub-block)
+        int dsum = 0, ssum = 0;
+        for (int base_i = 0; base_i < n_gs; base_i += 32) {
+            const int i = base_i + lane;
+            int dv = 0, sv = 0;
+            if (i < n_gs) {
+                const int nt = (counts[i / nsub] + kBM - 1) / kBM;
+                dv = nt >> 1;
+                sv = nt & 1;
+            }
+            int dp = dv, sp = sv;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a = __shfl_up_sync(0xffffffffu, dp, o), c = __shfl_up_sync(0xffffffffu, sp, o);
+                if (lane >= o) { dp += a; sp += c; }
+            }
+            if (i < n_gs) {
+                s_dbl[i] = dsum + dp - dv;
+                s_sgl[i] = ssum + sp - sv;
+            }
+            dsum += __shfl_sync(0xffffffffu, dp, 31);
+            ssum += __shfl_sync(0xffffffffu, sp, 31);
+        }
+        if (lane == 0) {
+            s_dbl[n_gs] = dsum;
+            s_sgl[n_gs] = ssum;
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_base = *L.tmem_slot;
-
-    const int nsub = G / BN;
-    const int n_items = (*n_work) * nsub;
+    const uint32_t tmem_base = *tmem_slot;
     const int nk = D / kBK;
 
     if (warp == 0) {
@@ -535,18 +631,18 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         if (lane == 0) {
             int it = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int pair = item / nsub, sub = item - pair * nsub;
-                const int g = work_list[2 * pair + 1];
-                const int crow = g * G + sub * BN;
+            GuSched sched(s_dbl, s_sgl, n_gs);
+            GuItem w;
+            while (ok && sched.next(w)) {
+                const int crow = (w.gs / nsub) * G + (w.gs % nsub) * BN;
                 for (int k = 0; k < nk; ++k, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
-                    if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(L.full + 8 * s, kBBytes);
-                    const uint32_t b_dst = smem_u32(L.stage_base + s * kStageBytes) + kABytes;
-                    tma_load_2d(b_dst, &tmG, k * kBK, crow, L.full + 8 * s);
-                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, crow, L.full + 8 * s);
+                    const int s = it % kStagesG;
+                    const uint32_t ph = (it / kStagesG) & 1;
+                    if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(full + 8 * s, kBBytes);
+                    const uint32_t b_dst = smem_u32(base + s * kStageBytes) + kAB;
+                    tma_load_2d(b_dst, &tmG, k * kBK, crow, full + 8 * s);
+                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, crow, full + 8 * s);
                 }
             }
             if (!ok) { report_timeout(status); abort_grace(); }
@@ -557,130 +653,145 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             constexpr uint32_t idesc = umma_idesc_bf16(kBM, 2 * BN);
             int it = 0, tc = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tc) {
-                const int buf = tc & 1;
-                const uint32_t tph = (tc >> 1) & 1;
-                if (!mbar_wait(L.tempty + 8 * buf, tph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
+            GuSched sched(s_dbl, s_sgl, n_gs);
+            GuItem w;
+            while (ok && sched.next(w)) {
+                if (!mbar_wait(tempty, (tc & 1) ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * kAccCols;
                 for (int k = 0; k < nk; ++k, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
-                    if (!mbar_wait(L.full + 8 * s, ph, wait_ns, L.abort_flag)) { ok = false; break; }
+                    const int s = it % kStagesG;
+                    const uint32_t ph = (it / kStagesG) & 1;
+                    if (!mbar_wait(full + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
                     fence_proxy_async_smem();  // the A rows were written through the generic proxy (cp.async)
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(L.stage_base + s * kStageBytes);
-                    const uint64_t adesc = umma_desc_sw128(a_addr);
-                    const uint64_t bdesc = umma_desc_sw128(a_addr + kABytes);
+                    const uint32_t a_addr = smem_u32(base + s * kStageBytes);
+                    const uint64_t adesc0 = umma_desc_sw128(a_addr);
+                    const uint64_t adesc1 = umma_desc_sw128(a_addr + kABytes);
+                    const uint64_t bdesc = umma_desc_sw128(a_addr + kAB);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBK / 16; ++k4)
-                        umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (k > 0 || k4 > 0) ? 1u : 0u);
-                    umma_commit(L.empty + 8 * s);
+                    for (int k4 = 0; k4 < kBK / 16; ++k4) {
+                        const uint32_t accumulate = (k > 0 || k4 > 0) ? 1u : 0u;
+                        umma_bf16(tmem_base, adesc0 + 2 * k4, bdesc + 2 * k4, idesc, accumulate);
+                        if (w.rows == 256) umma_bf16(tmem_base + 256, adesc1 + 2 * k4, bdesc + 2 * k4, idesc, accumulate);
+                    }
+                    umma_commit(empty + 8 * s);
                 }
-                if (ok) umma_commit(L.tfull + 8 * buf);
+                if (ok) umma_commit(tfull);
+                ++tc;
             }
             if (!ok) report_timeout(status);
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------------ A gather (warps 2..5)
-        // Each thread copies its row's 128 bytes with eight 16-byte cp.async and lets the stage's
-        // mbarrier count an arrival when they have landed; nothing waits on the issuing side, so
-        // the gather runs as far ahead as the ring allows.
-        // Coalesced mapping: 8 consecutive lanes copy the 8 chunks of one row, a warp instruction
-        // covers 4 whole rows (4 x 128 contiguous bytes); instruction i of warp w handles tile rows
-        // w*32 + 4*i + lane/8.
+        // 16-byte cp.async copies land in the 128-byte-swizzle pattern; the stage's mbarrier counts
+        // one arrival per thread when that thread's copies have landed, so the gather runs as far
+        // ahead as the ring allows.  Coalesced mapping: 8 consecutive lanes copy the 8 chunks of
+        // one row, one warp instruction covers 4 whole rows; instruction i of gather warp w copies
+        // tile rows 16*i + 4*w + lane/8  (i < 8 for a 128-row item, i < 16 for a 256-row item).
         const int chunk = lane & 7;
-        const int row0 = (warp - 2) * 32 + (lane >> 3);
-        uint32_t dst_off[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = row0 + 4 * i;
-            dst_off[i] = static_cast<uint32_t>(r) * 128u + ((static_cast<uint32_t>(chunk) ^ static_cast<uint32_t>(r & 7)) << 4);
-        }
+        const int row0 = (warp - 2) * 4 + (lane >> 3);
         int it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-            const int pair = item / nsub;
-            const int m = work_list[2 * pair], g = work_list[2 * pair + 1];
-            const uint8_t* src[8];
+        GuSched sched(s_dbl, s_sgl, n_gs);
+        GuItem w;
+        while (ok && sched.next(w)) {
+            const int g = w.gs / nsub;
+            const int ni = w.rows / 16;
+            const uint8_t* src[16];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                int j = m * kBM + row0 + 4 * i;
+            for (int i = 0; i < 16; ++i) {
+                int j = w.m * kBM + row0 + 16 * i;
                 if (j >= T) j = T - 1;
-                const int tok = perm[static_cast<size_t>(g) * T + j];
+                const int tok = i < ni ? perm[static_cast<size_t>(g) * T + j] : 0;
                 src[i] = reinterpret_cast<const uint8_t*>(X + static_cast<size_t>(tok) * D) + 16 * chunk;
             }
             for (int k = 0; k < nk; ++k, ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (it / kStages) & 1;
-                if (!mbar_wait(L.empty + 8 * s, ph ^ 1u, wait_ns, L.abort_flag)) { ok = false; break; }
-                const uint32_t a_dst = smem_u32(L.stage_base + s * kStageBytes);
+                const int s = it % kStagesG;
+                const uint32_t ph = (it / kStagesG) & 1;
+                if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
+                const uint32_t a_dst = smem_u32(base + s * kStageBytes);
                 const size_t koff = static_cast<size_t>(k) * (kBK * 2);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) cp_async_16(a_dst + dst_off[i], src[i] + koff);
-                cp_async_mbar_arrive_noinc(L.full + 8 * s);
+                for (int i = 0; i < 16; ++i) {
+                    if (i < ni) {
+                        const int r = row0 + 16 * i;
+                        cp_async_16(a_dst + static_cast<uint32_t>(r) * 128u +
+                                        ((static_cast<uint32_t>(chunk) ^ static_cast<uint32_t>(r & 7)) << 4),
+                                    src[i] + koff);
+                    }
+                }
+                cp_async_mbar_arrive_noinc(full + 8 * s);
             }
         }
         cp_async_wait_all();
         if (!ok && lane == 0) report_timeout(status);
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 6..9)
+        // ------------------------------------------------------------------ epilogue (warps 6..13)
+        // warp pair (w, w+4) shares a TMEM lane quarter and splits the item's channels in two
         const int q = warp & 3;
+        const int ew = warp - 6;
+        const int chalf = ew >> 2;
+        const int e = ew * 32 + lane;  // 0..255
+        constexpr int kCh = BN / 2;    // channels per epilogue warp
         int tc = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tc) {
-            const int pair = item / nsub, sub = item - pair * nsub;
-            const int m = work_list[2 * pair], g = work_list[2 * pair + 1];
-            const int j = m * kBM + q * 32 + lane;
-            const bool live = j < counts[g];
-            const int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
-            __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN;
+        GuSched sched(s_dbl, s_sgl, n_gs);
+        GuItem w;
+        while (ok && sched.next(w)) {
+            const int g = w.gs / nsub, sub = w.gs % nsub;
+            const int c = counts[g];
             {
                 // While the MMAs of this item run: zero this item's share of the group's INACTIVE
-                // rows of H (sorted positions [c, T) split evenly over the group's active tiles),
-                // so that the down projection reads exact zeros for every inactive (token, group)
-                // pair of a group that is active anywhere.  Groups nobody selected are never read.
-                const int c = counts[g];
+                // rows of H (sorted positions [c, T) split evenly over the group's row tiles), so
+                // that the down projection reads exact zeros for every inactive (token, group) pair
+                // of a group that is active anywhere.  Groups nobody selected are never read.
                 const int nt = (c + kBM - 1) / kBM;
                 const int per = (T - c + nt - 1) / nt;
-                const int j0 = c + m * per;
-                const int j1 = min(T, j0 + per);
-                for (int jj = j0 + (warp - 6) * 32 + lane; jj < j1; jj += 128) {
-                    const int tz = perm[static_cast<size_t>(g) * T + jj];
-                    uint4* z = reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN);
+                for (int mm = w.m; mm < w.m + w.rows / kBM; ++mm) {
+                    const int j0 = c + mm * per;
+                    const int j1 = min(T, j0 + per);
+                    for (int jj = j0 + e; jj < j1; jj += 256) {
+                        const int tz = perm[static_cast<size_t>(g) * T + jj];
+                        uint4* z = reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN);
 #pragma unroll
-                    for (int v = 0; v < BN / 8; ++v) z[v] = make_uint4(0u, 0u, 0u, 0u);
+                        for (int v = 0; v < BN / 8; ++v) z[v] = make_uint4(0u, 0u, 0u, 0u);
+                    }
                 }
             }
-            const int buf = tc & 1;
-            const uint32_t tph = (tc >> 1) & 1;
-            if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
+            if (!mbar_wait(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
+            for (int half = 0; half < w.rows / kBM; ++half) {
+                const int j = (w.m + half) * kBM + q * 32 + lane;
+                const bool live = j < c;
+                const int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
+                __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN + chalf * kCh;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256 + chalf * kCh;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t gr[32], ur[32];
-                tmem_ld_32x32(taddr + c0, gr);
-                tmem_ld_32x32(taddr + BN + c0, ur);
-                tmem_ld_wait();
-                if (live) {
-                    uint4* dst = reinterpret_cast<uint4*>(hrow + c0);
+                for (int c0 = 0; c0 < kCh; c0 += 32) {
+                    uint32_t gr[32], ur[32];
+                    tmem_ld_32x32(taddr + c0, gr);
+                    tmem_ld_32x32(taddr + BN + c0, ur);
+                    tmem_ld_wait();
+                    if (live) {
+                        uint4* dst = reinterpret_cast<uint4*>(hrow + c0);
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t o[4];
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int i = 8 * v + 2 * e;
-                            o[e] = pack_bf16(silu_mul(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
-                                             silu_mul(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
+                            for (int x4 = 0; x4 < 4; ++x4) {
+                                const int i = 8 * v + 2 * x4;
+                                o[x4] = pack_bf16(silu_mul_fast(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
+                                                  silu_mul_fast(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
+                            }
+                            dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
                         }
-                        dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(L.tempty + 8 * buf);
+            if (lane == 0) mbar_arrive(tempty);
+            ++tc;
         }
         if (!ok && lane == 0) report_timeout(status);
     }
@@ -768,16 +879,17 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
 
 template <int BN>
 int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, int T, int D,
-                  int Dff, int G, const int32_t* perm, const int32_t* counts, const int32_t* work_list,
-                  const int32_t* n_work, void* h) {
+                  int Dff, int G, const int32_t* perm, const int32_t* counts, void* h) {
     CUtensorMap tmG, tmU;
     if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
-    constexpr int smem = smem_bytes<2 * BN * kBK * 2>();
+    constexpr int stages = BN == 128 ? 3 : 4;
+    constexpr int smem = stages * (2 * kABytes + 2 * BN * kBK * 2) + (2 * stages + 2) * 8 + 16 + 1024;
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     WideLaunch l(ctx, s, "prefill_gateup");
-    gateup_kernel<BN><<<ctx->sm_count, 320, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm, counts,
-                                                       work_list, n_work, T, D, Dff, G,
-                                                       static_cast<__nv_bfloat16*>(h), ctx->d_status, ctx->wait_ns);
+    gateup_kernel<BN><<<ctx->sm_count, kGuThreads, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm,
+                                                              counts, Dff / G, T, D, Dff, G,
+                                                              static_cast<__nv_bfloat16*>(h), ctx->d_status,
+                                                              ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -790,8 +902,10 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
     if (T == 0) return WIDE_OK;
     // inactive (token, group) pairs of H must read as zero in the down projection: the gate/up
     // kernel's epilogue warps write those zeros themselves
-    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h)
-                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, work_list, n_work, h);
+    (void)work_list;
+    (void)n_work;  // the kernel derives its own schedule from `counts`
+    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, h)
+                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, h);
     if (rc != WIDE_OK) return rc;
     return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype);
 }
