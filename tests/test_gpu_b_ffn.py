@@ -135,6 +135,14 @@ def test_decode_matches_oracle(ctx, B, G):
     assert_close(y, ref, f"decode B{B} G{G}")
 
 
+@pytest.mark.parametrize("B", [2, 3, 4])
+def test_decode_tiny_batches(ctx, B):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=B, hidden=1024, d_ff=2048, group=128, k=7)
+    y, ref, _ = _run_ffn(ctx, cfg, 20 + B, binding.FLAG_NONE, with_meta=False, out_dtype=torch.float32)
+    assert_close(y, ref, f"decode B{B}")
+
+
 def test_decode_clustered_union_and_zero_cases(ctx):
     from paper_2607_28418_b200 import binding
     cfg = synth.WideConfig("t", tokens=16, hidden=512, d_ff=2048, group=128, k=8, router="clustered")
