@@ -179,11 +179,20 @@ WIDE_API int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int d
  *   n_union    out int32 [1]
  *   offsets    out int32 [n_groups + 1]       offsets[g] = sum_{g'<g} ceil(counts[g']/tile_m)*tile_m
  *                                             (row offsets of the packed-sorted layout)
+ *   token_order, token_rank  out int32 [tokens] each, or both NULL.  One token permutation that puts
+ *       tokens with the same mask next to each other, so that token tiles taken in this order share
+ *       their active groups: token_order = the tokens in a STABLE sort by key(t), token_rank its
+ *       inverse (token_rank[token_order[p]] = p), with
+ *           key(t) = h >> 24,  h = 0x811C9DC5;  for each mask word w of token t:  h = (h ^ w) * 0x01000193
+ *       (32-bit wrap-around).  The prefill FFN / O-projection keep their intermediate rows in this
+ *       order and walk token tiles in it; a (tile, group) block is skipped when no token of the tile
+ *       selected the group.
  * tile_m must be a power of two >= 16.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE.
  */
 WIDE_API int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
                  int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map, int32_t* work_list,
-                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets);
+                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets,
+                 int32_t* token_order, int32_t* token_rank);
 
 /*
  * wide_ffn -- Eq. 3:  y = ((silu(x Wg^T) * (x Wu^T)) (.)_G M) Wd^T.
@@ -192,10 +201,12 @@ WIDE_API int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits
  *
  *   x [tokens, hidden], w_gate/w_up [d_ff, hidden], w_down [hidden, d_ff]: dtype
  *   mask_bits [tokens, W], W = ceil((d_ff/group)/32)
- *   perm, counts, work_list, n_work: outputs of wide_reorder for this mask with tile_m = 128.
- *       Needed by the prefill tensor-core path; may all be NULL when tokens <=
- *       WIDE_DECODE_MAX_TOKENS (decode path: union of active groups, no reordering) or with
- *       WIDE_FLAG_SIMT.
+ *   perm, counts: outputs of wide_reorder for this mask.  Needed by the prefill tensor-core path;
+ *       may be NULL when tokens <= WIDE_DECODE_MAX_TOKENS (decode path: union of active groups, no
+ *       reordering) or with WIDE_FLAG_SIMT.
+ *   token_order, token_rank: the token clustering of wide_reorder, or both NULL (tokens are then
+ *       tiled in their original order).  Only the prefill tensor-core path uses them; the result
+ *       is the same either way, block skipping in the down projection is not.
  *   y  out [tokens, hidden] of out_dtype
  * Tensor-core paths need dtype bf16, hidden % 64 == 0, group in {64,128,256,512}; other shapes
  * need WIDE_FLAG_SIMT (hidden % 4 == 0, group % 4 == 0).
@@ -204,18 +215,19 @@ WIDE_API int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits
 WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
              const void* w_down, int dtype, int tokens, int hidden, int d_ff, int group,
              const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
-             const int32_t* work_list, const int32_t* n_work, void* y, int out_dtype,
+             const int32_t* token_order, const int32_t* token_rank, void* y, int out_dtype,
              void* workspace, size_t workspace_bytes, unsigned flags);
 
 /*
  * wide_oproj -- Eq. 2 / Eq. 10:  y[t,:] = sum_{g : M[t,g]=1} a[t, gG:(g+1)G] Wo[:, gG:(g+1)G]^T,
  * a = attention output flattened head-major [tokens, attn_dim], group g = channels [gG, (g+1)G).
- *   perm, counts, work_list, n_work as for wide_ffn (same NULL rules).
+ *   perm, counts: reserved (the current kernels do not read them; may be NULL).
+ *   token_order, token_rank as for wide_ffn.
  */
 WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
                int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,
-               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
-               const int32_t* n_work, void* y, int out_dtype, void* workspace,
+               const int32_t* perm, const int32_t* counts, const int32_t* token_order,
+               const int32_t* token_rank, void* y, int out_dtype, void* workspace,
                size_t workspace_bytes, unsigned flags);
 
 /*

@@ -15,6 +15,9 @@ route_scores          Routing components (Section 3.1): a linear map from the
 mask_pair_argmax      Eq. 4, inference branch: bit = [argmax over the class pair = 0].
 reorder               Eq. 6 / Algorithm 1 (per-column SortDesc, stable), the predicate
                       of Eq. 7-8 at level 0 (CTA tile), Appendix B's monotone shortcut.
+cluster_tokens        not in the paper: one global token permutation (stable sort by a
+                      hash of the mask row, the key is defined in the library header)
+                      under which tiles of tokens share their active groups.
 ffn                   Eq. 3 literally: (phi(X Wg^T) * (X Wu^T)) gated group-wise by the
                       mask, times Wd^T, with phi = SiLU.
 oproj                 Eq. 2 / Eq. 10: (A gated group-wise) Wo^T.
@@ -24,7 +27,9 @@ Parity pins (tests/test_oracle_*.py): exact-rational brute force for scores and
 top-k, closed-form one-hot routers, hand-worked reorder fixture, permutation /
 monotonicity / boundary-tile invariants, dense-SwiGLU special case against a library
 routine, brute-force single-group sums, additivity over disjoint masks (Eq. 10), the
-per-token gather formulation of Appendix A, constant-weight closed forms.
+per-token gather formulation of Appendix A, constant-weight closed forms; token
+clustering: permutation / inverse / sortedness / stability / grouping properties and
+two hand-expanded hash values.
 "Parity to values printed in the paper": unpinned -- the paper prints no worked
 numeric example for this path.
 
@@ -99,6 +104,31 @@ def unpack_mask_bits(bits: np.ndarray, n_groups: int) -> np.ndarray:
     return out
 
 
+# ----------------------------------------------------------------------------- token clustering
+def mask_key(words_row) -> int:
+    """Clustering key of one token: top 8 bits of an FNV-1a style hash over its packed mask words
+    (the definition stated in the library header; 32-bit wrap-around arithmetic)."""
+    h = 0x811C9DC5
+    for w in words_row:
+        h = ((h ^ int(w)) * 0x01000193) & 0xFFFFFFFF
+    return h >> 24
+
+
+def cluster_tokens(mask: np.ndarray) -> Dict[str, np.ndarray]:
+    """One token permutation that makes tiles of tokens share their active groups (the global
+    counterpart of the per-group sort of Eq. 6): tokens in a stable sort by mask_key, so tokens
+    with identical masks are neighbours.  token_rank is the inverse of token_order."""
+    bits = pack_mask_bits(mask)
+    T = bits.shape[0]
+    keys = [mask_key(bits[t]) for t in range(T)]
+    order = sorted(range(T), key=lambda t: (keys[t], t))
+    rank = [0] * T
+    for p, t in enumerate(order):
+        rank[t] = p
+    return {"token_order": np.asarray(order, dtype=np.int32).reshape(T),
+            "token_rank": np.asarray(rank, dtype=np.int32).reshape(T)}
+
+
 # ----------------------------------------------------------------------------- reorder
 def reorder(mask: np.ndarray, tile_m: int) -> Dict[str, np.ndarray]:
     """Mask reordering (Eq. 6, Algorithm 1) and the level-0 predicate (Eq. 7-8).
@@ -117,6 +147,7 @@ def reorder(mask: np.ndarray, tile_m: int) -> Dict[str, np.ndarray]:
       union_list  int32 [n_union]  groups with at least one active row, ascending
       n_union     int
       offsets     int32 [N_G + 1]  offsets[g] = sum_{g' < g} ceil(counts[g'] / BM) * BM
+      token_order, token_rank  int32 [T]  see cluster_tokens
     """
     mask = np.asarray(mask, dtype=bool)
     T, n_groups = mask.shape
@@ -142,7 +173,10 @@ def reorder(mask: np.ndarray, tile_m: int) -> Dict[str, np.ndarray]:
     offsets = np.zeros(n_groups + 1, dtype=np.int32)
     for g in range(n_groups):
         offsets[g + 1] = offsets[g] + ((int(counts[g]) + tile_m - 1) // tile_m) * tile_m
+    clustered = cluster_tokens(mask)
     return {
+        "token_order": clustered["token_order"],
+        "token_rank": clustered["token_rank"],
         "perm": perm,
         "sorted_mask": sorted_mask,
         "counts": counts,

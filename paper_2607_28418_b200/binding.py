@@ -66,7 +66,7 @@ def load_library() -> ctypes.CDLL:
                                _c_int, _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                                _c_size_t, _c_uint]
     lib.wide_route_static.argtypes = lib.wide_route.argtypes[:15] + [_c_uint]
-    lib.wide_reorder.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int] + [_c_void_p] * 8
+    lib.wide_reorder.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int] + [_c_void_p] * 10
     lib.wide_ffn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int,
                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                              _c_void_p, _c_int, _c_void_p, _c_size_t, _c_uint]
@@ -245,11 +245,13 @@ def wide_reorder(ctx: Context, mask_bits: torch.Tensor, n_groups: int, tile_m: i
             "union_list": torch.empty((n_groups,), **i32),
             "n_union": torch.empty((1,), **i32),
             "offsets": torch.empty((n_groups + 1,), **i32),
+            "token_order": torch.empty((T,), **i32),
+            "token_rank": torch.empty((T,), **i32),
         }
     rc = ctx.lib.wide_reorder(ctx.handle, _stream(), _ptr(mask_bits), T, n_groups, tile_m, _ptr(out["perm"]),
                               _ptr(out["counts"]), _ptr(out["tile_map"]), _ptr(out["work_list"]),
                               _ptr(out["n_work"]), _ptr(out["union_list"]), _ptr(out["n_union"]),
-                              _ptr(out["offsets"]))
+                              _ptr(out["offsets"]), _ptr(out.get("token_order")), _ptr(out.get("token_rank")))
     _check(rc, "wide_reorder")
     return out
 
@@ -268,7 +270,7 @@ def wide_ffn(ctx: Context, x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Te
     m = meta or {}
     rc = ctx.lib.wide_ffn(ctx.handle, _stream(), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), dt, T, D, d_ff,
                           group, _ptr(mask_bits), _ptr(m.get("perm")), _ptr(m.get("counts")),
-                          _ptr(m.get("work_list")), _ptr(m.get("n_work")), _ptr(y), _dtype_code(y), _ptr(ws),
+                          _ptr(m.get("token_order")), _ptr(m.get("token_rank")), _ptr(y), _dtype_code(y), _ptr(ws),
                           ws.numel(), flags)
     _check(rc, "wide_ffn")
     return y
@@ -287,8 +289,8 @@ def wide_oproj(ctx: Context, attn_out: torch.Tensor, w_o: torch.Tensor, group: i
     ws = ctx.workspace(nbytes, slot=0)
     m = meta or {}
     rc = ctx.lib.wide_oproj(ctx.handle, _stream(), _ptr(attn_out), _ptr(w_o), dt, T, D, K, group, _ptr(mask_bits),
-                            _ptr(m.get("perm")), _ptr(m.get("counts")), _ptr(m.get("work_list")),
-                            _ptr(m.get("n_work")), _ptr(y), _dtype_code(y), _ptr(ws), ws.numel(), flags)
+                            _ptr(m.get("perm")), _ptr(m.get("counts")), _ptr(m.get("token_order")),
+                            _ptr(m.get("token_rank")), _ptr(y), _dtype_code(y), _ptr(ws), ws.numel(), flags)
     _check(rc, "wide_oproj")
     return y
 

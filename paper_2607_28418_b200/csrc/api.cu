@@ -226,20 +226,23 @@ int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens
 
 int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
                  int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map, int32_t* work_list,
-                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets) {
+                 int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets, int32_t* token_order,
+                 int32_t* token_rank) {
     if (!ctx || !mask_bits || !perm || !counts || !tile_map || !work_list || !n_work || !union_list || !n_union ||
         !offsets)
         return WIDE_ERR_INVALID_ARG;
     if (tokens < 0 || n_groups <= 0 || !is_pow2(tile_m) || tile_m < 16) return WIDE_ERR_INVALID_ARG;
+    if ((token_order == nullptr) != (token_rank == nullptr)) return WIDE_ERR_INVALID_ARG;
     if (n_groups > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
     return wide_launch_reorder(ctx, static_cast<cudaStream_t>(stream), mask_bits, tokens, n_groups, tile_m, perm,
-                               counts, tile_map, work_list, n_work, union_list, n_union, offsets);
+                               counts, tile_map, work_list, n_work, union_list, n_union, offsets, token_order,
+                               token_rank);
 }
 
 int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
              const void* w_down, int dtype, int tokens, int hidden, int d_ff, int group,
              const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
-             const int32_t* work_list, const int32_t* n_work, void* y, int out_dtype,
+             const int32_t* token_order, const int32_t* token_rank, void* y, int out_dtype,
              void* workspace, size_t workspace_bytes, unsigned flags) {
     if (!ctx || !x || !w_gate || !w_up || !w_down || !mask_bits || !y) return WIDE_ERR_INVALID_ARG;
     if (!valid_dtype(dtype) || !valid_dtype(out_dtype)) return WIDE_ERR_INVALID_ARG;
@@ -248,7 +251,8 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
     const Path path = choose_path(dtype, tokens, hidden, d_ff, group, flags);
     if (path == PATH_NONE) return WIDE_ERR_UNSUPPORTED_SHAPE;
     if (path == PATH_SIMT && (hidden % 4 != 0 || group % 4 != 0)) return WIDE_ERR_UNSUPPORTED_SHAPE;
-    if (path == PATH_PREFILL_TC && (!perm || !counts || !work_list || !n_work)) return WIDE_ERR_INVALID_ARG;
+    if (path == PATH_PREFILL_TC && (!perm || !counts)) return WIDE_ERR_INVALID_ARG;
+    if ((token_order == nullptr) != (token_rank == nullptr)) return WIDE_ERR_INVALID_ARG;
     if (!wide_aligned16(x) || !wide_aligned16(w_gate) || !wide_aligned16(w_up) || !wide_aligned16(w_down) ||
         !wide_aligned16(y) || !wide_aligned16(workspace))
         return WIDE_ERR_ALIGNMENT;
@@ -260,7 +264,7 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
                                         out_dtype, workspace);
         case PATH_PREFILL_TC:
             return wide_launch_ffn_prefill_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
-                                              perm, counts, work_list, n_work, y, out_dtype, workspace);
+                                              perm, counts, token_order, token_rank, y, out_dtype, workspace);
         default:
             return wide_launch_ffn_decode_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
                                              y, out_dtype, workspace);
@@ -269,10 +273,11 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
 
 int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
                int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,
-               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
-               const int32_t* n_work, void* y, int out_dtype, void* workspace,
+               const int32_t* perm, const int32_t* counts, const int32_t* token_order,
+               const int32_t* token_rank, void* y, int out_dtype, void* workspace,
                size_t workspace_bytes, unsigned flags) {
-    (void)perm; (void)counts; (void)work_list; (void)n_work;
+    (void)perm; (void)counts;
+    if ((token_order == nullptr) != (token_rank == nullptr)) return WIDE_ERR_INVALID_ARG;
     if (!ctx || !attn_out || !w_o || !mask_bits || !y) return WIDE_ERR_INVALID_ARG;
     if (!valid_dtype(dtype) || !valid_dtype(out_dtype)) return WIDE_ERR_INVALID_ARG;
     if (tokens < 0 || hidden <= 0 || attn_dim <= 0 || group <= 0 || attn_dim % group != 0) return WIDE_ERR_INVALID_ARG;
@@ -291,8 +296,8 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
             return wide_launch_oproj_simt(ctx, s, attn_out, w_o, dtype, tokens, hidden, attn_dim, group, mask_bits, y,
                                           out_dtype);
         case PATH_PREFILL_TC:
-            return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
-                                                out_dtype, workspace);
+            return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits,
+                                                token_order, token_rank, y, out_dtype, workspace);
         default:
             return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
                                                out_dtype, workspace);

@@ -81,7 +81,7 @@ size_t wide_route_workspace(int T, int NG, int rank);
 int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
                         int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
                         int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
-                        int32_t* offsets);
+                        int32_t* offsets, int32_t* token_order, int32_t* token_rank);
 
 int wide_launch_unpermute(wide_ctx* ctx, cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
                           const int32_t* offsets, int T, int NG, int G, int elem_bytes, void* dst);
@@ -97,14 +97,14 @@ int wide_launch_oproj_simt(wide_ctx* ctx, cudaStream_t s, const void* a, const v
 int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg,
                                const void* wu, const void* wd, int T, int D, int Dff, int G,
                                const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
-                               const int32_t* work_list, const int32_t* n_work, void* y,
+                               const int32_t* token_order, const int32_t* token_rank, void* y,
                                int out_dtype, void* h);
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
                           int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out);
 // `a_masked` is scratch [T, K] bf16.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
-                                 int D, int K, int G, const uint32_t* mask_bits, void* y,
-                                 int out_dtype, void* a_masked);
+                                 int D, int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
+                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked);
 
 // tcgen05 decode path (bf16, T <= WIDE_DECODE_MAX_TOKENS).
 size_t wide_decode_workspace(int T, int D, int inner);

@@ -61,8 +61,9 @@ constexpr int smem_bytes() {
 }
 
 // OR of the mask words of tokens [t0, t0 + 128) computed by one warp; every lane gets the result.
-__device__ __forceinline__ void tile_mask_or(const uint32_t* __restrict__ mask_bits, int words, int T, int t0,
-                                             int lane, uint32_t (&act)[kMaskWords]) {
+// `order` (may be null = identity) maps a row position to its token.
+__device__ __forceinline__ void tile_mask_or(const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order,
+                                             int words, int T, int t0, int lane, uint32_t (&act)[kMaskWords]) {
 #pragma unroll
     for (int w = 0; w < kMaskWords; ++w) act[w] = 0u;
     if (mask_bits == nullptr) {
@@ -71,8 +72,9 @@ __device__ __forceinline__ void tile_mask_or(const uint32_t* __restrict__ mask_b
         return;
     }
     for (int i = lane; i < kBM; i += 32) {
-        const int t = t0 + i;
-        if (t < T) {
+        const int p = t0 + i;
+        if (p < T) {
+            const int t = order ? order[p] : p;
 #pragma unroll
             for (int w = 0; w < kMaskWords; ++w)
                 if (w < words) act[w] |= mask_bits[static_cast<size_t>(t) * words + w];
@@ -100,7 +102,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int BN>
 __global__ void __launch_bounds__(192, 1)
 down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const uint32_t* __restrict__ mask_bits, int words, int T, int N, int K, int G, void* __restrict__ Y,
+            const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N, int K,
+            int G, void* __restrict__ Y,
             int out_bf16, int ksplit, const __nv_bfloat16* __restrict__ aux_w, int aux_rows,
             float* __restrict__ aux_norm, int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = BN * kBK * 2;
@@ -147,7 +150,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int mn = tile % n_mn, only = ksplit > 1 ? tile / n_mn : -1;
             const int m = mn % n_m, n = mn / n_m;
             uint32_t act[kMaskWords];
-            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            tile_mask_or(mask_bits, order, words, T, m * kBM, lane, act);
             if (lane == 0) {
                 for (int g = 0; g < NG && ok; ++g) {
                     if (!((act[g >> 5] >> (g & 31)) & 1u) || (only >= 0 && g != only)) continue;
@@ -175,7 +178,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int mn = tile % n_mn, only = ksplit > 1 ? tile / n_mn : -1;
             const int m = mn % n_m;
             uint32_t act[kMaskWords];
-            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            tile_mask_or(mask_bits, order, words, T, m * kBM, lane, act);
             if (lane == 0) {
                 const int buf = tc & 1;
                 const uint32_t tph = (tc >> 1) & 1;
@@ -218,14 +221,15 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int mn = tile % n_mn, slab = ksplit > 1 ? tile / n_mn : 0;
             const int m = mn % n_m, n = mn / n_m;
             uint32_t act[kMaskWords];
-            tile_mask_or(mask_bits, words, T, m * kBM, lane, act);
+            tile_mask_or(mask_bits, order, words, T, m * kBM, lane, act);
             bool any = false;
             for (int g = 0; g < NG; ++g) any = any || ((act[g >> 5] >> (g & 31)) & 1u);
             const int buf = tc & 1;
             const uint32_t tph = (tc >> 1) & 1;
             if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const int row = m * kBM + q * 32 + lane;
+            const int pos = m * kBM + q * 32 + lane;              // row position of the tile
+            const int row = (order && pos < T) ? order[pos] : pos;  // token that owns this output row
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -310,7 +314,8 @@ constexpr int kSmem2 = kStages2 * kStage2Bytes + (2 * kStages2 + 2) * 8 + 16 + 1
 
 __global__ void __launch_bounds__(192, 1)
 down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const uint32_t* __restrict__ mask_bits, int words, int T, int N, int K, int G, void* __restrict__ Y,
+               const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N,
+               int K, int G, void* __restrict__ Y,
                int out_bf16, int* __restrict__ status, unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -349,8 +354,8 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // OR of the mask words of the tile's 256 tokens
     auto tile_mask = [&](int m, uint32_t (&act)[kMaskWords]) {
         uint32_t hi[kMaskWords];
-        tile_mask_or(mask_bits, words, T, m * 256, lane, act);
-        tile_mask_or(mask_bits, words, T, m * 256 + 128, lane, hi);
+        tile_mask_or(mask_bits, order, words, T, m * 256, lane, act);
+        tile_mask_or(mask_bits, order, words, T, m * 256 + 128, lane, hi);
 #pragma unroll
         for (int w = 0; w < kMaskWords; ++w) act[w] |= hi[w];
     };
@@ -437,7 +442,8 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tc_fence_after_sync();
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
-                const int row = m * 256 + half * 128 + q * 32 + lane;
+                const int pos = m * 256 + half * 128 + q * 32 + lane;
+                const int row = (order && pos < T) ? order[pos] : pos;   // token that owns this output row
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256;
 #pragma unroll 1
                 for (int c0 = 0; c0 < 256; c0 += 32) {
@@ -555,8 +561,8 @@ template <int BN>  // channels per item (UMMA N = 2*BN)
 __global__ void __launch_bounds__(kGuThreads, 1)
 gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
               const __nv_bfloat16* __restrict__ X, const int32_t* __restrict__ perm,
-              const int32_t* __restrict__ counts, int NG, int T, int D, int Dff, int G, __nv_bfloat16* __restrict__ H,
-              int* __restrict__ status, unsigned long long wait_ns) {
+              const int32_t* __restrict__ counts, const int32_t* __restrict__ token_rank, int NG, int T, int D, int Dff,
+              int G, __nv_bfloat16* __restrict__ H, int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kStagesG = BN == 128 ? 3 : 4;
     constexpr int kAB = 2 * kABytes;              // 256 rows x 128 B
     constexpr int kBBytes = 2 * BN * kBK * 2;
@@ -751,7 +757,8 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     const int j0 = c + mm * per;
                     const int j1 = min(T, j0 + per);
                     for (int jj = j0 + e; jj < j1; jj += 256) {
-                        const int tz = perm[static_cast<size_t>(g) * T + jj];
+                        int tz = perm[static_cast<size_t>(g) * T + jj];
+                        if (token_rank) tz = token_rank[tz];   // H rows are kept in clustered token order
                         uint4* z = reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN);
 #pragma unroll
                         for (int v = 0; v < BN / 8; ++v) z[v] = make_uint4(0u, 0u, 0u, 0u);
@@ -763,7 +770,8 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             for (int half = 0; half < w.rows / kBM; ++half) {
                 const int j = (w.m + half) * kBM + q * 32 + lane;
                 const bool live = j < c;
-                const int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
+                int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
+                if (live && token_rank) tok = token_rank[tok];   // H rows are kept in clustered token order
                 __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN + chalf * kCh;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256 + chalf * kCh;
 #pragma unroll 1
@@ -806,14 +814,16 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
 
 // H~[t, c] = M[t, c/G] ? a[t, c] : 0   (16-byte pieces; G*2 bytes is a multiple of 16)
 __global__ void __launch_bounds__(256) mask_rows_kernel(const uint4* __restrict__ a, const uint32_t* __restrict__ mask_bits,
-                                                        int words, int T, int K, int G, uint4* __restrict__ out) {
+                                                        const int32_t* __restrict__ token_rank, int words, int T, int K,
+                                                        int G, uint4* __restrict__ out) {
     const int vec_per_row = K / 8, vec_per_group = G / 8;
     const long long total = static_cast<long long>(T) * vec_per_row;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int t = static_cast<int>(i / vec_per_row);
         const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
-        out[i] = wide_mask_bit(mask_bits, words, t, g) ? a[i] : make_uint4(0u, 0u, 0u, 0u);
+        const long long o = token_rank ? static_cast<long long>(token_rank[t]) * vec_per_row + (i % vec_per_row) : i;
+        out[o] = wide_mask_bit(mask_bits, words, t, g) ? a[i] : make_uint4(0u, 0u, 0u, 0u);
     }
 }
 
@@ -840,7 +850,7 @@ bool make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uin
 template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                 int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down",
-                int ksplit = 1, float* aux_norm = nullptr) {
+                int ksplit = 1, float* aux_norm = nullptr, const int32_t* order = nullptr) {
     CUtensorMap tmA, tmB;
     if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
@@ -851,7 +861,7 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     if (aux_norm) grid = n_tiles + (b_rows + 5) / 6;  // spare CTAs for the row norms of B
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, name);
-    down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
+    down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                             ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm,
                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
@@ -860,26 +870,27 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
 // Picks the tile height for the down / output projection: 256-row tiles move fewer bytes per FLOP
 // (about 0.8 of the time per row), 128-row tiles quantise better over the SMs.
 int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
-                     int N, int K, int G, void* Y, int out_dtype) {
+                     int N, int K, int G, void* Y, int out_dtype, const int32_t* order) {
     const int sm = ctx->sm_count;
     const int t128 = ((T + 127) / 128) * ((N + 255) / 256), t256 = ((T + 255) / 256) * ((N + 255) / 256);
     const double cost128 = static_cast<double>((t128 + sm - 1) / sm);
     const double cost256 = static_cast<double>((t256 + sm - 1) / sm) * 2.0 * 0.8;
-    if (cost128 <= cost256) return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype);
+    if (cost128 <= cost256)
+        return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype, -1, "prefill_down", 1, nullptr, order);
     CUtensorMap tmA, tmB;
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, 256) || !make_tmap_bf16(ctx, &tmB, B, N, K, 256)) return WIDE_ERR_CUDA;
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2));
     const int grid = t256 < sm ? t256 : sm;
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
-    down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
+    down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                              ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
 template <int BN>
 int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, int T, int D,
-                  int Dff, int G, const int32_t* perm, const int32_t* counts, void* h) {
+                  int Dff, int G, const int32_t* perm, const int32_t* counts, const int32_t* token_rank, void* h) {
     CUtensorMap tmG, tmU;
     if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
     constexpr int stages = BN == 128 ? 3 : 4;
@@ -887,7 +898,7 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     WideLaunch l(ctx, s, "prefill_gateup");
     gateup_kernel<BN><<<ctx->sm_count, kGuThreads, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm,
-                                                              counts, Dff / G, T, D, Dff, G,
+                                                              counts, token_rank, Dff / G, T, D, Dff, G,
                                                               static_cast<__nv_bfloat16*>(h), ctx->d_status,
                                                               ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
@@ -897,22 +908,21 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
 
 int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
                                const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
-                               const int32_t* perm, const int32_t* counts, const int32_t* work_list,
-                               const int32_t* n_work, void* y, int out_dtype, void* h) {
+                               const int32_t* perm, const int32_t* counts, const int32_t* token_order,
+                               const int32_t* token_rank, void* y, int out_dtype, void* h) {
     if (T == 0) return WIDE_OK;
-    // inactive (token, group) pairs of H must read as zero in the down projection: the gate/up
-    // kernel's epilogue warps write those zeros themselves
-    (void)work_list;
-    (void)n_work;  // the kernel derives its own schedule from `counts`
-    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, h)
-                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, h);
+    // H [T, Dff] is kept in clustered token order when token_order / token_rank are given (row
+    // token_rank[t] holds token t), else in token order.  Inactive (token, group) pairs of H must
+    // read as zero in the down projection: the gate/up kernel's epilogue warps write those zeros.
+    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h)
+                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h);
     if (rc != WIDE_OK) return rc;
-    return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype);
+    return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype, token_order);
 }
 
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T, int D,
-                                 int K, int G, const uint32_t* mask_bits, void* y, int out_dtype,
-                                 void* a_masked) {
+                                 int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
+                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked) {
     if (T == 0) return WIDE_OK;
     const int words = (K / G + 31) / 32;
     const long long total = static_cast<long long>(T) * (K / 8);
@@ -920,11 +930,11 @@ int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, c
     if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
     {
     WideLaunch l(ctx, s, "prefill_mask_rows");
-    mask_rows_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(a), mask_bits, words, T, K, G,
-                                                              static_cast<uint4*>(a_masked));
+    mask_rows_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(a), mask_bits, token_rank, words,
+                                                              T, K, G, static_cast<uint4*>(a_masked));
     }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
-    return launch_down_auto(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype);
+    return launch_down_auto(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype, token_order);
 }
 
 // scores (fp32) = x[T, D] * w_router[NG, D]^T on the tensor cores, K split `ksplit` ways: slab ks

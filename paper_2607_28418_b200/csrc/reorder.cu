@@ -12,6 +12,70 @@ __device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_
                                int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
                                int32_t* __restrict__ offsets);
 
+// Token clustering key: 8 bits of an FNV-1a style hash over the token's mask words.  Tokens with
+// the same mask get the same key.
+__device__ __forceinline__ unsigned mask_key(const uint32_t* __restrict__ row, int words) {
+    uint32_t h = 0x811C9DC5u;
+    for (int w = 0; w < words; ++w) h = (h ^ row[w]) * 0x01000193u;
+    return h >> 24;
+}
+
+// Run by one whole CTA (kPartThreads threads): stable counting sort of the tokens by mask_key.
+// order[p] = token at clustered position p, rank[t] = position of token t.  Tokens that share a
+// mask end up next to each other, so token tiles taken in this order use few groups when the
+// router's decisions cluster.
+__device__ void cluster_tokens(const uint32_t* __restrict__ mask_bits, int T, int words, int32_t* __restrict__ order,
+                               int32_t* __restrict__ rank) {
+    constexpr int nwarps = kPartThreads / 32;
+    __shared__ unsigned s_next[256];                // next free position of every bucket
+    __shared__ unsigned short s_wcnt[nwarps][256];  // per-warp bucket counts of the current chunk
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid < 256) s_next[tid] = 0u;
+    __syncthreads();
+    for (int t = tid; t < T; t += kPartThreads) atomicAdd(&s_next[mask_key(mask_bits + static_cast<size_t>(t) * words, words)], 1u);
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive prefix over the 256 buckets: 8 per lane
+        unsigned v[8], sum = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { v[i] = s_next[lane * 8 + i]; sum += v[i]; }
+        unsigned incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned u = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += u;
+        }
+        unsigned run = incl - sum;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { s_next[lane * 8 + i] = run; run += v[i]; }
+    }
+    __syncthreads();
+    for (int c0 = 0; c0 < T; c0 += kPartThreads) {
+        const int t = c0 + tid;
+        const unsigned key = t < T ? mask_key(mask_bits + static_cast<size_t>(t) * words, words) : 0xFFFFFFFFu;
+        for (int i = tid; i < nwarps * 256; i += kPartThreads) (&s_wcnt[0][0])[i] = 0;
+        __syncthreads();
+        const unsigned peers = __match_any_sync(0xffffffffu, key);
+        const int in_warp = __popc(peers & ((1u << lane) - 1u));
+        if (t < T && in_warp == 0) s_wcnt[warp][key] = static_cast<unsigned short>(__popc(peers));
+        __syncthreads();
+        if (t < T) {
+            unsigned pos = s_next[key] + in_warp;
+            for (int w = 0; w < warp; ++w) pos += s_wcnt[w][key];
+            order[pos] = t;
+            rank[t] = static_cast<int32_t>(pos);
+        }
+        __syncthreads();
+        if (tid < 256) {
+            unsigned add = 0;
+#pragma unroll
+            for (int w = 0; w < nwarps; ++w) add += s_wcnt[w][tid];
+            s_next[tid] += add;
+        }
+        __syncthreads();
+    }
+}
+
 // One CTA per group.  Every thread owns kPerThread consecutive tokens of a chunk, so a token's
 // rank among the active rows is (active rows in earlier chunks) + (exclusive prefix over threads)
 // + (bits below it in the thread's own nibble): one warp scan and one 16-entry block scan per
@@ -39,10 +103,16 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t*
                                                                  int32_t* __restrict__ n_work,
                                                                  int32_t* __restrict__ union_list,
                                                                  int32_t* __restrict__ n_union,
-                                                                 int32_t* __restrict__ offsets, int* ticket) {
+                                                                 int32_t* __restrict__ offsets, int* ticket,
+                                                                 int32_t* __restrict__ token_order,
+                                                                 int32_t* __restrict__ token_rank) {
     __shared__ int warp_cnt[kPartThreads / 32];
     __shared__ int s_total;
     __shared__ int s_last;
+    if (static_cast<int>(blockIdx.x) == NG) {  // the extra CTA clusters the tokens
+        cluster_tokens(mask_bits, T, words, token_order, token_rank);
+        return;
+    }
     const int g = blockIdx.x;
     const int w = g >> 5, b = g & 31;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -199,12 +269,14 @@ __global__ void __launch_bounds__(256) unpermute_kernel(const uint4* __restrict_
 int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
                         int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
                         int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
-                        int32_t* offsets) {
+                        int32_t* offsets, int32_t* token_order, int32_t* token_rank) {
     const int words = (NG + 31) / 32;
     const int n_tiles = (T + tile_m - 1) / tile_m;
+    const int extra = (token_order && token_rank) ? 1 : 0;
     WideLaunch l(ctx, s, "reorder_partition");
-    partition_kernel<<<NG, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts, tile_m, n_tiles, tile_map,
-                                                 work_list, n_work, union_list, n_union, offsets, ctx->d_status + 1);
+    partition_kernel<<<NG + extra, kPartThreads, 0, s>>>(mask_bits, T, NG, words, perm, counts, tile_m, n_tiles,
+                                                         tile_map, work_list, n_work, union_list, n_union, offsets,
+                                                         ctx->d_status + 1, token_order, token_rank);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 

@@ -41,4 +41,6 @@ def meta_to_dev(meta: dict) -> dict:
         "work_list": torch.from_numpy(wl).cuda(),
         "n_work": torch.tensor([meta["n_work"]], dtype=torch.int32).cuda(),
         "offsets": torch.from_numpy(meta["offsets"]).cuda(),
+        "token_order": torch.from_numpy(meta["token_order"]).cuda(),
+        "token_rank": torch.from_numpy(meta["token_rank"]).cuda(),
     }

@@ -127,6 +127,8 @@ def _check_reorder(ctx, mask, tile_m):
     ul = out["union_list"].cpu().numpy()
     assert (ul[:nu] == ref["union_list"]).all() and (ul[nu:] == -1).all()
     assert (out["offsets"].cpu().numpy() == ref["offsets"]).all()
+    assert (out["token_order"].cpu().numpy() == ref["token_order"]).all()
+    assert (out["token_rank"].cpu().numpy() == ref["token_rank"]).all()
     return out, ref
 
 
@@ -144,6 +146,15 @@ def test_reorder_hand_worked_fixture(ctx):
                                            (300, 10, 128, 1.0), (4096, 256, 128, 0.5)])
 def test_reorder_bit_exact(ctx, T, NG, tile_m, p):
     _check_reorder(ctx, synth.bernoulli_mask(T + NG, T, NG, p), tile_m)
+
+
+def test_reorder_clusters_prototype_tokens(ctx):
+    rng = np.random.default_rng(3)
+    protos = rng.random((4, 112)) < 0.5
+    which = rng.integers(0, 4, size=1500)
+    out, ref = _check_reorder(ctx, protos[which], 128)
+    order = out["token_order"].cpu().numpy()
+    assert 1 + int((np.diff(which[order]) != 0).sum()) <= 5     # four runs (five if two keys collide)
 
 
 def test_reorder_after_route_chain_and_determinism(ctx):

@@ -31,12 +31,15 @@ def _ffn_inputs(cfg, seed, mask=None):
     return case, mask, dev
 
 
-def _run_ffn(ctx, cfg, seed, flags, mask=None, out_dtype=None, with_meta=True):
+def _run_ffn(ctx, cfg, seed, flags, mask=None, out_dtype=None, with_meta=True, clustered_order=True):
     from paper_2607_28418_b200 import binding
     case, mask, dev = _ffn_inputs(cfg, seed, mask)
     ref = wo.ffn(case["x"], case["w_gate"], case["w_up"], case["w_down"], mask, cfg.group)
     bits = bits_to_dev(wo.pack_mask_bits(mask))
     meta = meta_to_dev(wo.reorder(mask, 128)) if with_meta else None
+    if meta is not None and not clustered_order:
+        meta.pop("token_order")
+        meta.pop("token_rank")
     y = binding.wide_ffn(ctx, dev["x"], dev["w_gate"], dev["w_up"], dev["w_down"], cfg.group, bits, meta,
                          out_dtype=out_dtype, flags=flags)
     torch.cuda.synchronize()
@@ -113,6 +116,17 @@ def test_prefill_tc_closed_cases(ctx):
     m[128:, 2:] = True
     y, ref, _ = _run_ffn(ctx, cfg, 4, binding.FLAG_FORCE_PREFILL, mask=m)
     assert_close(y, ref, "block-clustered")
+
+
+def test_prefill_tc_token_order_is_optional_and_does_not_change_the_result(ctx):
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("t", tokens=700, hidden=512, d_ff=2048, group=128, k=6, router="clustered")
+    y1, ref, mask = _run_ffn(ctx, cfg, 14, binding.FLAG_FORCE_PREFILL)
+    y2, _, _ = _run_ffn(ctx, cfg, 14, binding.FLAG_FORCE_PREFILL, clustered_order=False)
+    assert len({r.tobytes() for r in mask}) <= 4
+    assert_close(y1, ref, "clustered order")
+    assert_close(y2, ref, "original order")
+    assert_close(y1, y2.float().cpu().numpy().astype(np.float64), "same result either way", rel=1e-2)
 
 
 def test_prefill_tc_agrees_with_simt_and_is_deterministic(ctx):

@@ -209,6 +209,39 @@ def test_union_single_token_is_its_own_groups():
     assert r["n_union"] == 13
 
 
+# ----------------------------------------------------------------------------- token clustering
+def test_cluster_tokens_permutation_grouping_and_stability():
+    rng = np.random.default_rng(12)
+    T, NG = 300, 70
+    protos = rng.random((5, NG)) < 0.5
+    which = rng.integers(0, 5, size=T)
+    mask = protos[which]
+    c = wo.cluster_tokens(mask)
+    order, rank = c["token_order"], c["token_rank"]
+    assert sorted(order.tolist()) == list(range(T))
+    assert (rank[order] == np.arange(T)).all() and (order[rank] == np.arange(T)).all()
+    bits = wo.pack_mask_bits(mask)
+    keys = np.array([wo.mask_key(bits[t]) for t in range(T)])
+    assert ((0 <= keys) & (keys < 256)).all()
+    assert (np.diff(keys[order]) >= 0).all()                        # sorted by key
+    for p in range(T - 1):                                           # stable inside a key
+        if keys[order[p]] == keys[order[p + 1]]:
+            assert order[p] < order[p + 1]
+    # identical masks are neighbours unless two prototypes collide on the 8-bit key
+    proto_keys = {wo.mask_key(wo.pack_mask_bits(protos[i:i + 1])[0]) for i in range(5)}
+    if len(proto_keys) == 5:
+        runs = 1 + int((np.diff(which[order]) != 0).sum())
+        assert runs == len(set(which.tolist()))
+
+
+def test_mask_key_is_the_header_hash():
+    # two worked values of h = (h ^ w) * 0x01000193 from h0 = 0x811C9DC5, top byte
+    assert wo.mask_key([0]) == ((0x811C9DC5 * 0x01000193) & 0xFFFFFFFF) >> 24
+    h = ((0x811C9DC5 ^ 0xFFFFFFFF) * 0x01000193) & 0xFFFFFFFF
+    h = ((h ^ 0x1) * 0x01000193) & 0xFFFFFFFF
+    assert wo.mask_key([0xFFFFFFFF, 1]) == h >> 24
+
+
 # ----------------------------------------------------------------------------- gather / scatter
 def test_gather_then_unpermute_full_mask_is_identity():
     rng = np.random.default_rng(8)
