@@ -106,208 +106,274 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 
 
 // ---------------------------------------------------------------------------- fast path (bf16)
-// Scores come from the tensor cores in fp32 (exact products, fp32 accumulation).  Their error is
-// bounded by eps_t = kAccumErr * D * ||x_t|| * max_g ||w_g|| (Cauchy-Schwarz on the sum of absolute
-// products times a per-step accumulation error).  A group whose fp32 score is further than
-// 2*eps_t from the selection boundary keeps its fp32 decision; the few groups inside that band
-// get their score recomputed exactly in fp64, and the band is re-ranked on those exact values.
-// The result equals the fp64 decision of the slow path.
+// Scores come from the tensor cores in fp32 (exact products, fp32 accumulation), as `nsplit`
+// partial slabs over K that are summed here in fp32.  Their error is bounded by
+//   eps_t = kAccumErr * (D / nsplit + nsplit) * ||x_t|| * max_g ||w_g||
+// (a per-element accumulation error along each slab's chain plus the slab sum, times the
+// Cauchy-Schwarz bound on the sum of absolute products).  A group whose fp32 score is further
+// than 2*eps_t from the selection boundary keeps its fp32 decision; the few groups inside that
+// band get their score recomputed exactly in fp64, and the band is re-ranked on those exact
+// values.  The result equals the fp64 decision of the slow path.
 constexpr float kAccumErr = 5.9604645e-8f;  // 2^-24 per accumulated element
 
-constexpr int kSelWarps = 4;   // tokens (warps) per CTA in select_band_kernel
-constexpr int kBatch = 4;      // 16-byte loads in flight per lane
+constexpr int kSelTokens = 2;  // tokens per CTA in select_band_kernel (two warps each)
+constexpr int kBatch = 8;      // 16-byte loads in flight per lane and operand
+constexpr int kMaxSlabs = 8;   // K-split partial score slabs summed by select_band_kernel
+constexpr int kBandMax = 16;   // band members re-scored per token between two block barriers
 
-// Exact x_t . w_g in fp64 by one warp: x row in shared memory, w row streamed from L2 with
-// kBatch loads in flight per lane (bf16 products are exact in fp64).
-__device__ __forceinline__ double warp_dot_f64(const uint4* __restrict__ xs, const __nv_bfloat16* __restrict__ wrow,
+// Exact x_t . w_g in fp64 by one warp, both rows streamed from L2 (bf16 products are exact in
+// fp64).  Four independent accumulators keep the dependent chain of fp64 FMAs short.  The result
+// is valid in every lane.
+__device__ __forceinline__ double warp_dot_f64(const __nv_bfloat16* __restrict__ xrow, const __nv_bfloat16* __restrict__ wrow,
                                                int nch, int lane) {
+    const uint4* xv = reinterpret_cast<const uint4*>(xrow);
     const uint4* wv = reinterpret_cast<const uint4*>(wrow);
-    double acc = 0.0;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
     for (int base = 0; base < nch; base += 32 * kBatch) {
-        uint4 b[kBatch];
+        uint4 a[kBatch], b[kBatch];
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
             const int i = base + lane + 32 * j;
-            b[j] = i < nch ? wv[i] : make_uint4(0u, 0u, 0u, 0u);
+            a[j] = i < nch ? __ldg(xv + i) : make_uint4(0u, 0u, 0u, 0u);
+            b[j] = i < nch ? __ldg(wv + i) : make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
-            const int i = base + lane + 32 * j;
-            if (i < nch) {
-                const uint4 a = xs[i];
-                const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
-                const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b[j]);
+            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a[j]);
+            const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b[j]);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 fa = __bfloat1622float2(ah[e]), fb = __bfloat1622float2(bh[e]);
-                    acc = fma(static_cast<double>(fa.x), static_cast<double>(fb.x), acc);
-                    acc = fma(static_cast<double>(fa.y), static_cast<double>(fb.y), acc);
-                }
+            for (int e = 0; e < 4; ++e) {
+                const float2 fa = __bfloat1622float2(ah[e]), fb = __bfloat1622float2(bh[e]);
+                acc[e] = fma(static_cast<double>(fa.x), static_cast<double>(fb.x), acc[e]);
+                acc[e] = fma(static_cast<double>(fa.y), static_cast<double>(fb.y), acc[e]);
             }
         }
     }
+    double r = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    return acc;
+    for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+    return r;
 }
 
-// One CTA (4 warps) per token.  scores: nsplit partial slabs [nsplit][T, ld] that are summed on
-// load.  Thread g ranks group g (and g + 128); the exact re-scoring of the band is spread over
-// the four warps.
-__global__ void __launch_bounds__(32 * kSelWarps, 12)
+// Two warps per token, two tokens per CTA.  What bounds this kernel is the length of one warp's
+// chain of dependent instructions and load round trips, not throughput, so the two independent
+// halves of the work run side by side: the SELECT warp sums the score slabs and finds the kt-th
+// largest, the NORM warp reads the x row for ||x_t||.  Lane l of the select warp holds the groups
+// g = 32*j + l, j < KPL, which is also the layout of the packed mask words.  Scores map to
+// unsigned keys that order like the floats; the kt-th largest key is found by a 32-step binary
+// search on its bits with warp votes (no quadratic rank count), ties at that key go to the lower
+// group index.  Band members (rare) are re-scored by all four warps of the CTA.
+template <int KPL>
+__global__ void __launch_bounds__(64 * kSelTokens, 8)   // every CTA of a 2048-token batch resident at once
 select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
                    const __nv_bfloat16* __restrict__ w, const float* __restrict__ wnorm, int T, int NG, int D, int k,
                    const int32_t* __restrict__ k_per_token, uint32_t* __restrict__ mask_bits,
                    float* __restrict__ scores_out) {
-    extern __shared__ uint4 sh_x[];  // [D / 8]
-    __shared__ float s[WIDE_MAX_GROUPS];
-    __shared__ __align__(16) unsigned long long skey[WIDE_MAX_GROUPS + 2];  // (ordered score bits, NG - index)
-    __shared__ double ex[WIDE_MAX_GROUPS];
-    __shared__ int band[WIDE_MAX_GROUPS];
-    __shared__ float red[2 * kSelWarps];
-    __shared__ float sh_b[2];
-    __shared__ int n_band, n_band_hi;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int t = blockIdx.x;
+    __shared__ float s_xsq[kSelTokens];
+    __shared__ int s_nb[kSelTokens];
+    __shared__ int s_band[kSelTokens][kBandMax];
+    __shared__ double s_ex[kSelTokens][kBandMax];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int tt = warp >> 1;                       // token slot in the CTA
+    const bool select_warp = (warp & 1) == 0;
+    const int t = blockIdx.x * kSelTokens + tt;
+    const bool live = t < T;                        // warp-uniform
     const int nch = D / 8;
     const int words = (NG + 31) >> 5;
     const size_t slab = static_cast<size_t>(T) * ld;
-    constexpr int kThreads = 32 * kSelWarps;
-    constexpr int kPer = WIDE_MAX_GROUPS / kThreads;  // groups per thread (2)
-
-    float wmax = 0.f;
-#pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        const int g = tid + q * kThreads;
-        if (g < NG) {
-            float v = 0.f;
-            for (int ks = 0; ks < nsplit; ++ks) v += scores[ks * slab + static_cast<size_t>(t) * ld + g];
-            s[g] = v;
-            // total order "score descending, index ascending" as one unsigned 64-bit compare
-            const uint32_t u = __float_as_uint(v + 0.0f);  // -0 -> +0
-            const uint32_t ord = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-            skey[g] = (static_cast<unsigned long long>(ord) << 32) | static_cast<uint32_t>(NG - g);
-            wmax = fmaxf(wmax, wnorm[g]);
-            if (scores_out) scores_out[static_cast<size_t>(t) * NG + g] = v;
-        } else if (g < NG + 2) {
-            skey[g] = 0ull;  // padding: beats nobody
-        }
-    }
-    const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const int kt = live ? min(max(k_per_token ? k_per_token[t] : k, 0), NG) : 0;
     const bool boundary = kt > 0 && kt < NG;
 
-    // x row -> shared memory, partial ||x_t||^2 on the way
-    float xsq = 0.f;
-    if (boundary) {
-        const uint4* xv = reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * D);
-        for (int base = 0; base < nch; base += kThreads * kBatch) {
-            uint4 a[kBatch];
+    float sv[KPL];
+    uint32_t key[KPL];   // 0 for slots past NG, >= 1 for real groups
+    bool sel[KPL], in_band[KPL];
+    float wmax = 0.f, v_k = 0.f, v_k1 = 0.f;
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int i = base + tid + kThreads * j;
-                a[j] = i < nch ? xv[i] : make_uint4(0u, 0u, 0u, 0u);
-            }
+    for (int j = 0; j < KPL; ++j) { sv[j] = 0.f; key[j] = 0u; sel[j] = false; in_band[j] = false; }
+
+    if (!select_warp) {
+        // ------------------------------------------------------------ NORM warp: ||x_t||^2
+        float q[4] = {0.f, 0.f, 0.f, 0.f};
+        if (boundary) {
+            const uint4* xv = reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * D);
+            for (int base = 0; base < nch; base += 32 * kBatch) {
+                uint4 a[kBatch];
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int i = base + tid + kThreads * j;
-                if (i < nch) {
-                    sh_x[i] = a[j];
+                for (int j = 0; j < kBatch; ++j) {
+                    const int i = base + lane + 32 * j;
+                    a[j] = i < nch ? __ldg(xv + i) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
                     const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a[j]);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 f = __bfloat1622float2(ah[e]);
-                        xsq = fmaf(f.x, f.x, fmaf(f.y, f.y, xsq));
+                        q[e] = fmaf(f.x, f.x, fmaf(f.y, f.y, q[e]));
                     }
                 }
             }
         }
-    }
+        float xsq = (q[0] + q[1]) + (q[2] + q[3]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
-        wmax = fmaxf(wmax, __shfl_xor_sync(0xffffffffu, wmax, o));
-    }
-    if (lane == 0) { red[warp] = xsq; red[kSelWarps + warp] = wmax; }
-    if (tid == 0) { sh_b[0] = 0.f; sh_b[1] = 0.f; n_band = 0; n_band_hi = 0; }
-    __syncthreads();
-    xsq = 0.f;
-    wmax = 0.f;
+        for (int o = 16; o > 0; o >>= 1) xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
+        if (lane == 0) s_xsq[tt] = xsq;
+    } else if (live) {
+        // ------------------------------------------------------------ SELECT warp
+        // scores: every slab load of the warp is issued before the first sum
+        float part[KPL][kMaxSlabs];
+        float wn[KPL];
 #pragma unroll
-    for (int i = 0; i < kSelWarps; ++i) { xsq += red[i]; wmax = fmaxf(wmax, red[kSelWarps + i]); }
-
-    // fp32 ranks; remember the k-th and (k+1)-th largest
-    int rank[kPer];
+        for (int j = 0; j < KPL; ++j) {
+            const int g = 32 * j + lane;
+            const float* sp = scores + static_cast<size_t>(t) * ld + g;
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        rank[q] = NG;
-        const int g = tid + q * kThreads;
-        if (g < NG) {
-            const float v = s[g];
-            const unsigned long long mine = skey[g];
-            int beats = 0;
-            const ulonglong2* kp = reinterpret_cast<const ulonglong2*>(skey);
-#pragma unroll 4
-            for (int h = 0; h < (NG + 1) / 2; ++h) {
-                const ulonglong2 kk = kp[h];
-                beats += (kk.x > mine) + (kk.y > mine);
+            for (int ks = 0; ks < kMaxSlabs; ++ks) part[j][ks] = (g < NG && ks < nsplit) ? __ldg(sp + ks * slab) : 0.f;
+            wn[j] = g < NG ? __ldg(wnorm + g) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            const int g = 32 * j + lane;
+            float v = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < kMaxSlabs; ++ks) v += part[j][ks];
+            v += 0.0f;  // -0 -> +0
+            sv[j] = v;
+            const uint32_t u = __float_as_uint(v);
+            const uint32_t ord = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+            key[j] = g < NG ? max(ord, 1u) : 0u;
+            wmax = fmaxf(wmax, wn[j]);
+            sel[j] = kt == NG && g < NG;
+            if (scores_out && g < NG) scores_out[static_cast<size_t>(t) * NG + g] = v;
+        }
+        if (boundary) {
+            wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(wmax)));  // norms are >= 0
+            // kt-th largest key
+            uint32_t key_k = 0u;
+#pragma unroll 8
+            for (int bit = 31; bit >= 0; --bit) {
+                const uint32_t cand = key_k | (1u << bit);
+                int c = 0;
+#pragma unroll
+                for (int j = 0; j < KPL; ++j) c += __popc(__ballot_sync(0xffffffffu, key[j] >= cand));
+                if (c >= kt) key_k = cand;
             }
-            rank[q] = beats;
-            if (beats == kt - 1) sh_b[0] = v;
-            if (beats == kt) sh_b[1] = v;
+            int n_gt = 0;
+#pragma unroll
+            for (int j = 0; j < KPL; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, key[j] > key_k));
+            const int need = kt - n_gt;   // how many of the groups tied at key_k are taken (>= 1)
+            int n_tie = 0;
+            uint32_t below = 0u;          // largest key under key_k
+#pragma unroll
+            for (int j = 0; j < KPL; ++j) {
+                const bool tie = key[j] == key_k;
+                const uint32_t b = __ballot_sync(0xffffffffu, tie);
+                sel[j] = key[j] > key_k || (tie && n_tie + __popc(b & lt_mask) < need);
+                n_tie += __popc(b);
+                if (key[j] < key_k) below = max(below, key[j]);
+            }
+            below = __reduce_max_sync(0xffffffffu, below);
+            // kt-th and (kt+1)-th largest scores, back from their keys; the latter is the tied
+            // value itself when more groups tie than are taken
+            v_k = __uint_as_float((key_k & 0x80000000u) ? (key_k & 0x7fffffffu) : ~key_k);
+            v_k1 = n_tie > need ? v_k : __uint_as_float((below & 0x80000000u) ? (below & 0x7fffffffu) : ~below);
         }
     }
-    __syncthreads();
-    const float v_k = sh_b[0], v_k1 = sh_b[1];
+    __syncthreads();   // ||x_t||^2 is there
+
     // band half-width 2 * eps_t (a little slack for the fp32 evaluation of the bound itself)
-    const float tau = boundary ? 2.f * kAccumErr * static_cast<float>(D) * sqrtf(xsq) * 1.0001f * wmax : 0.f;
-
-    bool in_band[kPer];
+    int nb = 0, m_hi = 0;
+    if (select_warp && boundary) {
+        const float steps = static_cast<float>((D + nsplit - 1) / nsplit + nsplit);
+        const float tau = 2.f * kAccumErr * steps * sqrtf(s_xsq[tt]) * 1.0001f * wmax;
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        in_band[q] = false;
-        const int g = tid + q * kThreads;
-        if (boundary && g < NG) {
-            const bool hi = rank[q] < kt;
-            const bool u = hi ? (s[g] - v_k1 <= tau) : (v_k - s[g] <= tau);
-            if (u) {
-                in_band[q] = true;
-                band[atomicAdd(&n_band, 1)] = g;
-                if (hi) atomicAdd(&n_band_hi, 1);
+        for (int j = 0; j < KPL; ++j) {
+            const bool valid = key[j] != 0u;
+            in_band[j] = valid && (sel[j] ? (sv[j] - v_k1 <= tau) : (v_k - sv[j] <= tau));
+            const uint32_t b = __ballot_sync(0xffffffffu, in_band[j]);
+            if (in_band[j]) {
+                const int slot = nb + __popc(b & lt_mask);
+                if (slot < kBandMax) s_band[tt][slot] = 32 * j + lane;
             }
+            nb += __popc(b);
+            m_hi += __popc(__ballot_sync(0xffffffffu, in_band[j] && sel[j]));
         }
     }
-    __syncthreads();
-    const int nb = n_band, m_hi = n_band_hi;
-    for (int i = warp; i < nb; i += kSelWarps) {
-        const int gg = band[i];
-        const double e = warp_dot_f64(sh_x, w + static_cast<size_t>(gg) * D, nch, lane);
-        if (lane == 0) ex[gg] = e;
-    }
-    __syncthreads();
+    if (select_warp && lane == 0) s_nb[tt] = nb;
+    __syncthreads();   // band lists are there
 
-    // final decision: band members are re-ranked among themselves on the exact scores
+    // Exact re-scoring.  The common case (at most kBandMax members per token) is spread over all
+    // warps of the CTA; a longer band is re-scored by its own select warp alone.
+    int total = 0;
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-        const int g = tid + q * kThreads;
-        bool sel = false;
-        if (g < NG) {
-            if (in_band[q]) {
-                const double v = ex[g];
-                int beats = 0;
-                for (int i = 0; i < nb; ++i) {
-                    const int h = band[i];
-                    const double u = ex[h];
-                    beats += (u > v) || (u == v && h < g);
-                }
-                sel = beats < m_hi;
+    for (int i = 0; i < kSelTokens; ++i) total += min(s_nb[i], kBandMax);
+    if (total > 0) {
+        for (int item = warp; item < total; item += 2 * kSelTokens) {
+            int tok = 0, i = item;
+            while (i >= min(s_nb[tok], kBandMax)) { i -= min(s_nb[tok], kBandMax); ++tok; }
+            const int t2 = blockIdx.x * kSelTokens + tok;
+            const double e = warp_dot_f64(x + static_cast<size_t>(t2) * D, w + static_cast<size_t>(s_band[tok][i]) * D, nch, lane);
+            if (lane == 0) s_ex[tok][i] = e;
+        }
+    }
+    __syncthreads();   // exact scores are there
+
+    if (select_warp && nb > 0) {   // then the band holds at least the two groups on either side of the boundary
+        double ex[KPL];
+        int seen = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            ex[j] = 0.0;
+            uint32_t bits = __ballot_sync(0xffffffffu, in_band[j]);
+            const int first = seen;
+            seen += __popc(bits);
+            if (nb <= kBandMax) {
+                if (in_band[j]) ex[j] = s_ex[tt][first + __popc(bits & lt_mask)];
             } else {
-                sel = rank[q] < kt;
+                while (bits) {
+                    const int l = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    const double e = warp_dot_f64(x + static_cast<size_t>(t) * D, w + static_cast<size_t>(32 * j + l) * D, nch, lane);
+                    if (lane == l) ex[j] = e;
+                }
             }
         }
-        const unsigned word = __ballot_sync(0xffffffffu, sel);
-        const int widx = warp + q * kSelWarps;
-        if (lane == 0 && widx < words) mask_bits[static_cast<size_t>(t) * words + widx] = word;
+        // band members are re-ranked among themselves on the exact scores
+        int beats[KPL];
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) beats[j] = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            uint32_t bits = __ballot_sync(0xffffffffu, in_band[j]);
+            while (bits) {
+                const int l = __ffs(bits) - 1;
+                bits &= bits - 1;
+                const double u = __shfl_sync(0xffffffffu, ex[j], l);
+                const int h = 32 * j + l;
+#pragma unroll
+                for (int jj = 0; jj < KPL; ++jj) beats[jj] += (u > ex[jj]) || (u == ex[jj] && h < 32 * jj + lane);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < KPL; ++j)
+            if (in_band[j]) sel[j] = beats[j] < m_hi;
     }
+    if (select_warp && live) {
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            const uint32_t word = __ballot_sync(0xffffffffu, sel[j]);
+            if (lane == 0 && j < words) mask_bits[static_cast<size_t>(t) * words + j] = word;
+        }
+    }
+}
+
+template <int KPL>
+void launch_select_band(cudaStream_t s, int T, const float* sc32, int ksplit, int ld, const __nv_bfloat16* x,
+                        const __nv_bfloat16* w, const float* wn, int NG, int D, int k, const int32_t* k_per_token,
+                        uint32_t* mask_bits, float* scores) {
+    select_band_kernel<KPL><<<(T + kSelTokens - 1) / kSelTokens, 64 * kSelTokens, 0, s>>>(
+        sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores);
 }
 
 template <typename TA, typename TB>
@@ -341,17 +407,22 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
         // as many K-split slabs as the first part of the workspace holds (at most 8)
         const size_t part0 = wide_route_workspace(T, NG, rank) - 1024;
         int max_split = static_cast<int>(part0 / (static_cast<size_t>(T) * ld * sizeof(float)));
-        if (max_split > 8) max_split = 8;
+        if (max_split > kMaxSlabs) max_split = kMaxSlabs;
         if (max_split < 1) max_split = 1;
         int ksplit = 1;
         const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32, wn, max_split, &ksplit);
         if (rc != WIDE_OK) return rc;
-        const int sel_smem = (D / 8) * static_cast<int>(sizeof(uint4));
-        WIDE_CUDA_CHECK(cudaFuncSetAttribute(select_band_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sel_smem));
         WideLaunch l(ctx, s, "route_select_band");
-        select_band_kernel<<<T, 32 * kSelWarps, sel_smem, s>>>(
-            sc32, ksplit, ld, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router), wn, T,
-            NG, D, k, k_per_token, mask_bits, scores);
+        const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+        const __nv_bfloat16* wb = static_cast<const __nv_bfloat16*>(w_router);
+        switch ((NG + 31) / 32) {   // mask words per token = groups held per lane
+#define WIDE_SEL_CASE(n) \
+    case n: launch_select_band<n>(s, T, sc32, ksplit, ld, xb, wb, wn, NG, D, k, k_per_token, mask_bits, scores); break;
+            WIDE_SEL_CASE(1) WIDE_SEL_CASE(2) WIDE_SEL_CASE(3) WIDE_SEL_CASE(4)
+            WIDE_SEL_CASE(5) WIDE_SEL_CASE(6) WIDE_SEL_CASE(7) WIDE_SEL_CASE(8)
+#undef WIDE_SEL_CASE
+            default: return WIDE_ERR_UNSUPPORTED_SHAPE;
+        }
         return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
     }
     double* sc = static_cast<double*>(ws);
