@@ -553,7 +553,14 @@ struct GuSched {
     }
 };
 
-__device__ __forceinline__ float silu_mul_fast(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+// silu(g) * u with one special-function instruction: silu(g) = h + h * tanh(h), h = g / 2
+// (tanh.approx is good to about 2^-11, below the bf16 rounding of the result).
+__device__ __forceinline__ float silu_mul_fast(float g, float u) {
+    const float h = 0.5f * g;
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(h));
+    return fmaf(h, t, h) * u;
+}
 
 constexpr int kGuThreads = 448;  // TMA, MMA, 4 gather warps, 8 epilogue warps
 
@@ -739,6 +746,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         const int chalf = ew >> 2;
         const int e = ew * 32 + lane;  // 0..255
         constexpr int kCh = BN / 2;    // channels per epilogue warp
+        uint4* ep_stage = reinterpret_cast<uint4*>(base + kStagesG * kStageBytes + 128) + ew * 128;  // 2 KB per warp
         int tc = 0;
         bool ok = true;
         GuSched sched(s_dbl, s_sgl, n_gs);
@@ -751,28 +759,36 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                 // rows of H (sorted positions [c, T) split evenly over the group's row tiles), so
                 // that the down projection reads exact zeros for every inactive (token, group) pair
                 // of a group that is active anywhere.  Groups nobody selected are never read.
+                // kLpr consecutive lanes write one row's piece, so a warp store touches whole
+                // lines (scattered 16-byte stores would keep the L1 busy and starve the gather).
+                constexpr int kLpr = BN / 8;          // lanes per row: one 16-byte store each
+                constexpr int kRows = 256 / kLpr;     // rows per sweep of the 8 warps
                 const int nt = (c + kBM - 1) / kBM;
                 const int per = (T - c + nt - 1) / nt;
+                const int zr = e / kLpr, zp = e % kLpr;
                 for (int mm = w.m; mm < w.m + w.rows / kBM; ++mm) {
                     const int j0 = c + mm * per;
                     const int j1 = min(T, j0 + per);
-                    for (int jj = j0 + e; jj < j1; jj += 256) {
+                    for (int jj = j0 + zr; jj < j1; jj += kRows) {
                         int tz = perm[static_cast<size_t>(g) * T + jj];
                         if (token_rank) tz = token_rank[tz];   // H rows are kept in clustered token order
-                        uint4* z = reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN);
-#pragma unroll
-                        for (int v = 0; v < BN / 8; ++v) z[v] = make_uint4(0u, 0u, 0u, 0u);
+                        reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN)[zp] =
+                            make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
+            }
+            // the H rows of this item's tokens, fetched before the accumulators are ready
+            int tokh[2];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int j = (w.m + half) * kBM + q * 32 + lane;
+                int tok = (half < w.rows / kBM && j < c) ? perm[static_cast<size_t>(g) * T + j] : -1;
+                if (tok >= 0 && token_rank) tok = token_rank[tok];   // H rows are kept in clustered token order
+                tokh[half] = tok;
             }
             if (!mbar_wait(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             for (int half = 0; half < w.rows / kBM; ++half) {
-                const int j = (w.m + half) * kBM + q * 32 + lane;
-                const bool live = j < c;
-                int tok = live ? perm[static_cast<size_t>(g) * T + j] : 0;
-                if (live && token_rank) tok = token_rank[tok];   // H rows are kept in clustered token order
-                __nv_bfloat16* hrow = H + static_cast<size_t>(tok) * Dff + g * G + sub * BN + chalf * kCh;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256 + chalf * kCh;
 #pragma unroll 1
                 for (int c0 = 0; c0 < kCh; c0 += 32) {
@@ -780,20 +796,31 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     tmem_ld_32x32(taddr + c0, gr);
                     tmem_ld_32x32(taddr + BN + c0, ur);
                     tmem_ld_wait();
-                    if (live) {
-                        uint4* dst = reinterpret_cast<uint4*>(hrow + c0);
+                    // lane = row here; transpose through shared memory so that 4 lanes write one
+                    // row's 64 bytes (a warp store then touches 8 rows instead of 32)
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint32_t o[4];
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t o[4];
 #pragma unroll
-                            for (int x4 = 0; x4 < 4; ++x4) {
-                                const int i = 8 * v + 2 * x4;
-                                o[x4] = pack_bf16(silu_mul_fast(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
-                                                  silu_mul_fast(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
-                            }
-                            dst[v] = make_uint4(o[0], o[1], o[2], o[3]);
+                        for (int x4 = 0; x4 < 4; ++x4) {
+                            const int i = 8 * v + 2 * x4;
+                            o[x4] = pack_bf16(silu_mul_fast(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
+                                              silu_mul_fast(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
                         }
+                        // piece v of row `lane` sits in slot v ^ ((lane >> 1) & 3): no bank conflicts
+                        // on the way in (8 rows, one piece) nor on the way out (2 rows, 4 pieces)
+                        ep_stage[lane * 4 + (v ^ ((lane >> 1) & 3))] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = 8 * i + (lane >> 2), pc = lane & 3;
+                        const int tr = __shfl_sync(0xffffffffu, tokh[half], r);
+                        const uint4 val = ep_stage[r * 4 + (pc ^ ((r >> 1) & 3))];
+                        if (tr >= 0)
+                            *reinterpret_cast<uint4*>(H + static_cast<size_t>(tr) * Dff + g * G + sub * BN + chalf * kCh + c0 + pc * 8) = val;
+                    }
+                    __syncwarp();
                 }
             }
             tc_fence_before_sync();
@@ -894,7 +921,7 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
     CUtensorMap tmG, tmU;
     if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
     constexpr int stages = BN == 128 ? 3 : 4;
-    constexpr int smem = stages * (2 * kABytes + 2 * BN * kBK * 2) + (2 * stages + 2) * 8 + 16 + 1024;
+    constexpr int smem = stages * (2 * kABytes + 2 * BN * kBK * 2) + 128 + 8 * 2048 + 1024;  // ring, barriers, epilogue staging
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     WideLaunch l(ctx, s, "prefill_gateup");
     gateup_kernel<BN><<<ctx->sm_count, kGuThreads, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm,
