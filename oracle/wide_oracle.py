@@ -22,6 +22,11 @@ ffn                   Eq. 3 literally: (phi(X Wg^T) * (X Wu^T)) gated group-wise
                       mask, times Wd^T, with phi = SiLU.
 oproj                 Eq. 2 / Eq. 10: (A gated group-wise) Wo^T.
 unpermute/gather      the scatter epilogue of Algorithm 2 as a standalone step.
+masked_attention      Eq. 1 with the head-group mask of Section 3.1 and the causal key
+                      range of Algorithm 4 (delta = T_k - T_q): plain softmax attention
+                      for every active (token, head group) pair, zeros elsewhere.  The
+                      tiling, online softmax and pipelines of Algorithm 4 reach this
+                      result up to rounding order, so the oracle is the definition.
 
 Parity pins (tests/test_oracle_*.py): exact-rational brute force for scores and
 top-k, closed-form one-hot routers, hand-worked reorder fixture, permutation /
@@ -29,7 +34,9 @@ monotonicity / boundary-tile invariants, dense-SwiGLU special case against a lib
 routine, brute-force single-group sums, additivity over disjoint masks (Eq. 10), the
 per-token gather formulation of Appendix A, constant-weight closed forms; token
 clustering: permutation / inverse / sortedness / stability / grouping properties and
-two hand-expanded hash values.
+two hand-expanded hash values; attention: a library attention routine for the all-ones
+mask (MHA and GQA, with and without a key prefix), single-key / constant-V / zero-Q closed
+forms, an explicit-loop brute force, key-shift invariance, exact zeros for inactive pairs.
 "Parity to values printed in the paper": unpinned -- the paper prints no worked
 numeric example for this path.
 
@@ -223,6 +230,43 @@ def oproj(attn_out: ArrayLike, w_o: ArrayLike, mask: np.ndarray, group: int) -> 
 
 
 # ----------------------------------------------------------------------------- gather / scatter
+def masked_attention(q: ArrayLike, k: ArrayLike, v: ArrayLike, mask: np.ndarray, heads_per_group: int,
+                     causal: bool = True, scale: Optional[float] = None) -> np.ndarray:
+    """Head-group-masked softmax attention (Eq. 1, Section 3.1; key range of Algorithm 4).
+
+    q [T_q, H_q, d]; k, v [T_k, H_kv, d] (H_q a multiple of H_kv: query head h reads KV head
+    h // (H_q / H_kv)); mask [T_q, N_G] bool with routing group g = heads [g*hpg, (g+1)*hpg).
+    For an active pair (t, g) and each head h of g:
+        o[t, h] = sum_j softmax_j(scale * q[t, h] . k[j, h_kv]) * v[j, h_kv]
+    over keys j <= t + (T_k - T_q) when causal, all keys otherwise; scale defaults to
+    1/sqrt(d).  Inactive pairs give exact zeros, and so does a query that sees no key at all
+    (t + T_k - T_q < 0; Algorithm 4 leaves such a row's state at its zero initial value).
+    """
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    t_q, h_q, d = q.shape
+    t_k, h_kv, _ = k.shape
+    rep = h_q // h_kv
+    delta = t_k - t_q
+    sc = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    out = np.zeros((t_q, h_q, d))
+    key_pos = np.arange(t_k)[None, :]
+    qry_pos = np.arange(t_q)[:, None] + delta
+    for h in range(h_q):
+        rows = np.nonzero(mask[:, h // heads_per_group])[0]
+        if rows.size == 0:
+            continue
+        s = sc * (q[rows, h, :] @ k[:, h // rep, :].T)            # [rows, T_k]
+        if causal:
+            seen = qry_pos[rows, 0] >= 0          # a query before the first key sees nothing: zeros
+            rows, s = rows[seen], s[seen]
+            s = np.where(key_pos <= qry_pos[rows], s, -np.inf)
+        s = s - s.max(axis=1, keepdims=True)
+        p = np.exp(s)
+        p /= p.sum(axis=1, keepdims=True)
+        out[rows, h, :] = p @ v[:, h // rep, :]
+    return out
+
+
 def gather_packed(dense: np.ndarray, perm: np.ndarray, counts: np.ndarray,
                   offsets: np.ndarray, group: int) -> np.ndarray:
     """Dense [T, N_G*G] -> packed-sorted [offsets[N_G], G]: row offsets[g]+j holds the
