@@ -6,6 +6,7 @@
  *   wide_reorder    per-group mask reordering + tile predicates   (Section 3.3, Eq. 6-8, Algorithm 1)
  *   wide_ffn        block-skipping SwiGLU FFN                     (Eq. 3; Algorithms 2 and 3)
  *   wide_oproj      head-group-masked attention output projection (Eq. 2; Eq. 10, Algorithm 3)
+ *   wide_attn       head-group-masked causal attention, prefill   (Eq. 1; Algorithm 4)
  *   wide_unpermute  the scatter epilogue as a standalone step     (Algorithm 2, epilogue)
  *
  * General rules
@@ -229,6 +230,31 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
                const int32_t* perm, const int32_t* counts, const int32_t* token_order,
                const int32_t* token_rank, void* y, int out_dtype, void* workspace,
                size_t workspace_bytes, unsigned flags);
+
+/*
+ * wide_attn -- Eq. 1 under the head-group mask, prefill form of Algorithm 4.  For every active
+ * pair (token t, routing group g) and every query head h of g:
+ *     o[t, h, :] = sum_j softmax_j(scale * q[t, h, :] . k[j, h_kv, :]) v[j, h_kv, :]
+ * over the keys j <= t + (tokens_k - tokens_q) when causal != 0, over all keys otherwise;
+ * h_kv = h / (n_q_heads / n_kv_heads), routing group g = h / heads_per_group.  Inactive pairs,
+ * and queries that see no key, give exact zeros.  K and V are dense (every token has them).
+ *
+ *   q   [tokens_q, n_q_heads * head_dim]  bf16, head-major (one sequence; tokens are positions)
+ *   k,v [tokens_k, n_kv_heads * head_dim] bf16
+ *   perm [n_groups, tokens_q], counts [n_groups]: outputs of wide_reorder for the attention mask
+ *       [tokens_q, n_groups], n_groups = n_q_heads / heads_per_group <= WIDE_MAX_GROUPS
+ *   scale: multiplies the logits (<= 0 selects 1/sqrt(head_dim))
+ *   o   out [tokens_q, n_q_heads * head_dim] bf16, fully overwritten
+ * All device pointers, 16-byte aligned, owned by the caller; nothing is allocated; work is
+ * enqueued on `stream`.  Needs dtype bf16, head_dim 64 or 128, n_q_heads % n_kv_heads == 0,
+ * n_q_heads % heads_per_group == 0.
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, ALIGNMENT, CUDA; a bounded device wait that expires
+ * sets the status word (WIDE_ERR_TIMEOUT from wide_status).
+ */
+WIDE_API int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const void* v, int dtype,
+              int tokens_q, int tokens_k, int n_q_heads, int n_kv_heads, int head_dim,
+              int heads_per_group, const int32_t* perm, const int32_t* counts, int causal, float scale,
+              void* o, unsigned flags);
 
 /*
  * wide_unpermute -- scatter epilogue of Algorithm 2 as its own call: packed-sorted rows back to

@@ -27,7 +27,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
            "wide_profile_end", "wide_launch_count", "wide_strerror",
            "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_ffn",
-           "wide_oproj", "wide_unpermute"]
+           "wide_oproj", "wide_attn", "wide_unpermute"]
 
 _c_void_p, _c_int, _c_size_t, _c_uint = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
 
@@ -73,6 +73,8 @@ def load_library() -> ctypes.CDLL:
     lib.wide_oproj.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_int,
                                _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                _c_void_p, _c_size_t, _c_uint]
+    lib.wide_attn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
+                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_int, ctypes.c_float, _c_void_p, _c_uint]
     lib.wide_unpermute.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                    _c_int, _c_int, _c_int, _c_void_p]
     for name in EXPORTS:
@@ -293,6 +295,21 @@ def wide_oproj(ctx: Context, attn_out: torch.Tensor, w_o: torch.Tensor, group: i
                             _ptr(m.get("token_rank")), _ptr(y), _dtype_code(y), _ptr(ws), ws.numel(), flags)
     _check(rc, "wide_oproj")
     return y
+
+
+def wide_attn(ctx: Context, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, n_q_heads: int, n_kv_heads: int,
+              heads_per_group: int, meta: Dict[str, torch.Tensor], causal: bool = True, scale: float = 0.0,
+              flags: int = 0, o: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [T_q, H_q*d], k/v [T_k, H_kv*d] bf16; meta = wide_reorder outputs of the attention mask."""
+    Tq, Tk = q.shape[0], k.shape[0]
+    head_dim = q.shape[1] // n_q_heads
+    if o is None:
+        o = torch.empty_like(q)
+    rc = ctx.lib.wide_attn(ctx.handle, _stream(), _ptr(q), _ptr(k), _ptr(v), _dtype_code(q), Tq, Tk, n_q_heads,
+                           n_kv_heads, head_dim, heads_per_group, _ptr(meta["perm"]), _ptr(meta["counts"]),
+                           1 if causal else 0, float(scale), _ptr(o), flags)
+    _check(rc, "wide_attn")
+    return o
 
 
 def wide_unpermute(ctx: Context, src_packed: torch.Tensor, meta: Dict[str, torch.Tensor], tokens: int,

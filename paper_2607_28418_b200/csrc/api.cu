@@ -2,6 +2,8 @@
 #include <cstdio>
 #include <new>
 
+#include <math.h>
+
 #include "internal.h"
 
 namespace {
@@ -302,6 +304,24 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
             return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
                                                out_dtype, workspace);
     }
+}
+
+int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const void* v, int dtype, int tokens_q,
+              int tokens_k, int n_q_heads, int n_kv_heads, int head_dim, int heads_per_group,
+              const int32_t* perm, const int32_t* counts, int causal, float scale, void* o, unsigned flags) {
+    (void)flags;
+    if (!ctx || !q || !k || !v || !perm || !counts || !o) return WIDE_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return WIDE_ERR_INVALID_ARG;
+    if (tokens_q < 0 || tokens_k <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || heads_per_group <= 0)
+        return WIDE_ERR_INVALID_ARG;
+    if (n_q_heads % n_kv_heads != 0 || n_q_heads % heads_per_group != 0) return WIDE_ERR_INVALID_ARG;
+    if (dtype != WIDE_BF16 || (head_dim != 64 && head_dim != 128) || !ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (n_q_heads / heads_per_group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(q) || !wide_aligned16(k) || !wide_aligned16(v) || !wide_aligned16(o)) return WIDE_ERR_ALIGNMENT;
+    if (tokens_q == 0) return WIDE_OK;
+    if (!(scale > 0.f)) scale = 1.0f / sqrtf(static_cast<float>(head_dim));
+    return wide_launch_attn_prefill_tc(ctx, static_cast<cudaStream_t>(stream), q, k, v, tokens_q, tokens_k, n_q_heads,
+                                       n_kv_heads, head_dim, heads_per_group, perm, counts, causal ? 1 : 0, scale, o);
 }
 
 int wide_unpermute(wide_ctx* ctx, void* stream, const void* src_packed, const int32_t* perm,

@@ -1,6 +1,7 @@
 // Internal declarations shared by the .cu files of libwide (not part of the public ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stddef.h>
@@ -114,3 +115,12 @@ int wide_launch_ffn_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* x, cons
 int wide_launch_oproj_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                 int D, int K, int G, const uint32_t* mask_bits, void* y,
                                 int out_dtype, void* ws);
+
+// 2-D bf16 row-major [rows, cols] tensor map, box = [box_rows, 64 columns], 128-byte swizzle.
+bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
+                         uint32_t box_rows);
+
+// tcgen05 masked attention prefill (bf16, head_dim 64 or 128).
+int wide_launch_attn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, const void* v, int Tq,
+                                int Tk, int Hq, int Hkv, int head_dim, int hpg, const int32_t* perm,
+                                const int32_t* counts, int causal, float scale, void* o);

@@ -933,6 +933,11 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
 
 }  // namespace
 
+bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
+                         uint32_t box_rows) {
+    return make_tmap_bf16(ctx, map, base, rows, cols, box_rows);
+}
+
 int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
                                const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
                                const int32_t* perm, const int32_t* counts, const int32_t* token_order,

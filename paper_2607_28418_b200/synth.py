@@ -178,6 +178,18 @@ def make_oproj_case(cfg: WideConfig, seed: int, tokens: Optional[int] = None) ->
     }
 
 
+def make_attn_case(seed: int, tokens_q: int, tokens_k: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                   dtype: str = "bf16") -> Dict[str, np.ndarray]:
+    """Host buffers for head-group-masked attention: q [T_q, H_q, d], k, v [T_k, H_kv, d] ~ N(0, 1)
+    (the scale of normalised, RoPE-rotated projections), drawn independently."""
+    rng = np.random.default_rng(seed + 611953)
+    return {
+        "q": make_activations(rng, tokens_q * n_q_heads, head_dim, dtype, "random").reshape(tokens_q, n_q_heads, head_dim),
+        "k": make_activations(rng, tokens_k * n_kv_heads, head_dim, dtype, "random").reshape(tokens_k, n_kv_heads, head_dim),
+        "v": make_activations(rng, tokens_k * n_kv_heads, head_dim, dtype, "random").reshape(tokens_k, n_kv_heads, head_dim),
+    }
+
+
 def make_pair_router(cfg: WideConfig, seed: int, rank: int = 16) -> Dict[str, np.ndarray]:
     """Bottleneck router weights W1 [D, r], W2 [r, 2*N_G] (Section 3.1, routing components)."""
     rng = np.random.default_rng(seed + 104729)

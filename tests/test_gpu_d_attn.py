@@ -1,0 +1,84 @@
+"""Parity of wide_attn (masked FlashAttention prefill, Algorithm 4) with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import wide_oracle as wo
+from paper_2607_28418_b200 import synth
+from tests.gpu_util import assert_close, bits_to_dev, meta_to_dev, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2607_28418_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.status() == 0
+    c.close()
+
+
+def _run(ctx, case, mask, h_q, h_kv, d, hpg, causal=True, scale=0.0):
+    from paper_2607_28418_b200 import binding
+    t_q, t_k = case["q"].shape[0], case["k"].shape[0]
+    meta = meta_to_dev(wo.reorder(mask, 128))     # stage-wise: the oracle's permutation goes in
+    o = binding.wide_attn(ctx, to_dev(case["q"].reshape(t_q, h_q * d), "bf16"), to_dev(case["k"].reshape(t_k, h_kv * d), "bf16"),
+                          to_dev(case["v"].reshape(t_k, h_kv * d), "bf16"), h_q, h_kv, hpg, meta, causal=causal, scale=scale)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    return o.reshape(t_q, h_q, d)
+
+
+@pytest.mark.parametrize("t_q,t_k,h_q,h_kv,d,hpg,p", [
+    (128, 128, 4, 4, 128, 2, 0.5),
+    (300, 300, 8, 2, 128, 4, 0.5),       # GQA, ragged last tile
+    (517, 517, 4, 4, 64, 1, 0.3),        # head_dim 64
+    (200, 455, 4, 2, 128, 2, 0.7),       # keys ahead of the queries (delta > 0)
+    (1024, 1024, 8, 8, 128, 4, 0.5),     # several key tiles per query tile
+])
+@pytest.mark.parametrize("causal", [True, False])
+def test_attn_matches_oracle(ctx, t_q, t_k, h_q, h_kv, d, hpg, p, causal):
+    case = synth.make_attn_case(3, t_q, t_k, h_q, h_kv, d)
+    mask = synth.bernoulli_mask(5, t_q, h_q // hpg, p)
+    got = _run(ctx, case, mask, h_q, h_kv, d, hpg, causal=causal)
+    ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg, causal=causal)
+    head_mask = np.repeat(mask, hpg, axis=1)
+    assert (got.float().cpu().numpy()[~head_mask] == 0.0).all()   # inactive pairs: exact zeros
+    assert_close(got, ref, "attn")
+
+
+def test_attn_closed_cases(ctx):
+    t, h_q, h_kv, d, hpg = 260, 4, 2, 128, 2
+    case = synth.make_attn_case(9, t, t, h_q, h_kv, d)
+    ones = np.ones((t, h_q // hpg), dtype=bool)
+    zeros = np.zeros_like(ones)
+    assert (_run(ctx, case, zeros, h_q, h_kv, d, hpg) == 0.0).all().item()
+    # the same value vector at every key: every active output row is that vector
+    case["v"][:] = synth.round_to_bf16(np.linspace(-1, 1, d).astype(np.float32))
+    got = _run(ctx, case, ones, h_q, h_kv, d, hpg).float().cpu().numpy()
+    np.testing.assert_allclose(got, np.broadcast_to(case["v"][0, 0], got.shape), atol=1e-2)
+    # the first token attends to itself only
+    case = synth.make_attn_case(10, t, t, h_q, h_kv, d)
+    got = _run(ctx, case, ones, h_q, h_kv, d, hpg).float().cpu().numpy()
+    np.testing.assert_allclose(got[0], np.repeat(case["v"][0], h_q // h_kv, axis=0), atol=1e-2)
+
+
+def test_attn_one_group_active_per_token_and_custom_scale(ctx):
+    t, h_q, h_kv, d, hpg = 384, 8, 4, 128, 2
+    case = synth.make_attn_case(11, t, t, h_q, h_kv, d)
+    mask = synth.random_mask(12, t, h_q // hpg, 1)
+    got = _run(ctx, case, mask, h_q, h_kv, d, hpg, scale=0.05)
+    ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg, scale=0.05)
+    assert_close(got, ref, "attn, custom scale")
+
+
+def test_attn_rejects_bad_arguments(ctx):
+    from paper_2607_28418_b200 import binding
+    q = torch.zeros((128, 4 * 96), dtype=torch.bfloat16, device="cuda")
+    meta = meta_to_dev(wo.reorder(np.ones((128, 2), dtype=bool), 128))
+    with pytest.raises(binding.WideError):
+        binding.wide_attn(ctx, q, q, q, 4, 4, 2, meta)             # head_dim 96
+    q = torch.zeros((128, 4 * 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.WideError):
+        binding.wide_attn(ctx, q, q, q, 4, 3, 2, meta)             # heads not divisible
