@@ -484,6 +484,193 @@ def run_ours(args):
     return line
 
 
+# ------------------------------------------------------------------------------- attention op
+def run_attn(args):
+    """--op attn: route (attention router) -> reorder -> head-group-masked causal attention on the
+    attention half of the workload (one sequence of `tokens` positions, MHA heads of 128)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_28418_b200 import binding
+    to_dev = binding.upload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    cfg = make_config(args)
+    if not cfg.attn_group:
+        raise SystemExit(f"workload {cfg.name} has no attention half")
+    peaks = load_peaks()
+    ctx = binding.Context(local)
+    T, hd = cfg.tokens, 128
+    H = cfg.attn_dim // hd
+    hpg = cfg.attn_group // hd
+    NG, k = cfg.attn_n_groups, cfg.attn_k
+    oc = synth.make_oproj_case(cfg, 1000 * rank)
+    ac = synth.make_attn_case(1000 * rank, T, T, H, H, hd)
+    host = {"x": oc["x"], "q": ac["q"].reshape(T, H * hd), "k": ac["k"].reshape(T, H * hd), "v": ac["v"].reshape(T, H * hd)}
+    w_router = to_dev(oc["w_router_attn"], "bf16")
+    pinned = {n: torch.from_numpy(synth.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).pin_memory() for n, a in host.items()}
+    bufs = [{n: t.to(dev) for n, t in pinned.items()} for _ in range(2)]
+    obuf = [torch.empty((T, H * hd), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    o_host = [torch.empty((T, H * hd), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    bits = torch.empty((T, (NG + 31) // 32), dtype=torch.int32, device=dev)
+    state = {"meta": None}
+
+    def attn_only(slot=0):
+        b = bufs[slot]
+        binding.wide_attn(ctx, b["q"], b["k"], b["v"], H, H, hpg, state["meta"], causal=True, o=obuf[slot])
+
+    def step(slot=0, kk=k):
+        binding.wide_route(ctx, bufs[slot]["x"], w_router, NG, kk, mask_bits=bits)
+        state["meta"] = binding.wide_reorder(ctx, bits, NG, 128, out=state["meta"])
+        attn_only(slot)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync_all()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        sync_all()
+        return reduce_max_ms(e0.elapsed_time(e1), world, dev)
+
+    def graphed(fn):
+        if args.no_graph:
+            return fn
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g.replay
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during warm-up")
+    run_step = graphed(step)
+    run_step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_total = timed(run_step, args.steps)
+    value = aggregate(T, args.steps, ms_total, world)
+    run_attn_only = graphed(attn_only)
+    run_attn_only()
+    attn_ms = timed(run_attn_only, args.steps) / args.steps
+
+    launches0 = ctx.launch_count()
+    ctx.profile_begin(16 * args.steps + 16)
+    for _ in range(args.steps):
+        step()
+    prof = ctx.profile_end()
+    launches = ctx.launch_count() - launches0
+
+    # end to end: x, q, k, v from pinned host memory every step, o back to the host
+    s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev = {n: [torch.cuda.Event(), torch.cuda.Event()] for n in ("in", "run", "out")}
+
+    def e2e_loop(steps):
+        cur = torch.cuda.current_stream()
+        for st in (s_in, s_run, s_out):
+            st.wait_stream(cur)
+        for i in range(steps):
+            b = i % 2
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev["run"][b])
+                for n in pinned:
+                    bufs[b][n].copy_(pinned[n], non_blocking=True)
+                ev["in"][b].record()
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev["in"][b])
+                if i >= 2:
+                    s_run.wait_event(ev["out"][b])
+                step(slot=b)
+                ev["run"][b].record()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev["run"][b])
+                o_host[b].copy_(obuf[b], non_blocking=True)
+                ev["out"][b].record()
+        for st in (s_in, s_run, s_out):
+            cur.wait_stream(st)
+
+    e2e_loop(2)
+    e2e_steps = max(4, min(args.steps, 20))
+    ms_e2e = timed(lambda: e2e_loop(e2e_steps), 1)
+    clocks = sampler.stop() if rank == 0 else None
+
+    dense_ms = None
+    if not args.no_dense:
+        for _ in range(2):
+            step(kk=NG)
+        run_dense = graphed(lambda: step(kk=NG))
+        run_dense()
+        dense_ms = timed(run_dense, max(3, min(args.steps, 10))) / max(3, min(args.steps, 10))
+        step()
+
+    line = None
+    if rank == 0:
+        # algorithmic FLOPs: every active (token t, head) pair does 4 * d * (t + 1) (QK^T and PV over its keys)
+        mask = np.unpackbits(bits.cpu().numpy().view(np.uint8), axis=1, bitorder="little")[:, :NG].astype(bool)
+        flops = float((mask.sum(axis=1) * hpg * 4.0 * hd * (np.arange(T) + 1.0)).sum())
+        ach = flops / (attn_ms * 1e-3) / 1e12
+        kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
+                       "share": round(v["total_ms"] / max(sum(p["total_ms"] for p in prof.values()), 1e-9), 4)}
+                   for n, v in prof.items()}
+        line = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "op": "attn", "tokens_per_gpu": T, "heads": H, "head_dim": hd,
+                       "heads_per_group": hpg, "n_groups": NG, "k": k, "causal": True, "router": cfg.router,
+                       "parallelism": f"sequence-sharded x{world} (independent sequences), no collective",
+                       "l2": "q, k, v, o of one step are %.0f MB (larger than L2)" % (4 * T * H * hd * 2 / 1e6)},
+            "e2e": {"value": aggregate(T, e2e_steps, ms_e2e, world), "unit": "tokens/s",
+                    "h2d_bytes_per_step": sum(t.numel() * 2 for t in pinned.values()),
+                    "d2h_bytes_per_step": o_host[0].numel() * 2},
+            "launch": "one CUDA graph replay per step" if not args.no_graph else "direct launches",
+            "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": {"kernel": "attn_prefill", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                         "traffic": NCU_TRAFFIC_BYTES.get(("attn_prefill", cfg.name)), "peak_source": peaks["source"]},
+            "kernels": kernels,
+            "attn": {"graph_ms": attn_ms, "active_gflop": flops / 1e9},
+            "dense": {"ms_per_step": dense_ms, "speedup_vs_dense": (dense_ms / (ms_total / args.steps)) if dense_ms else None,
+                      "ideal": NG / k if k else None},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            sample = min(T, 1024)
+            t0 = time.perf_counter()
+            m_s = mask[:sample]
+            from oracle import wide_oracle as wo
+            wo.masked_attention(ac["q"][:sample], ac["k"][:sample], ac["v"][:sample], m_s, hpg)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": sample / dt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"first {sample} of {T} positions, masked attention only, fp64 numpy ({dt:.1f} s)"}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return line
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -495,7 +682,8 @@ def main():
     ap.add_argument("--router", default="", choices=["", "random", "clustered", "clustered_corr"])
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--group", type=int, default=0)
-    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj"], help="oproj needs a workload with an attention half")
+    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn"],
+                    help="oproj and attn need a workload with an attention half")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")
@@ -504,6 +692,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.op == "attn":
+        run_attn(args)
     else:
         run_ours(args)
 

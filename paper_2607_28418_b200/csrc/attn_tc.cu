@@ -9,15 +9,21 @@
 //     S  = Q K_t^T                (UMMA, fp32 in TMEM, two buffers)
 //     P  = exp2(S*c - m), row statistics m, l   (softmax warps: one thread per row, S read twice from
 //                                  TMEM so that a row never has to live in registers)
-//     PV = P V_t                  (UMMA; P goes through shared memory as a bf16 K-major operand,
-//                                  V_t is used as loaded, as an MN-major operand; two TMEM buffers)
-//     O  = O * alpha + PV         (softmax warps, O in registers)
+//     O += P V_t                  (UMMA accumulating in TMEM; P goes through shared memory as a bf16
+//                                  K-major operand, V_t is used as loaded, as an MN-major operand)
+// O stays in TMEM for the whole key loop.  A row's reference maximum m is only raised when the
+// running maximum has grown by more than 2^8 since it was set (P then stays below 2^8, harmless in
+// bf16 / fp32); raising it rescales that warp's rows of O in TMEM (load, multiply, store), which
+// after the first tiles is rare, so the softmax warps carry no accumulator registers at all.
 // The UMMA warp issues S of tile t+1 before PV of tile t, so the tensor core works on the next
-// scores while the softmax warps are busy.  Causal attention shortens the key range to the largest
+// scores while the softmax warps are busy.  The softmax is the slower side (one exponential per
+// score), so two groups of four warps share the rows: group 0 takes the even key tiles, group 1
+// the odd ones, each with its own (m, l, O) per row and its own S / P / O buffers; the two
+// partial results are merged once at the end (the split-key form of the online softmax).  Causal attention shortens the key range to the largest
 // active query position of the tile (+ delta = T_k - T_q); only tiles that straddle a row's limit
 // evaluate element-wise predicates.
 //
-// Outputs of inactive (token, group) pairs are zeroed by a few extra CTAs of the same grid.
+// Outputs of inactive (token, group) pairs are zeroed by a small kernel of its own.
 // Every mbarrier wait is bounded.
 #include <cuda.h>
 #include <math_constants.h>
@@ -33,7 +39,7 @@ constexpr int kQ = 128;        // query rows per tile (UMMA M)
 constexpr int kKV = 128;       // keys per tile
 constexpr int kBK = 64;        // bf16 elements per 128-byte swizzle row
 constexpr int kBlk = 16384;    // bytes of one [128 rows x 64 elements] swizzled block
-constexpr int kThreads = 192;  // TMA warp, UMMA warp, 4 softmax warps
+constexpr int kThreads = 320;  // TMA warp, UMMA warp, 2 groups of 4 softmax warps
 
 // Shared-memory descriptor of an MN-major operand in the 128-byte swizzle: the tile is stored as
 // loaded by TMA, rows = K index (128 bytes = 64 elements of the MN dimension each).  Blocks of 64
@@ -70,36 +76,35 @@ constexpr int attn_smem_bytes() {
     return (HD / kBK) * kBlk + 4 * (HD / kBK) * kBlk + 2 * (kKV / kBK) * kBlk + 256 + 1024;
 }
 
+// o[row, heads of g, :] = 0 for every inactive (row, g) pair: sorted positions [counts[g], T_q).
+__global__ void __launch_bounds__(256)
+attn_zero_kernel(const int32_t* __restrict__ perm, const int32_t* __restrict__ counts, int Tq, int NG, int ppr,
+                 size_t ldq, __nv_bfloat16* __restrict__ o) {
+    // ppr = 16-byte pieces per (row, group); blockIdx.y = group
+    const int g = blockIdx.y;
+    const int c = counts[g];
+    const long long total = static_cast<long long>(Tq - c) * ppr;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int j = c + static_cast<int>(i / ppr), piece = static_cast<int>(i % ppr);
+        const int row = perm[static_cast<size_t>(g) * Tq + j];
+        reinterpret_cast<uint4*>(o + row * ldq + static_cast<size_t>(g) * ppr * 8)[piece] = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
 // q [T_q, H_q*HD], o likewise; K/V come through the tensor maps ([T_k, H_kv*HD], box 64 x 128).
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
             const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ perm, const int32_t* __restrict__ counts,
-            int Tq, int Tk, int Hq, int Hkv, int hpg, int causal, float scale_log2e, int n_main,
+            int Tq, int Tk, int Hq, int Hkv, int hpg, int causal, float scale_log2e,
             __nv_bfloat16* __restrict__ o, int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kKB = HD / kBK;          // 64-wide blocks along the head dimension
     constexpr int kQBytes = kKB * kBlk;
     constexpr int kKVBytes = kKB * kBlk;   // one K (or V) tile
     constexpr int kPBytes = (kKV / kBK) * kBlk;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int NG = Hq / hpg;
     const size_t ldq = static_cast<size_t>(Hq) * HD;
-
-    if (static_cast<int>(blockIdx.x) >= n_main) {
-        // ------------------------------------------------ zero the outputs of inactive pairs
-        const int nz = gridDim.x - n_main, zi = blockIdx.x - n_main;
-        const int ppr = hpg * HD / 8;  // 16-byte pieces per (row, group)
-        for (int g = 0; g < NG; ++g) {
-            const int c = counts[g];
-            const long long total = static_cast<long long>(Tq - c) * ppr;
-            for (long long i = static_cast<long long>(zi) * kThreads + tid; i < total; i += static_cast<long long>(nz) * kThreads) {
-                const int j = c + static_cast<int>(i / ppr), piece = static_cast<int>(i % ppr);
-                const int row = perm[static_cast<size_t>(g) * Tq + j];
-                reinterpret_cast<uint4*>(o + row * ldq + static_cast<size_t>(g) * hpg * HD)[piece] = make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
-        return;
-    }
 
     // heavy (late, long key range) tiles first
     const int n_mt = (Tq + kQ - 1) / kQ;
@@ -141,9 +146,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             mbar_init(s_free + 8 * i, 128);
             mbar_init(p_ready + 8 * i, 128);
             mbar_init(pv_full + 8 * i, 1);
-            mbar_init(pv_free + 8 * i, 128);
         }
-        mbar_init(q_ready, 128);
+        mbar_init(q_ready, 256);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmK);
@@ -209,14 +213,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
                 const uint32_t ph = (t >> 1) & 1;
                 if (!mbar_wait(v_full + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(p_ready + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(pv_free + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
                 fence_proxy_async_smem();
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k16 = 0; k16 < kKV / 16; ++k16) {
                     const uint64_t adesc = umma_desc_sw128(smem_u32(p_s + s * kPBytes + (k16 / 4) * kBlk)) + 2 * (k16 % 4);
                     const uint64_t bdesc = umma_desc_sw128_mn(smem_u32(v_s + s * kKVBytes + k16 * 2048), kBlk);
-                    umma_bf16(tmem_base + 256 + s * HD, adesc, bdesc, idesc_pv, k16 > 0 ? 1u : 0u);
+                    umma_bf16(tmem_base + 256 + s * HD, adesc, bdesc, idesc_pv, (t >= 2 || k16 > 0) ? 1u : 0u);
                 }
                 umma_commit(v_empty + 8 * s);
                 umma_commit(pv_full + 8 * s);
@@ -224,8 +227,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             if (!ok) atomicExch(status, WIDE_ERR_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------------------------ softmax warps (2..5)
-        const int st = tid - 64;                     // 0..127
+        // ------------------------------------------------------------------ softmax warps (2..9)
+        const int st = tid - 64;                     // 0..255
+        const int grp = (warp - 2) >> 2;             // 0: even key tiles, 1: odd key tiles
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
         const int r = quarter * 32 + lane;           // row of the tile owned by this thread
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -235,8 +239,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
         if (NT > 0) {
             const int chunk = st & 7;
 #pragma unroll
-            for (int i = 0; i < kQ / 16; ++i) {
-                const int row = (st >> 3) + 16 * i;
+            for (int i = 0; i < kQ / 32; ++i) {
+                const int row = (st >> 3) + 32 * i;
                 const int src_row = rows[min(row, n_valid - 1)];
                 const uint8_t* src = reinterpret_cast<const uint8_t*>(q + src_row * ldq + static_cast<size_t>(h) * HD) + 16 * chunk;
 #pragma unroll
@@ -250,100 +254,138 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
 
         const int pos = rows[min(r, n_valid - 1)];
         const int lim = causal ? min(pos + delta, Tk - 1) : Tk - 1;   // last visible key of this row
-        float mrow = -CUDART_INF_F, lrow = 0.f, alpha_pending = 1.f;
-        float acc[HD];
-#pragma unroll
-        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
+        float mref = -CUDART_INF_F, lrow = 0.f;      // reference maximum (log2 units, scaled), row sum
+        const int b = grp;                           // this group's S / P / O buffer
+        const uint32_t o_addr = lane_addr + 256 + b * HD;
+        constexpr float kRaise = 8.f;                // raise the reference only for a growth above 2^8
 
-        auto accumulate = [&](int u, float alpha) -> bool {
-            const int b = u & 1;
-            const uint32_t ph = (u >> 1) & 1;
-            if (!mbar_wait(pv_full + 8 * b, ph, wait_ns, abort_flag)) return false;
-            tc_fence_after_sync();
-#pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(lane_addr + 256 + b * HD + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) acc[c0 + i] = fmaf(acc[c0 + i], alpha, __uint_as_float(v[i]));
-            }
-            tc_fence_before_sync();
-            mbar_arrive(pv_free + 8 * b);
-            return true;
-        };
-
-        for (int t = 0; t < NT; ++t) {
-            const int b = t & 1;
+        int last = -1;
+        for (int t = grp; t < NT; t += 2) {
             const uint32_t ph = (t >> 1) & 1;
             if (!mbar_wait(s_full + 8 * b, ph, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const int j0 = t * kKV;
             const bool edge = j0 + kKV - 1 > lim;     // this row needs element-wise predicates here
-            // pass 1: row maximum
-            float mx = -CUDART_INF_F;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kKV; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(lane_addr + b * kKV + c0, v);
-                tmem_ld_wait();
+            // The whole score row comes into registers with one TMEM round trip (the latency of a
+            // tcgen05.ld is what a chunked loop would pay per chunk), and S is handed back to the
+            // UMMA warp before any arithmetic: the next scores of this group are computed meanwhile.
+            uint32_t v[kKV];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float sv = __uint_as_float(v[i]) * scale_log2e;
-                    mx = fmaxf(mx, (!edge || j0 + c0 + i <= lim) ? sv : -CUDART_INF_F);
-                }
-            }
-            const float m_new = fmaxf(mrow, mx);
-            const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;   // a row that has seen no key yet
-            const float alpha = fast_exp2(mrow - m_use);
-            // pass 2: P = exp2(S*c - m) as bf16 into the operand layout, row sum
-            float rs = 0.f;
-            uint8_t* prow = p_s + b * kPBytes + r * 128;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kKV; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(lane_addr + b * kKV + c0, v);
-                tmem_ld_wait();
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale_log2e, -m_use));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale_log2e, -m_use));
-                    if (edge) {
-                        if (j0 + c0 + i > lim) p0 = 0.f;
-                        if (j0 + c0 + i + 1 > lim) p1 = 0.f;
-                    }
-                    rs += p0 + p1;
-                    pk[i >> 1] = pack2(p0, p1);
-                }
-                uint8_t* blk = prow + (c0 / kBK) * kBlk;
-                const int ch0 = (c0 % kBK) / 8;
-#pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4)
-                    *reinterpret_cast<uint4*>(blk + (((ch0 + v4) ^ (r & 7)) << 4)) =
-                        make_uint4(pk[4 * v4], pk[4 * v4 + 1], pk[4 * v4 + 2], pk[4 * v4 + 3]);
-            }
-            lrow = fmaf(lrow, alpha, rs);
-            mrow = m_new;
+            for (int c0 = 0; c0 < kKV; c0 += 32) tmem_ld_32x32(lane_addr + b * kKV + c0, reinterpret_cast<uint32_t(&)[32]>(v[c0]));
+            tmem_ld_wait();
             tc_fence_before_sync();
             mbar_arrive(s_free + 8 * b);
+            // row maximum of the raw scores (the scale is positive)
+            float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+            if (!edge) {
+#pragma unroll
+                for (int i = 0; i < kKV; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(v[i]));
+            } else {
+#pragma unroll
+                for (int i = 0; i < kKV; ++i) {
+                    if (j0 + i > lim) v[i] = 0xff800000u;   // -inf: exp2 gives an exact zero below
+                    mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(v[i]));
+                }
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2e;
+            // the previous PV of this group has to be complete before P is overwritten or O rescaled
+            if (last >= 0 && !mbar_wait(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
+            float alpha = 1.f;
+            const bool raise = mx > mref + kRaise || (mref == -CUDART_INF_F && mx > mref);
+            if (raise) {
+                alpha = fast_exp2(mref - mx);        // 0 when this is the first key the row sees
+                mref = mx;
+            }
+            if (last >= 0 && __any_sync(0xffffffffu, raise)) {
+                tc_fence_after_sync();
+#pragma unroll 1
+                for (int c0 = 0; c0 < HD; c0 += 16) {
+                    uint32_t w[16];
+                    tmem_ld_32x16(o_addr + c0, w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+                    tmem_st_32x16(o_addr + c0, w);
+                }
+                tmem_st_wait();
+            }
+            const float m_use = mref == -CUDART_INF_F ? 0.f : mref;     // a row that has seen no key yet
+            // P = exp2(S*c - m) as bf16 into the operand layout, row sum
+            float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+            uint8_t* prow = p_s + b * kPBytes + r * 128;
+#pragma unroll
+            for (int c0 = 0; c0 < kKV; c0 += 8) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(v[c0 + i]), scale_log2e, -m_use));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(v[c0 + i + 1]), scale_log2e, -m_use));
+                    rs4[(i >> 1) & 3] += p0 + p1;
+                    pk[i >> 1] = pack2(p0, p1);
+                }
+                *reinterpret_cast<uint4*>(prow + (c0 / kBK) * kBlk + ((((c0 % kBK) / 8) ^ (r & 7)) << 4)) =
+                    make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            lrow = fmaf(lrow, alpha, (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
+            tc_fence_before_sync();
             fence_proxy_async_smem();
             mbar_arrive(p_ready + 8 * b);
-            // O of the previous tile while the tensor core works on this one
-            if (t > 0 && !accumulate(t - 1, alpha_pending)) { ok = false; break; }
-            alpha_pending = alpha;
+            last = t;
         }
-        if (ok && NT > 0) ok = accumulate(NT - 1, alpha_pending);
+        if (ok && last >= 0) ok = mbar_wait(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag);
+        tc_fence_after_sync();
         if (NT > 0) cp_async_wait_all();
+        const float mrow = mref;
 
-        // epilogue: normalise and scatter the active rows
-        if (ok && r < n_valid) {
-            const float inv = lrow > 0.f ? 1.f / lrow : 0.f;
-            uint4* dst = reinterpret_cast<uint4*>(o + pos * ldq + static_cast<size_t>(h) * HD);
+        // Merge the two groups' partial results.  By now every S = Q K^T has completed (the PV of a
+        // tile is issued after the S of the next one and UMMAs complete in order), so the K stages
+        // are free: group 1 parks (m, l, O) there, column-major so that a warp writes 128 bytes.
+        float* xo = reinterpret_cast<float*>(k_s);                  // [HD][128]
+        float* xml = reinterpret_cast<float*>(q_s);                 // [2][128]
+        const bool two = NT > 1;   // with a single key tile group 1 has nothing (and S may still be running)
+        if (grp == 1 && two) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(o_addr + c0, v);
+                tmem_ld_wait();
 #pragma unroll
-            for (int v8 = 0; v8 < HD / 8; ++v8)
-                dst[v8] = make_uint4(pack2(acc[8 * v8] * inv, acc[8 * v8 + 1] * inv), pack2(acc[8 * v8 + 2] * inv, acc[8 * v8 + 3] * inv),
-                                     pack2(acc[8 * v8 + 4] * inv, acc[8 * v8 + 5] * inv), pack2(acc[8 * v8 + 6] * inv, acc[8 * v8 + 7] * inv));
+                for (int i = 0; i < 32; ++i) xo[(c0 + i) * kQ + r] = __uint_as_float(v[i]);
+            }
+            xml[r] = mrow;
+            xml[kQ + r] = lrow;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (grp == 0) {
+            const float m1 = two ? xml[r] : -CUDART_INF_F, l1 = two ? xml[kQ + r] : 0.f;
+            const float m_all = fmaxf(mrow, m1);
+            const float m_use = m_all == -CUDART_INF_F ? 0.f : m_all;
+            const float a0 = fast_exp2(mrow - m_use), a1 = fast_exp2(m1 - m_use);
+            const float l_all = lrow * a0 + l1 * a1;
+            const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+            // epilogue: normalise and scatter the active rows (O of group 0 comes straight from TMEM)
+            uint4* dst = reinterpret_cast<uint4*>(o + pos * ldq + static_cast<size_t>(h) * HD);
+#pragma unroll 1
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+                uint32_t v[32];
+                if (last >= 0) {
+                    tmem_ld_32x32(o_addr + c0, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0u;
+                }
+                if (ok && r < n_valid) {
+#pragma unroll
+                    for (int v8 = 0; v8 < 4; ++v8) {
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            f[e] = (__uint_as_float(v[8 * v8 + e]) * a0 + (two ? xo[(c0 + 8 * v8 + e) * kQ + r] : 0.f) * a1) * inv;
+                        dst[c0 / 8 + v8] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+                    }
+                }
+            }
         }
         if (!ok && lane == 0) atomicExch(status, WIDE_ERR_TIMEOUT);
     }
@@ -366,11 +408,16 @@ int launch_attn(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, con
     constexpr int smem = attn_smem_bytes<HD>();
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(attn_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int n_main = ((Tq + kQ - 1) / kQ) * Hq;
-    const int n_zero = ctx->sm_count / 4 > 0 ? ctx->sm_count / 4 : 1;
+    const int NG = Hq / hpg, ppr = hpg * HD / 8;
+    {
+        WideLaunch l(ctx, s, "attn_zero");
+        attn_zero_kernel<<<dim3(32, NG), 256, 0, s>>>(perm, counts, Tq, NG, ppr, static_cast<size_t>(Hq) * HD,
+                                                      static_cast<__nv_bfloat16*>(o));
+    }
     WideLaunch l(ctx, s, "attn_prefill");
-    attn_kernel<HD><<<n_main + n_zero, kThreads, smem, s>>>(
+    attn_kernel<HD><<<n_main, kThreads, smem, s>>>(
         tmK, tmV, static_cast<const __nv_bfloat16*>(q), perm, counts, Tq, Tk, Hq, Hkv, hpg, causal,
-        scale * 1.4426950408889634f, n_main, static_cast<__nv_bfloat16*>(o), ctx->d_status, ctx->wait_ns);
+        scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(o), ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
