@@ -15,8 +15,10 @@
 // running maximum has grown by more than 2^8 since it was set (P then stays below 2^8, harmless in
 // bf16 / fp32); raising it rescales that warp's rows of O in TMEM (load, multiply, store), which
 // after the first tiles is rare, so the softmax warps carry no accumulator registers at all.
-// The UMMA warp issues S of tile t+1 before PV of tile t, so the tensor core works on the next
-// scores while the softmax warps are busy.  The softmax is the slower side (one exponential per
+// A softmax group hands its S buffer back as soon as the row is in registers, and the UMMA warp
+// then issues the group's next scores (tile t+2) BEFORE the PV of tile t, so a group never waits
+// for its scores and the tensor core works while the softmax warps are busy.  K and V have a
+// producer warp each: their rings drain at different points of the loop.  The softmax is the slower side (one exponential per
 // score), so two groups of four warps share the rows: group 0 takes the even key tiles, group 1
 // the odd ones, each with its own (m, l, O) per row and its own S / P / O buffers; the two
 // partial results are merged once at the end (the split-key form of the online softmax).  Causal attention shortens the key range to the largest
@@ -39,7 +41,7 @@ constexpr int kQ = 128;        // query rows per tile (UMMA M)
 constexpr int kKV = 128;       // keys per tile
 constexpr int kBK = 64;        // bf16 elements per 128-byte swizzle row
 constexpr int kBlk = 16384;    // bytes of one [128 rows x 64 elements] swizzled block
-constexpr int kThreads = 320;  // TMA warp, UMMA warp, 2 groups of 4 softmax warps
+constexpr int kThreads = 352;  // K producer, UMMA warp, 2 groups of 4 softmax warps, V producer
 
 // Shared-memory descriptor of an MN-major operand in the 128-byte swizzle: the tile is stored as
 // loaded by TMA, rows = K index (128 bytes = 64 elements of the MN dimension each).  Blocks of 64
@@ -162,21 +164,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (K, V)
+    if (warp == 0 || warp == 10) {
+        // ------------------------------------------------------------------ TMA producers: K (warp 0), V (warp 10)
         if (lane == 0) {
+            const bool is_k = warp == 0;
+            const uint32_t full = is_k ? k_full : v_full, empty = is_k ? k_empty : v_empty;
+            uint8_t* ring = is_k ? k_s : v_s;
+            const CUtensorMap* tm = is_k ? &tmK : &tmV;
             bool ok = true;
-            for (int t = 0; t < NT && ok; ++t) {
+            for (int t = 0; t < NT; ++t) {
                 const int s = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
-                if (!mbar_wait(k_empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
-                mbar_arrive_expect_tx(k_full + 8 * s, kKVBytes);
+                if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
+                mbar_arrive_expect_tx(full + 8 * s, kKVBytes);
                 for (int kb = 0; kb < kKB; ++kb)
-                    tma_load_2d(smem_u32(k_s + s * kKVBytes + kb * kBlk), &tmK, hkv * HD + kb * kBK, t * kKV, k_full + 8 * s);
-                if (!mbar_wait(v_empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
-                mbar_arrive_expect_tx(v_full + 8 * s, kKVBytes);
-                for (int kb = 0; kb < kKB; ++kb)
-                    tma_load_2d(smem_u32(v_s + s * kKVBytes + kb * kBlk), &tmV, hkv * HD + kb * kBK, t * kKV, v_full + 8 * s);
+                    tma_load_2d(smem_u32(ring + s * kKVBytes + kb * kBlk), tm, hkv * HD + kb * kBK, t * kKV, full + 8 * s);
             }
             if (!ok) {
                 atomicExch(status, WIDE_ERR_TIMEOUT);
@@ -194,7 +196,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
                 const int s = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
                 if (!mbar_wait(k_full + 8 * s, ph, wait_ns, abort_flag)) return false;
-                if (!mbar_wait(s_free + 8 * s, ph ^ 1u, wait_ns, abort_flag)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k16 = 0; k16 < HD / 16; ++k16) {
@@ -207,10 +208,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
                 return true;
             };
             if (ok && NT > 0) ok = issue_qk(0);
+            if (ok && NT > 1) ok = issue_qk(1);
             for (int t = 0; t < NT && ok; ++t) {
-                if (t + 1 < NT && !issue_qk(t + 1)) { ok = false; break; }
                 const int s = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
+                // the group of tile t has its scores in registers: its next scores can be computed now
+                if (t + 2 < NT) {
+                    if (!mbar_wait(s_free + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
+                    if (!issue_qk(t + 2)) { ok = false; break; }
+                }
                 if (!mbar_wait(v_full + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(p_ready + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
                 fence_proxy_async_smem();
