@@ -17,8 +17,10 @@
 // after the first tiles is rare, so the softmax warps carry no accumulator registers at all.
 // A softmax group hands its S buffer back as soon as the row is in registers, and the UMMA warp
 // then issues the group's next scores (tile t+2) BEFORE the PV of tile t, so a group never waits
-// for its scores and the tensor core works while the softmax warps are busy.  K and V have a
-// producer warp each: their rings drain at different points of the loop.  The softmax is the slower side (one exponential per
+// for its scores and the tensor core works while the softmax warps are busy.  The two kinds of
+// UMMA have an issuing thread each (a single thread's waits, fences and commits for both took
+// longer per tile than the tensor core needs), and K and V have a producer warp each: their
+// rings drain at different points of the loop.  The softmax is the slower side (one exponential per
 // score), so two groups of four warps share the rows: group 0 takes the even key tiles, group 1
 // the odd ones, each with its own (m, l, O) per row and its own S / P / O buffers; the two
 // partial results are merged once at the end (the split-key form of the online softmax).  Causal attention shortens the key range to the largest
@@ -41,7 +43,7 @@ constexpr int kQ = 128;        // query rows per tile (UMMA M)
 constexpr int kKV = 128;       // keys per tile
 constexpr int kBK = 64;        // bf16 elements per 128-byte swizzle row
 constexpr int kBlk = 16384;    // bytes of one [128 rows x 64 elements] swizzled block
-constexpr int kThreads = 352;  // K producer, UMMA warp, 2 groups of 4 softmax warps, V producer
+constexpr int kThreads = 384;  // K producer, QK issuer, 2 groups of 4 softmax warps, V producer, PV issuer
 
 // Shared-memory descriptor of an MN-major operand in the 128-byte swizzle: the tile is stored as
 // loaded by TMA, rows = K index (128 bytes = 64 elements of the MN dimension each).  Blocks of 64
@@ -186,47 +188,54 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ UMMA issuer
+        // ------------------------------------------------------------------ UMMA issuer: S = Q K^T
         if (lane == 0) {
             constexpr uint32_t idesc_qk = idesc_bf16(kQ, kKV, false);
-            constexpr uint32_t idesc_pv = idesc_bf16(kQ, HD, true);
             bool ok = NT == 0 || mbar_wait(q_ready, 0, wait_ns, abort_flag);
-            fence_proxy_async_smem();  // Q rows and P tiles are written through the generic proxy
+            fence_proxy_async_smem();  // the Q rows were written through the generic proxy (cp.async)
+            uint64_t qdesc[kKB];
+#pragma unroll
+            for (int kb = 0; kb < kKB; ++kb) qdesc[kb] = umma_desc_sw128(smem_u32(q_s + kb * kBlk));
             auto issue_qk = [&](int t) -> bool {
                 const int s = t & 1;
-                const uint32_t ph = (t >> 1) & 1;
-                if (!mbar_wait(k_full + 8 * s, ph, wait_ns, abort_flag)) return false;
+                if (!mbar_wait(k_full + 8 * s, (t >> 1) & 1, wait_ns, abort_flag)) return false;
                 tc_fence_after_sync();
+                const uint64_t kdesc = umma_desc_sw128(smem_u32(k_s + s * kKVBytes));
 #pragma unroll
-                for (int k16 = 0; k16 < HD / 16; ++k16) {
-                    const uint64_t adesc = umma_desc_sw128(smem_u32(q_s + (k16 / 4) * kBlk)) + 2 * (k16 % 4);
-                    const uint64_t bdesc = umma_desc_sw128(smem_u32(k_s + s * kKVBytes + (k16 / 4) * kBlk)) + 2 * (k16 % 4);
-                    umma_bf16(tmem_base + s * kKV, adesc, bdesc, idesc_qk, k16 > 0 ? 1u : 0u);
-                }
+                for (int k16 = 0; k16 < HD / 16; ++k16)
+                    umma_bf16(tmem_base + s * kKV, qdesc[k16 / 4] + 2 * (k16 % 4),
+                              kdesc + (k16 / 4) * (kBlk >> 4) + 2 * (k16 % 4), idesc_qk, k16 > 0 ? 1u : 0u);
                 umma_commit(k_empty + 8 * s);
                 umma_commit(s_full + 8 * s);
                 return true;
             };
             if (ok && NT > 0) ok = issue_qk(0);
             if (ok && NT > 1) ok = issue_qk(1);
-            for (int t = 0; t < NT && ok; ++t) {
+            // the group of tile t has its scores in registers: its next scores can be computed now
+            for (int t = 0; t + 2 < NT && ok; ++t) {
+                if (!mbar_wait(s_free + 8 * (t & 1), (t >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
+                ok = issue_qk(t + 2);
+            }
+            if (!ok) atomicExch(status, WIDE_ERR_TIMEOUT);
+        }
+    } else if (warp == 11) {
+        // ------------------------------------------------------------------ UMMA issuer: O += P V
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = idesc_bf16(kQ, HD, true);
+            bool ok = true;
+            for (int t = 0; t < NT; ++t) {
                 const int s = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
-                // the group of tile t has its scores in registers: its next scores can be computed now
-                if (t + 2 < NT) {
-                    if (!mbar_wait(s_free + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
-                    if (!issue_qk(t + 2)) { ok = false; break; }
-                }
                 if (!mbar_wait(v_full + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(p_ready + 8 * s, ph, wait_ns, abort_flag)) { ok = false; break; }
-                fence_proxy_async_smem();
+                fence_proxy_async_smem();   // P was written through the generic proxy
                 tc_fence_after_sync();
+                const uint64_t pdesc = umma_desc_sw128(smem_u32(p_s + s * kPBytes));
+                const uint64_t vdesc = umma_desc_sw128_mn(smem_u32(v_s + s * kKVBytes), kBlk);
 #pragma unroll
-                for (int k16 = 0; k16 < kKV / 16; ++k16) {
-                    const uint64_t adesc = umma_desc_sw128(smem_u32(p_s + s * kPBytes + (k16 / 4) * kBlk)) + 2 * (k16 % 4);
-                    const uint64_t bdesc = umma_desc_sw128_mn(smem_u32(v_s + s * kKVBytes + k16 * 2048), kBlk);
-                    umma_bf16(tmem_base + 256 + s * HD, adesc, bdesc, idesc_pv, (t >= 2 || k16 > 0) ? 1u : 0u);
-                }
+                for (int k16 = 0; k16 < kKV / 16; ++k16)
+                    umma_bf16(tmem_base + 256 + s * HD, pdesc + (k16 / 4) * (kBlk >> 4) + 2 * (k16 % 4),
+                              vdesc + k16 * (2048 >> 4), idesc_pv, (t >= 2 || k16 > 0) ? 1u : 0u);
                 umma_commit(v_empty + 8 * s);
                 umma_commit(pv_full + 8 * s);
             }
