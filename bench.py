@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
 # (profiles/), keyed by (kernel, workload); None until captured.
 NCU_TRAFFIC_BYTES = {
-    ("prefill_gateup", "llama7b_prefill"): 237.1e6,
+    ("prefill_gateup", "llama7b_prefill"): 355.4e6,
     ("prefill_down", "llama7b_prefill"): 140.1e6,
     # decode: captured at batch 8 (union 111 groups, 357.3 MB); traffic is proportional to the union
     ("decode_ffn_fused", "llama8b_decode"): 357.3e6 / 111,
