@@ -95,6 +95,12 @@ WIDE_API int wide_status(wide_ctx* ctx, void* stream, int* status);
 /* Override the bound of every device-side wait (nanoseconds; default 2e9). */
 WIDE_API int wide_set_wait_limit_ns(wide_ctx* ctx, uint64_t ns);
 
+/* Self-test of the failure path (no counterpart in the paper): one CTA waits, with the context's
+ * wait bound, on an mbarrier that is never completed; when the bound expires it sets the status
+ * word as a hot-path kernel would and returns.  After that wide_status reports WIDE_ERR_TIMEOUT
+ * and the context stays usable.  Nothing faults or hangs.  Errors: INVALID_ARG, CUDA. */
+WIDE_API int wide_selftest_wait(wide_ctx* ctx, void* stream);
+
 /* Per-kernel timing (tracing aid).  wide_profile_begin creates `max_records` CUDA event pairs;
  * until wide_profile_end every kernel the library launches is bracketed by one pair on its
  * stream.  wide_profile_end synchronises `stream` and writes one text line per kernel name,

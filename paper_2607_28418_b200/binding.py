@@ -25,7 +25,7 @@ MAX_GROUPS = 256
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
-           "wide_profile_end", "wide_launch_count", "wide_strerror",
+           "wide_profile_end", "wide_launch_count", "wide_selftest_wait", "wide_strerror",
            "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_ffn",
            "wide_oproj", "wide_attn", "wide_unpermute"]
 
@@ -54,6 +54,7 @@ def load_library() -> ctypes.CDLL:
     lib.wide_destroy.argtypes = [_c_void_p]
     lib.wide_status.argtypes = [_c_void_p, _c_void_p, ctypes.POINTER(_c_int)]
     lib.wide_set_wait_limit_ns.argtypes = [_c_void_p, ctypes.c_uint64]
+    lib.wide_selftest_wait.argtypes = [_c_void_p, _c_void_p]
     lib.wide_profile_begin.argtypes = [_c_void_p, _c_int]
     lib.wide_profile_end.argtypes = [_c_void_p, _c_void_p, ctypes.c_char_p, _c_size_t]
     lib.wide_launch_count.argtypes = [_c_void_p, ctypes.POINTER(ctypes.c_ulonglong)]
@@ -151,6 +152,13 @@ class Context:
         v = _c_int(0)
         _check(self.lib.wide_status(self.handle, _stream(), ctypes.byref(v)), "wide_status")
         return v.value
+
+    def set_wait_limit_ns(self, ns: int):
+        _check(self.lib.wide_set_wait_limit_ns(self.handle, int(ns)), "wide_set_wait_limit_ns")
+
+    def selftest_wait(self):
+        """Enqueue the kernel whose only wait can never be satisfied (see wide_selftest_wait)."""
+        _check(self.lib.wide_selftest_wait(self.handle, _stream()), "wide_selftest_wait")
 
     def profile_begin(self, max_records: int = 4096):
         _check(self.lib.wide_profile_begin(self.handle, max_records), "wide_profile_begin")
