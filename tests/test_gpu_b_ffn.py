@@ -129,6 +129,19 @@ def test_prefill_tc_token_order_is_optional_and_does_not_change_the_result(ctx):
     assert_close(y1, y2.float().cpu().numpy().astype(np.float64), "same result either way", rel=1e-2)
 
 
+def test_prefill_tc_token_level_skipping_is_the_one_decision_per_token_case(ctx):
+    """M-axis (dynamic depth) routing of Section 3.3: one decision per token for the whole FFN is
+    the mask whose columns are all equal; skipped tokens give exact zeros."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("depth", tokens=700, hidden=512, d_ff=1024, group=128, k=8)
+    rng = np.random.default_rng(21)
+    keep = rng.random(cfg.tokens) < 0.4
+    mask = np.repeat(keep[:, None], cfg.n_groups, axis=1)
+    y, ref, _ = _run_ffn(ctx, cfg, 6, binding.FLAG_FORCE_PREFILL, mask=mask)
+    assert (y.float().cpu().numpy()[~keep] == 0.0).all()
+    assert_close(y, ref, "token-level skipping")
+
+
 def test_prefill_tc_agrees_with_simt_and_is_deterministic(ctx):
     from paper_2607_28418_b200 import binding
     cfg = synth.WideConfig("t", tokens=300, hidden=512, d_ff=1024, group=128, k=4)
