@@ -213,10 +213,15 @@ def run_ours(args):
     cfg = make_config(args)
     peaks = load_peaks()
     ctx = binding.Context(local)
-    oproj = args.op == "oproj"
+    qproj = args.op == "qproj"
+    oproj = args.op == "oproj" or qproj    # both run on the attention half: one GEMM, attention groups
     if oproj:
         case = synth.make_oproj_case(cfg, 1000 * rank)  # every rank its own token shard
         case["w_router"] = case.pop("w_router_attn")
+        if qproj:   # routed query projection: W_q [H*d, D], output [T, H*d]
+            case.pop("w_o")
+            case.pop("attn_out")
+            case["w_q"] = synth.make_weight(np.random.default_rng(1000 * rank + 17), cfg.attn_dim, cfg.hidden, 0.02, cfg.dtype)
         cfg = cfg.with_(d_ff=cfg.attn_dim, group=cfg.attn_group, k=cfg.attn_k)  # the op's inner dim / groups
     else:
         case = synth.make_ffn_case(cfg, 1000 * rank)
@@ -224,7 +229,8 @@ def run_ours(args):
     T, NG = cfg.tokens, cfg.n_groups
     W = (NG + 31) // 32
     bits = torch.empty((T, W), dtype=torch.int32, device=dev)
-    y = torch.empty((T, cfg.hidden), dtype=torch.bfloat16, device=dev)
+    out_dim = cfg.d_ff if qproj else cfg.hidden
+    y = torch.empty((T, out_dim), dtype=torch.bfloat16, device=dev)
     meta = None
     decode = T <= binding.DECODE_MAX_TOKENS
 
@@ -238,13 +244,15 @@ def run_ours(args):
     if decode and not args.flush_l2:
         per_copy = (1 if oproj else 3) * cfg.d_ff * cfg.hidden * 2
         n_copies = max(2, -(-(640 << 20) // per_copy))
-    wkeys = ("w_o",) if oproj else ("w_gate", "w_up", "w_down")
+    wkeys = ("w_q",) if qproj else ("w_o",) if oproj else ("w_gate", "w_up", "w_down")
     wsets = [{k: d[k] for k in wkeys}]
     for _ in range(n_copies - 1):
         wsets.append({k: d[k].clone() for k in wkeys})
 
     def main_op(x_in, w, y_out):
-        if oproj:
+        if qproj:
+            binding.wide_qproj(ctx, x_in, w["w_q"], cfg.group, meta, y=y_out)
+        elif oproj:
             binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out)
         else:
             binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out)
@@ -356,7 +364,7 @@ def run_ours(args):
     # ---- end to end: pinned host input -> device, whole path, result -> host, every step;
     # double-buffered over three streams so the copies of neighbouring steps overlap the compute
     x_host = torch.from_numpy(synth.to_bf16_bits(case["x"]).view(np.int16)).view(torch.bfloat16).pin_memory()
-    y_host = [torch.empty((T, cfg.hidden), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    y_host = [torch.empty((T, out_dim), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
     ev = {n: [torch.cuda.Event(), torch.cuda.Event()] for n in ("in", "run", "out")}
 
@@ -682,8 +690,8 @@ def main():
     ap.add_argument("--router", default="", choices=["", "random", "clustered", "clustered_corr"])
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--group", type=int, default=0)
-    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn"],
-                    help="oproj and attn need a workload with an attention half")
+    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn", "qproj"],
+                    help="oproj, qproj and attn need a workload with an attention half")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")

@@ -7,6 +7,7 @@
  *   wide_ffn        block-skipping SwiGLU FFN                     (Eq. 3; Algorithms 2 and 3)
  *   wide_oproj      head-group-masked attention output projection (Eq. 2; Eq. 10, Algorithm 3)
  *   wide_attn       head-group-masked causal attention, prefill   (Eq. 1; Algorithm 4)
+ *   wide_qproj      routed query projection, GEMM-MN              (Eq. 1 under the mask; Algorithm 2)
  *   wide_unpermute  the scatter epilogue as a standalone step     (Algorithm 2, epilogue)
  *
  * General rules
@@ -261,6 +262,20 @@ WIDE_API int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k
               int tokens_q, int tokens_k, int n_q_heads, int n_kv_heads, int head_dim,
               int heads_per_group, const int32_t* perm, const int32_t* counts, int causal, float scale,
               void* o, unsigned flags);
+
+/*
+ * wide_qproj -- the query projection under the head-group mask (Section 3.1: only the active head
+ * groups of a token compute their queries), Algorithm 2 (GEMM-MN) with a plain store epilogue:
+ *     y[t, gG:(g+1)G] = x[t, :] W[gG:(g+1)G, :]^T   if group g is active for token t, else 0.
+ *   x [tokens, hidden], w [n_out, hidden] (Linear layout), y out [tokens, n_out]: bf16
+ *   perm [n_groups, tokens], counts [n_groups]: outputs of wide_reorder for the mask,
+ *       n_groups = n_out / group <= WIDE_MAX_GROUPS
+ * Needs dtype bf16, hidden % 64 == 0, group in {128, 256, 512}.  y is fully overwritten.
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, ALIGNMENT, CUDA; WIDE_ERR_TIMEOUT through wide_status.
+ */
+WIDE_API int wide_qproj(wide_ctx* ctx, void* stream, const void* x, const void* w, int dtype, int tokens,
+               int hidden, int n_out, int group, const int32_t* perm, const int32_t* counts, void* y,
+               unsigned flags);
 
 /*
  * wide_unpermute -- scatter epilogue of Algorithm 2 as its own call: packed-sorted rows back to

@@ -22,6 +22,8 @@ ffn                   Eq. 3 literally: (phi(X Wg^T) * (X Wu^T)) gated group-wise
                       mask, times Wd^T, with phi = SiLU.
 oproj                 Eq. 2 / Eq. 10: (A gated group-wise) Wo^T.
 unpermute/gather      the scatter epilogue of Algorithm 2 as a standalone step.
+qproj                 the query projection under the head-group mask: (X Wq^T) gated
+                      group-wise (N-axis gating of Section 3.3, Appendix A's N-axis form).
 masked_attention      Eq. 1 with the head-group mask of Section 3.1 and the causal key
                       range of Algorithm 4 (delta = T_k - T_q): plain softmax attention
                       for every active (token, head group) pair, zeros elsewhere.  The
@@ -230,6 +232,13 @@ def oproj(attn_out: ArrayLike, w_o: ArrayLike, mask: np.ndarray, group: int) -> 
 
 
 # ----------------------------------------------------------------------------- gather / scatter
+def qproj(x: ArrayLike, w: ArrayLike, mask: np.ndarray, group: int) -> np.ndarray:
+    """Routed query projection (Section 3.1; the N-axis case of Section 3.3): the output channels of
+    group g are computed for the tokens that selected g and are zero for the others,
+    y = (x W^T) gated group-wise by the mask.  x [T, D], w [n_out, D], mask [T, n_out/group]."""
+    return (_f64(x) @ _f64(w).T) * expand_group_mask(mask, group)
+
+
 def masked_attention(q: ArrayLike, k: ArrayLike, v: ArrayLike, mask: np.ndarray, heads_per_group: int,
                      causal: bool = True, scale: Optional[float] = None) -> np.ndarray:
     """Head-group-masked softmax attention (Eq. 1, Section 3.1; key range of Algorithm 4).

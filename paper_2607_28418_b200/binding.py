@@ -27,7 +27,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
            "wide_profile_end", "wide_launch_count", "wide_selftest_wait", "wide_strerror",
            "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_ffn",
-           "wide_oproj", "wide_attn", "wide_unpermute"]
+           "wide_oproj", "wide_attn", "wide_qproj", "wide_unpermute"]
 
 _c_void_p, _c_int, _c_size_t, _c_uint = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
 
@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
                                _c_void_p, _c_size_t, _c_uint]
     lib.wide_attn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
                               _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_int, ctypes.c_float, _c_void_p, _c_uint]
+    lib.wide_qproj.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_int,
+                               _c_void_p, _c_void_p, _c_void_p, _c_uint]
     lib.wide_unpermute.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                    _c_int, _c_int, _c_int, _c_void_p]
     for name in EXPORTS:
@@ -318,6 +320,19 @@ def wide_attn(ctx: Context, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, n
                            1 if causal else 0, float(scale), _ptr(o), flags)
     _check(rc, "wide_attn")
     return o
+
+
+def wide_qproj(ctx: Context, x: torch.Tensor, w: torch.Tensor, group: int, meta: Dict[str, torch.Tensor],
+               flags: int = 0, y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x [T, D], w [n_out, D] bf16; meta = wide_reorder outputs of the [T, n_out/group] mask."""
+    T, D = x.shape
+    n_out = w.shape[0]
+    if y is None:
+        y = torch.empty((T, n_out), dtype=x.dtype, device=x.device)
+    rc = ctx.lib.wide_qproj(ctx.handle, _stream(), _ptr(x), _ptr(w), _dtype_code(x), T, D, n_out, group,
+                            _ptr(meta["perm"]), _ptr(meta["counts"]), _ptr(y), flags)
+    _check(rc, "wide_qproj")
+    return y
 
 
 def wide_unpermute(ctx: Context, src_packed: torch.Tensor, meta: Dict[str, torch.Tensor], tokens: int,

@@ -324,6 +324,20 @@ int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const v
                                        n_kv_heads, head_dim, heads_per_group, perm, counts, causal ? 1 : 0, scale, o);
 }
 
+int wide_qproj(wide_ctx* ctx, void* stream, const void* x, const void* w, int dtype, int tokens, int hidden,
+               int n_out, int group, const int32_t* perm, const int32_t* counts, void* y, unsigned flags) {
+    (void)flags;
+    if (!ctx || !x || !w || !perm || !counts || !y) return WIDE_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || n_out <= 0 || group <= 0 || n_out % group != 0) return WIDE_ERR_INVALID_ARG;
+    if (dtype != WIDE_BF16 || hidden % 64 != 0 || (group != 128 && group != 256 && group != 512) || !ctx->encode_tiled)
+        return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (n_out / group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(x) || !wide_aligned16(w) || !wide_aligned16(y)) return WIDE_ERR_ALIGNMENT;
+    return wide_launch_linear_mn_tc(ctx, static_cast<cudaStream_t>(stream), x, w, tokens, hidden, n_out, group, perm,
+                                    counts, y);
+}
+
 int wide_unpermute(wide_ctx* ctx, void* stream, const void* src_packed, const int32_t* perm,
                    const int32_t* counts, const int32_t* offsets, int tokens, int n_groups,
                    int group, int elem_bytes, void* dst) {

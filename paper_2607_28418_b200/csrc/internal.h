@@ -124,3 +124,7 @@ bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base
 int wide_launch_attn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, const void* v, int Tq,
                                 int Tk, int Hq, int Hkv, int head_dim, int hpg, const int32_t* perm,
                                 const int32_t* counts, int causal, float scale, void* o);
+
+// tcgen05 routed linear layer (GEMM-MN, bf16): y [T, Nout] bf16, zeros for inactive (token, group) pairs.
+int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w, int T, int D, int Nout,
+                             int G, const int32_t* perm, const int32_t* counts, void* y);

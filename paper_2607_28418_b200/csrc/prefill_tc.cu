@@ -564,7 +564,10 @@ __device__ __forceinline__ float silu_mul_fast(float g, float u) {
 
 constexpr int kGuThreads = 448;  // TMA, MMA, 4 gather warps, 8 epilogue warps
 
-template <int BN>  // channels per item (UMMA N = 2*BN)
+// kLinear = false: gate/up + SwiGLU, an item covers BN channels (B = BN rows of W_gate stacked on
+// BN rows of W_up).  kLinear = true: the same GEMM-MN for ONE weight and no activation (the
+// routed Q projection): an item covers 2*BN output channels (B = 2*BN consecutive rows of W).
+template <int BN, bool kLinear>  // UMMA N = 2*BN
 __global__ void __launch_bounds__(kGuThreads, 1)
 gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
               const __nv_bfloat16* __restrict__ X, const int32_t* __restrict__ perm,
@@ -585,7 +588,8 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStagesG + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nsub = G / BN;
+    constexpr int kItemCh = kLinear ? 2 * BN : BN;   // output channels of one item
+    const int nsub = G / kItemCh;
     const int n_gs = NG * nsub;
 
     if (tid == 0) {
@@ -647,7 +651,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             GuSched sched(s_dbl, s_sgl, n_gs);
             GuItem w;
             while (ok && sched.next(w)) {
-                const int crow = (w.gs / nsub) * G + (w.gs % nsub) * BN;
+                const int crow = (w.gs / nsub) * G + (w.gs % nsub) * kItemCh;
                 for (int k = 0; k < nk; ++k, ++it) {
                     const int s = it % kStagesG;
                     const uint32_t ph = (it / kStagesG) & 1;
@@ -655,7 +659,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     mbar_arrive_expect_tx(full + 8 * s, kBBytes);
                     const uint32_t b_dst = smem_u32(base + s * kStageBytes) + kAB;
                     tma_load_2d(b_dst, &tmG, k * kBK, crow, full + 8 * s);
-                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, crow, full + 8 * s);
+                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, kLinear ? crow + BN : crow, full + 8 * s);
                 }
             }
             if (!ok) { report_timeout(status); abort_grace(); }
@@ -749,6 +753,17 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         uint4* ep_stage = reinterpret_cast<uint4*>(base + kStagesG * kStageBytes + 128) + ew * 128;  // 2 KB per warp
         int tc = 0;
         bool ok = true;
+        if constexpr (kLinear) {
+            // the output is a result, not scratch: a group nobody selected has no item that would
+            // zero its columns, so the CTAs share those rows here
+            for (int g0 = 0; g0 < NG; ++g0) {
+                if (counts[g0] != 0) continue;
+                const int ppr = G / 8;   // 16-byte pieces per row
+                for (long long i = static_cast<long long>(blockIdx.x) * 256 + e; i < static_cast<long long>(T) * ppr;
+                     i += static_cast<long long>(gridDim.x) * 256)
+                    reinterpret_cast<uint4*>(H + (i / ppr) * Dff + g0 * G)[i % ppr] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
         GuSched sched(s_dbl, s_sgl, n_gs);
         GuItem w;
         while (ok && sched.next(w)) {
@@ -761,7 +776,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                 // of a group that is active anywhere.  Groups nobody selected are never read.
                 // kLpr consecutive lanes write one row's piece, so a warp store touches whole
                 // lines (scattered 16-byte stores would keep the L1 busy and starve the gather).
-                constexpr int kLpr = BN / 8;          // lanes per row: one 16-byte store each
+                constexpr int kLpr = kItemCh / 8;     // lanes per row: one 16-byte store each
                 constexpr int kRows = 256 / kLpr;     // rows per sweep of the 8 warps
                 const int nt = (c + kBM - 1) / kBM;
                 const int per = (T - c + nt - 1) / nt;
@@ -772,7 +787,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     for (int jj = j0 + zr; jj < j1; jj += kRows) {
                         int tz = perm[static_cast<size_t>(g) * T + jj];
                         if (token_rank) tz = token_rank[tz];   // H rows are kept in clustered token order
-                        reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * BN)[zp] =
+                        reinterpret_cast<uint4*>(H + static_cast<size_t>(tz) * Dff + g * G + sub * kItemCh)[zp] =
                             make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
@@ -798,29 +813,40 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     tmem_ld_wait();
                     // lane = row here; transpose through shared memory so that 4 lanes write one
                     // row's 64 bytes (a warp store then touches 8 rows instead of 32)
+                    // one pass (SwiGLU) or two (linear: the "gate" and the "up" columns are two
+                    // separate blocks of output channels, BN apart)
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t o[4];
+                    for (int pass = 0; pass < (kLinear ? 2 : 1); ++pass) {
 #pragma unroll
-                        for (int x4 = 0; x4 < 4; ++x4) {
-                            const int i = 8 * v + 2 * x4;
-                            o[x4] = pack_bf16(silu_mul_fast(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
-                                              silu_mul_fast(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int x4 = 0; x4 < 4; ++x4) {
+                                const int i = 8 * v + 2 * x4;
+                                if constexpr (kLinear) {
+                                    const uint32_t (&src)[32] = pass == 0 ? gr : ur;
+                                    o[x4] = pack_bf16(__uint_as_float(src[i]), __uint_as_float(src[i + 1]));
+                                } else {
+                                    o[x4] = pack_bf16(silu_mul_fast(__uint_as_float(gr[i]), __uint_as_float(ur[i])),
+                                                      silu_mul_fast(__uint_as_float(gr[i + 1]), __uint_as_float(ur[i + 1])));
+                                }
+                            }
+                            // piece v of row `lane` sits in slot v ^ ((lane >> 1) & 3): no bank conflicts
+                            // on the way in (8 rows, one piece) nor on the way out (2 rows, 4 pieces)
+                            ep_stage[lane * 4 + (v ^ ((lane >> 1) & 3))] = make_uint4(o[0], o[1], o[2], o[3]);
                         }
-                        // piece v of row `lane` sits in slot v ^ ((lane >> 1) & 3): no bank conflicts
-                        // on the way in (8 rows, one piece) nor on the way out (2 rows, 4 pieces)
-                        ep_stage[lane * 4 + (v ^ ((lane >> 1) & 3))] = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                    __syncwarp();
+                        __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int r = 8 * i + (lane >> 2), pc = lane & 3;
-                        const int tr = __shfl_sync(0xffffffffu, tokh[half], r);
-                        const uint4 val = ep_stage[r * 4 + (pc ^ ((r >> 1) & 3))];
-                        if (tr >= 0)
-                            *reinterpret_cast<uint4*>(H + static_cast<size_t>(tr) * Dff + g * G + sub * BN + chalf * kCh + c0 + pc * 8) = val;
+                        for (int i = 0; i < 4; ++i) {
+                            const int r = 8 * i + (lane >> 2), pc = lane & 3;
+                            const int tr = __shfl_sync(0xffffffffu, tokh[half], r);
+                            const uint4 val = ep_stage[r * 4 + (pc ^ ((r >> 1) & 3))];
+                            if (tr >= 0)
+                                *reinterpret_cast<uint4*>(H + static_cast<size_t>(tr) * Dff + g * G + sub * kItemCh + pass * BN +
+                                                          chalf * kCh + c0 + pc * 8) = val;
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
             }
             tc_fence_before_sync();
@@ -915,19 +941,18 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
-template <int BN>
+template <int BN, bool kLinear>
 int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu, int T, int D,
                   int Dff, int G, const int32_t* perm, const int32_t* counts, const int32_t* token_rank, void* h) {
     CUtensorMap tmG, tmU;
     if (!make_tmap_bf16(ctx, &tmG, wg, Dff, D, BN) || !make_tmap_bf16(ctx, &tmU, wu, Dff, D, BN)) return WIDE_ERR_CUDA;
     constexpr int stages = BN == 128 ? 3 : 4;
     constexpr int smem = stages * (2 * kABytes + 2 * BN * kBK * 2) + 128 + 8 * 2048 + 1024;  // ring, barriers, epilogue staging
-    WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    WideLaunch l(ctx, s, "prefill_gateup");
-    gateup_kernel<BN><<<ctx->sm_count, kGuThreads, smem, s>>>(tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm,
-                                                              counts, token_rank, Dff / G, T, D, Dff, G,
-                                                              static_cast<__nv_bfloat16*>(h), ctx->d_status,
-                                                              ctx->wait_ns);
+    WIDE_CUDA_CHECK(cudaFuncSetAttribute(gateup_kernel<BN, kLinear>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    WideLaunch l(ctx, s, kLinear ? "prefill_linear_mn" : "prefill_gateup");
+    gateup_kernel<BN, kLinear><<<ctx->sm_count, kGuThreads, smem, s>>>(
+        tmG, tmU, static_cast<const __nv_bfloat16*>(x), perm, counts, token_rank, Dff / G, T, D, Dff, G,
+        static_cast<__nv_bfloat16*>(h), ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -946,10 +971,19 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
     // H [T, Dff] is kept in clustered token order when token_order / token_rank are given (row
     // token_rank[t] holds token t), else in token order.  Inactive (token, group) pairs of H must
     // read as zero in the down projection: the gate/up kernel's epilogue warps write those zeros.
-    int rc = (G == 64) ? launch_gateup<64>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h)
-                       : launch_gateup<128>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h);
+    int rc = (G == 64) ? launch_gateup<64, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h)
+                       : launch_gateup<128, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h);
     if (rc != WIDE_OK) return rc;
     return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype, token_order);
+}
+
+// y[t, gG:(g+1)G] = x_t W[gG:(g+1)G, :]^T for active (t, g), exact zeros elsewhere (Algorithm 2 with a
+// plain store epilogue).  G = 128 runs items of 128 channels, G >= 256 items of 256.
+int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w, int T, int D, int Nout,
+                             int G, const int32_t* perm, const int32_t* counts, void* y) {
+    if (T == 0) return WIDE_OK;
+    return (G == 128) ? launch_gateup<64, true>(ctx, s, x, w, w, T, D, Nout, G, perm, counts, nullptr, y)
+                      : launch_gateup<128, true>(ctx, s, x, w, w, T, D, Nout, G, perm, counts, nullptr, y);
 }
 
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T, int D,

@@ -82,3 +82,37 @@ def test_attn_rejects_bad_arguments(ctx):
     q = torch.zeros((128, 4 * 128), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(binding.WideError):
         binding.wide_attn(ctx, q, q, q, 4, 3, 2, meta)             # heads not divisible
+
+
+# ----------------------------------------------------------------------------- routed Q projection
+@pytest.mark.parametrize("T,D,n_out,G,p", [(300, 512, 1024, 128, 0.5), (640, 1024, 2048, 512, 0.5),
+                                           (200, 256, 1024, 256, 0.3), (1100, 512, 1536, 128, 0.7)])
+def test_qproj_matches_oracle(ctx, T, D, n_out, G, p):
+    from paper_2607_28418_b200 import binding
+    rng = np.random.default_rng(T + G)
+    x = synth.make_activations(rng, T, D, "bf16", "random")
+    w = synth.make_weight(rng, n_out, D, 0.02, "bf16")
+    mask = synth.bernoulli_mask(T, T, n_out // G, p)
+    meta = meta_to_dev(wo.reorder(mask, 128))
+    y = binding.wide_qproj(ctx, to_dev(x, "bf16"), to_dev(w, "bf16"), G, meta)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    ref = wo.qproj(x, w, mask, G)
+    assert (y.float().cpu().numpy()[~wo.expand_group_mask(mask, G)] == 0.0).all()
+    assert_close(y, ref, "qproj")
+
+
+def test_qproj_closed_cases(ctx):
+    from paper_2607_28418_b200 import binding
+    T, D, n_out, G = 260, 256, 512, 128
+    rng = np.random.default_rng(4)
+    x = synth.make_activations(rng, T, D, "bf16", "random")
+    w = synth.make_weight(rng, n_out, D, 0.02, "bf16")
+    xd, wd = to_dev(x, "bf16"), to_dev(w, "bf16")
+    ones = np.ones((T, n_out // G), dtype=bool)
+    y = binding.wide_qproj(ctx, xd, wd, G, meta_to_dev(wo.reorder(ones, 128)))
+    assert_close(y, x.astype(np.float64) @ w.astype(np.float64).T, "qproj dense")
+    y0 = binding.wide_qproj(ctx, xd, wd, G, meta_to_dev(wo.reorder(~ones, 128)))
+    assert (y0 == 0).all().item()
+    with pytest.raises(binding.WideError):
+        binding.wide_qproj(ctx, xd, wd, 64, meta_to_dev(wo.reorder(np.ones((T, n_out // 64), dtype=bool), 128)))

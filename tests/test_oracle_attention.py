@@ -96,3 +96,21 @@ def test_shifting_every_key_changes_nothing():
     a = wo.masked_attention(q, k, v, mask, 2)
     b = wo.masked_attention(q, k + np.linspace(-1, 1, 8), v, mask, 2)
     np.testing.assert_allclose(a, b, rtol=1e-9, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- routed Q projection
+def test_qproj_is_a_masked_library_matmul_and_matches_loops():
+    rng = np.random.default_rng(12)
+    T, D, G, NG = 9, 5, 4, 3
+    x, w = rng.standard_normal((T, D)), rng.standard_normal((NG * G, D))
+    mask = rng.random((T, NG)) < 0.5
+    got = wo.qproj(x, w, mask, G)
+    ref = (torch.from_numpy(x) @ torch.from_numpy(w).T).numpy()
+    for t in range(T):
+        for c in range(NG * G):
+            want = sum(x[t, i] * w[c, i] for i in range(D)) if mask[t, c // G] else 0.0
+            assert abs(got[t, c] - want) < 1e-12
+            if mask[t, c // G]:
+                assert abs(got[t, c] - ref[t, c]) < 1e-12
+    assert (wo.qproj(x, w, np.zeros_like(mask), G) == 0).all()
+    np.testing.assert_allclose(wo.qproj(x, w, np.ones_like(mask), G), ref, atol=1e-12)
