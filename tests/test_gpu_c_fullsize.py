@@ -99,3 +99,42 @@ def test_llama13b_layer_oproj_and_ffn(ctx):
     assert ctx.status() == 0
     # FFN half of the layer, prefill
     _chain(ctx, cfg, 1, n_sample=32)
+
+
+def test_llama13b_layer_attention_and_qproj(ctx):
+    """Masked attention and the routed Q projection at the 13B layer's full size (one causal
+    sequence of 4096 positions, 40 heads of 128, 10 routing groups).  Attention heads are
+    independent, so the oracle computes three whole heads from different groups; a Q-projection
+    row depends only on its own token."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.CONFIGS["llama13b_layer"]
+    T, hd = cfg.tokens, 128
+    H, hpg, NG = cfg.attn_dim // hd, cfg.attn_group // hd, cfg.attn_n_groups
+    case = synth.make_oproj_case(cfg, 0)
+    xd, wr = to_dev(case["x"], "bf16"), to_dev(case["w_router_attn"], "bf16")
+    bits, _ = binding.wide_route(ctx, xd, wr, NG, cfg.attn_k)
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router_attn"]), cfg.attn_k)
+    assert (bits_to_host(bits) == wo.pack_mask_bits(mask)).all()
+    meta = binding.wide_reorder(ctx, bits, NG, 128)
+    ac = synth.make_attn_case(0, T, T, H, H, hd)
+    o = binding.wide_attn(ctx, to_dev(ac["q"].reshape(T, -1), "bf16"), to_dev(ac["k"].reshape(T, -1), "bf16"),
+                          to_dev(ac["v"].reshape(T, -1), "bf16"), H, H, hpg, meta)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    got = o.float().cpu().numpy().reshape(T, H, hd)
+    head_mask = np.repeat(mask, hpg, axis=1)
+    assert (got[~head_mask] == 0.0).all()
+    for h in (0, 17, 39):
+        g = h // hpg
+        ref = wo.masked_attention(ac["q"][:, h:h + 1], ac["k"][:, h:h + 1], ac["v"][:, h:h + 1], mask[:, g:g + 1], 1)
+        err = np.abs(got[:, h] - ref[:, 0]).max()
+        assert err <= REL_TOL * np.abs(ref).max(), f"head {h}: {err:.3e}"
+    # routed Q projection on sampled rows
+    wq = synth.make_weight(np.random.default_rng(3), cfg.attn_dim, cfg.hidden, 0.02, "bf16")
+    yq = binding.wide_qproj(ctx, xd, to_dev(wq, "bf16"), cfg.attn_group, meta)
+    rows = np.random.default_rng(1).integers(0, T, size=64)
+    ref = wo.qproj(case["x"][rows], wq, mask[rows], cfg.attn_group)
+    gq = yq[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert (gq[~wo.expand_group_mask(mask[rows], cfg.attn_group)] == 0.0).all()
+    assert np.abs(gq - ref).max() <= REL_TOL * np.abs(ref).max()
+    assert ctx.status() == 0
