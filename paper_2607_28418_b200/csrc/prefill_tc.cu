@@ -306,6 +306,9 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // (1.5x fewer bytes per FLOP than the 128 x 256 tile) and the 3-stage ring covers 1.5x more
 // latency.  The two accumulators fill all 512 TMEM columns, so the epilogue of a tile does not
 // overlap the next tile's MMAs (a few percent); with one or two tiles per CTA that is cheap.
+// The N extent is cut into n_n column tiles whose widths are multiples of 16 and differ by at
+// most 16 (the host picks n_n so that the tiles fill the SMs evenly: 18 tiles of 224/240 columns
+// instead of 16 of 256 put 144 CTAs to work at T=2048, N=4096 where 128 would leave 20 SMs idle).
 constexpr int kStages2 = 3;
 constexpr int kA2Bytes = 2 * kABytes;            // 256 rows x 128 B
 constexpr int kB2Bytes = 256 * kBK * 2;          // 256 rows x 128 B
@@ -316,7 +319,7 @@ __global__ void __launch_bounds__(192, 1)
 down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N,
                int K, int G, void* __restrict__ Y,
-               int out_bf16, int* __restrict__ status, unsigned long long wait_ns) {
+               int out_bf16, int n_n, int box_n, int* __restrict__ status, unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStages2 * kStage2Bytes);
@@ -347,9 +350,14 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_m = (T + 255) / 256, n_n = (N + 255) / 256;
+    const int n_m = (T + 255) / 256;
     const int n_tiles = n_m * n_n;
     const int NG = K / G, ksub = G / kBK;
+    // column tile n covers [col0(n), col0(n) + width(n)): sixteenths of N dealt as evenly as possible
+    const int q16 = (N + 15) / 16, q_base = q16 / n_n, q_rem = q16 % n_n;
+    auto col0 = [&](int n) { return 16 * (n * q_base + min(n, q_rem)); };
+    auto width = [&](int n) { return 16 * (q_base + (n < q_rem ? 1 : 0)); };
+    const uint32_t stage_tx = kA2Bytes + static_cast<uint32_t>(box_n) * (kBK * 2);   // TMA always moves whole boxes
 
     // OR of the mask words of the tile's 256 tokens
     auto tile_mask = [&](int m, uint32_t (&act)[kMaskWords]) {
@@ -375,11 +383,11 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int s = it % kStages2;
                         const uint32_t ph = (it / kStages2) & 1;
                         if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
-                        mbar_arrive_expect_tx(full + 8 * s, kStage2Bytes);
+                        mbar_arrive_expect_tx(full + 8 * s, stage_tx);
                         const uint32_t a_dst = smem_u32(base + s * kStage2Bytes);
                         const int kcol = g * G + kk * kBK;
                         tma_load_2d(a_dst, &tmA, kcol, m * 256, full + 8 * s);
-                        tma_load_2d(a_dst + kA2Bytes, &tmB, kcol, n * 256, full + 8 * s);
+                        tma_load_2d(a_dst + kA2Bytes, &tmB, kcol, col0(n), full + 8 * s);
                     }
                 }
             }
@@ -388,11 +396,11 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!ok && lane == 0) { report_timeout(status); abort_grace(); }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ UMMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(kBM, 256);
         int it = 0, tc = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
             const int m = tile % n_m;
+            const uint32_t idesc = umma_idesc_bf16(kBM, width(tile / n_m));
             uint32_t act[kMaskWords];
             tile_mask(m, act);
             if (lane == 0) {
@@ -445,18 +453,30 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int pos = m * 256 + half * 128 + q * 32 + lane;
                 const int row = (order && pos < T) ? order[pos] : pos;   // token that owns this output row
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256;
+                const int wn = width(n), cbase = col0(n);
 #pragma unroll 1
-                for (int c0 = 0; c0 < 256; c0 += 32) {
+                for (int c0 = 0; c0 < wn; c0 += 32) {
+                    // widths are multiples of 16: the last chunk of a tile may hold 16 columns
+                    const bool whole = c0 + 32 <= wn;
                     uint32_t r[32];
                     if (any) {
-                        tmem_ld_32x32(taddr + c0, r);
-                        tmem_ld_wait();
+                        if (whole) {
+                            tmem_ld_32x32(taddr + c0, r);
+                            tmem_ld_wait();
+                        } else {
+                            uint32_t r16[16];
+                            tmem_ld_32x16(taddr + c0, r16);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) { r[i] = r16[i]; r[16 + i] = 0u; }
+                        }
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = 0u;
                     }
-                    const int col = n * 256 + c0;
-                    if (row < T && col + 32 <= N) {
+                    const int col = cbase + c0;
+                    const int ncol = whole ? 32 : 16;
+                    if (row < T && col + ncol <= N) {
                         if (out_bf16) {
                             uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(row) * N + col);
 #pragma unroll
@@ -466,12 +486,13 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
                                 o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
                                 o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-                                dst[v] = o;
+                                if (8 * v < ncol) dst[v] = o;
                             }
                         } else {
                             uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(Y) + static_cast<size_t>(row) * N + col);
 #pragma unroll
-                            for (int v = 0; v < 8; ++v) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                            for (int v = 0; v < 8; ++v)
+                                if (4 * v < ncol) dst[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                         }
                     }
                 }
@@ -920,24 +941,43 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
+// Column tiling of the 256-row kernel: the number of column tiles n_n (widths = sixteenths of N
+// dealt evenly, at most 256) that minimises waves x width, with a mild penalty for narrow tiles
+// (a narrower B tile is reused by fewer FLOPs).  Returns the cost in units of a 256-wide tile.
+double pick_down256_tiling(int sm, int T, int N, int* n_n_out, int* wmax_out) {
+    const int n_m = (T + 255) / 256, q16 = (N + 15) / 16;
+    const int nn0 = (N + 255) / 256;
+    double best = 1e30;
+    for (int nn = nn0; nn <= nn0 + nn0 / 2 + 1 && nn <= q16; ++nn) {
+        const int wmax = 16 * ((q16 + nn - 1) / nn);
+        if (wmax > 256 || wmax < 160) continue;
+        const int waves = (n_m * nn + sm - 1) / sm;
+        const double cost = waves * (wmax / 256.0) * (1.0 + 0.5 * (256 - wmax) / 256.0);
+        if (cost < best - 1e-9) { best = cost; *n_n_out = nn; *wmax_out = wmax; }
+    }
+    return best;
+}
+
 // Picks the tile height for the down / output projection: 256-row tiles move fewer bytes per FLOP
 // (about 0.8 of the time per row), 128-row tiles quantise better over the SMs.
 int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                      int N, int K, int G, void* Y, int out_dtype, const int32_t* order) {
     const int sm = ctx->sm_count;
-    const int t128 = ((T + 127) / 128) * ((N + 255) / 256), t256 = ((T + 255) / 256) * ((N + 255) / 256);
+    const int t128 = ((T + 127) / 128) * ((N + 255) / 256);
+    int n_n = (N + 255) / 256, wmax = 256;
     const double cost128 = static_cast<double>((t128 + sm - 1) / sm);
-    const double cost256 = static_cast<double>((t256 + sm - 1) / sm) * 2.0 * 0.8;
+    const double cost256 = pick_down256_tiling(sm, T, N, &n_n, &wmax) * 2.0 * 0.8;
     if (cost128 <= cost256)
         return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype, -1, "prefill_down", 1, nullptr, order);
     CUtensorMap tmA, tmB;
-    if (!make_tmap_bf16(ctx, &tmA, A, T, K, 256) || !make_tmap_bf16(ctx, &tmB, B, N, K, 256)) return WIDE_ERR_CUDA;
+    if (!make_tmap_bf16(ctx, &tmA, A, T, K, 256) || !make_tmap_bf16(ctx, &tmB, B, N, K, wmax)) return WIDE_ERR_CUDA;
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2));
+    const int t256 = ((T + 255) / 256) * n_n;
     const int grid = t256 < sm ? t256 : sm;
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
     down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
-                                             ctx->d_status, ctx->wait_ns);
+                                             n_n, wmax, ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
