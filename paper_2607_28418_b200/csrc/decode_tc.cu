@@ -48,8 +48,9 @@ struct DecodeArgs {
     int is_ffn;
     int B, NT;
     int D, inner, G, NG, words;
-    int rows_valid;        // gate/up weight rows fetched per tile: min(G, 128)
+    int rows_valid;        // gate/up weight rows fetched per TMA box: min(G, 128)
     int blocks_per_group;  // gate/up: max(1, G / 128)
+    int gpb;               // gate/up: union groups per 128-row tile, max(1, 128 / G)
     int row_tiles;         // pass 2: ceil(D / 128)
     const uint32_t* mask_bits;
     const __nv_bfloat16* act_in;  // O-proj: attention output [B, inner]
@@ -100,6 +101,20 @@ struct Share {
 __device__ __forceinline__ int pieces_of_block(int blk, int spb, int L) {
     const int first = blk * spb, last = first + spb - 1;
     return last / L - first / L + 1;
+}
+
+// Gate/up tiles: channel of tile row r of block `slot_blk` (= union slot * blocks_per_group + block,
+// or, for groups narrower than a tile, the index of a pack of `gpb` consecutive union slots).
+__device__ __forceinline__ int gateup_channel(const DecodeArgs& a, const int* s_union, int n_union, int slot_blk, int r,
+                                              bool& valid) {
+    if (a.gpb > 1) {
+        const int slot = slot_blk * a.gpb + r / a.G;
+        valid = slot < n_union;
+        return valid ? s_union[slot] * a.G + r % a.G : 0;
+    }
+    const int ch = s_union[slot_blk / a.blocks_per_group] * a.G + (slot_blk % a.blocks_per_group) * kRows + r;
+    valid = r < a.rows_valid && ch < a.inner;
+    return ch;
 }
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
@@ -154,7 +169,8 @@ struct PassGeom {
 __device__ __forceinline__ PassGeom geom_of(int mode, const DecodeArgs& a, int n_union) {
     PassGeom g;
     if (mode == MODE_GATEUP) {
-        g.n_blocks = n_union * a.blocks_per_group * 2;   // block index = (slot * bpg + blk) * 2 + mat
+        // block index = (slot * bpg + blk) * 2 + mat; groups narrower than a tile share one (gpb per tile)
+        g.n_blocks = ((n_union + a.gpb - 1) / a.gpb) * a.blocks_per_group * 2;
         g.spb = a.D / kBKD;
     } else {
         g.n_blocks = a.row_tiles;
@@ -174,20 +190,26 @@ __device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* t
     const PassGeom g = geom_of(mode, a, n_union);
     const int ksub = a.G / kBKD;
     const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
-    const uint32_t stage_tx = static_cast<uint32_t>(rows_valid * kBKD * 2 + a.NT * kBKD * 2);
+    const uint32_t act_tx = static_cast<uint32_t>(a.NT * kBKD * 2);
     Share sh(blockIdx.x, g.total, g.L, g.spb);
     Segment sg;
     int step = 0;
     int n = P.n;
     while (sh.next(sg)) {
-        int row0, mat = 0;
+        int row0[2] = {0, 0}, nbox = 1, mat = 0;
         if (mode == MODE_GATEUP) {
             mat = sg.blk & 1;
             const int r = sg.blk >> 1;
-            row0 = s_union[r / a.blocks_per_group] * a.G + (r % a.blocks_per_group) * kRows;
+            if (a.gpb > 1) {
+                nbox = min(a.gpb, n_union - r * a.gpb);     // the last pack may be short
+                for (int j = 0; j < nbox; ++j) row0[j] = s_union[r * a.gpb + j] * a.G;
+            } else {
+                row0[0] = s_union[r / a.blocks_per_group] * a.G + (r % a.blocks_per_group) * kRows;
+            }
         } else {
-            row0 = sg.blk * kRows;
+            row0[0] = sg.blk * kRows;
         }
+        const uint32_t stage_tx = static_cast<uint32_t>(nbox * rows_valid * kBKD * 2) + act_tx;
         const CUtensorMap* tw = mat ? tmW1 : tmW0;
         for (int i = 0; i < sg.nsteps; ++i, ++step, ++n) {
             if (weights_only_steps >= 0 && step >= weights_only_steps) return true;  // pre-issue done
@@ -199,7 +221,8 @@ __device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* t
                 const uint32_t ph = (n / P.nstages) & 1;
                 if (!mbar_wait(P.empty + 8 * s, ph ^ 1u, a.wait_ns, P.abort_flag)) return false;
                 mbar_arrive_expect_tx(P.full + 8 * s, stage_tx);
-                tma_load_2d(dst, tw, col, row0, P.full + 8 * s);
+                for (int j = 0; j < nbox; ++j)
+                    tma_load_2d(dst + j * rows_valid * (kBKD * 2), tw, col, row0[j], P.full + 8 * s);
             }
             if (weights_only_steps < 0) tma_load_2d(dst + kWBytes, tmAct, col, 0, P.full + 8 * s);
         }
@@ -256,10 +279,10 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
             int prow;
             float* pbase;
             if (mode == MODE_GATEUP) {
-                const int sb = ps.blk >> 1;
-                prow = s_union[sb / a.blocks_per_group] * a.G + (sb % a.blocks_per_group) * kRows + e;
+                bool valid;
+                prow = gateup_channel(a, s_union, n_union, ps.blk >> 1, e, valid);
                 pbase = (ps.blk & 1) ? a.up : a.gate;
-                if (e >= rows_valid || prow >= a.inner) continue;
+                if (!valid) continue;
             } else {
                 prow = ps.blk * kRows + e;
                 pbase = a.yacc;
@@ -273,18 +296,18 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
     Share sh(blockIdx.x, g.total, g.L, g.spb);
     Segment sg;
     while (sh.next(sg)) {
-        int row0, mat = 0, slot_blk = 0;
+        int mat = 0, slot_blk = 0;
+        const int rloc = q * 32 + lane;
+        int row;
+        bool live;
         if (mode == MODE_GATEUP) {
             mat = sg.blk & 1;
             slot_blk = sg.blk >> 1;
-            row0 = s_union[slot_blk / a.blocks_per_group] * a.G + (slot_blk % a.blocks_per_group) * kRows;
+            row = gateup_channel(a, s_union, n_union, slot_blk, rloc, live);
         } else {
-            row0 = sg.blk * kRows;
+            row = sg.blk * kRows + rloc;
+            live = row < a.D;
         }
-        const int rloc = q * 32 + lane;
-        const int row = row0 + rloc;
-        const int rows_total = mode == MODE_GATEUP ? a.inner : a.D;
-        const bool live = rloc < rows_valid && row < rows_total;
         float* out = (mode == MODE_GATEUP ? (mat ? a.up : a.gate) : a.yacc) + static_cast<size_t>(row) * a.NT;
         const int buf = P.tc & 1;
         const uint32_t tph = (P.tc >> 1) & 1;
@@ -332,16 +355,20 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
             constexpr int kB4 = 8;  // 16-byte pieces per round: 2 * kB4 loads in flight per thread
             if (mode == MODE_GATEUP) {
                 // h[b, ch] for the 128 (or G) channels of this block; re-zero gate / up
-                const int gidx = s_union[slot_blk / a.blocks_per_group];
-                // which tokens execute this group: thread e < 64 looks at token e
-                const bool tb = e < a.B && wide_mask_bit(a.mask_bits, a.words, e, gidx);
+                // which tokens execute which group of the tile: thread e looks at token e % 64 for
+                // the group of the tile half e / 64 (one group per tile: both halves see the same)
+                const int vslot = a.gpb > 1 ? slot_blk * a.gpb + (e >> 6) : slot_blk / a.blocks_per_group;
+                const int vg = vslot < n_union ? s_union[vslot] : -1;
+                const bool tb = vg >= 0 && (e & 63) < a.B && wide_mask_bit(a.mask_bits, a.words, e & 63, vg);
                 const unsigned vote = __ballot_sync(0xffffffffu, tb);
-                if (lane == 0 && e < 64) s_tokmask[e >> 5] = vote;
+                if (lane == 0) s_tokmask[e >> 5] = vote;
                 epilogue_bar_sync();
+                bool ch_valid;
+                const int ch = gateup_channel(a, s_union, n_union, slot_blk, e, ch_valid);
+                const int mh = a.gpb > 1 ? 2 * (e / a.G) : 0;   // the mask words of this thread's group
                 const unsigned long long tokmask =
-                    static_cast<unsigned long long>(s_tokmask[0]) | (static_cast<unsigned long long>(s_tokmask[1]) << 32);
-                const int ch = gidx * a.G + (slot_blk % a.blocks_per_group) * kRows + e;
-                if (e < rows_valid) {
+                    static_cast<unsigned long long>(s_tokmask[mh]) | (static_cast<unsigned long long>(s_tokmask[mh + 1]) << 32);
+                if (ch_valid) {
                     float4* gp = reinterpret_cast<float4*>(a.gate + static_cast<size_t>(ch) * a.NT);
                     float4* up = reinterpret_cast<float4*>(a.up + static_cast<size_t>(ch) * a.NT);
                     for (int b0 = 0; b0 < nb4; b0 += kB4) {
@@ -414,7 +441,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
     __shared__ int s_union[WIDE_MAX_GROUPS];
     __shared__ int s_nunion;
     __shared__ int s_flag;
-    __shared__ unsigned s_tokmask[2];
+    __shared__ unsigned s_tokmask[4];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kRingBytesD);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStagesD + 4);
@@ -576,6 +603,7 @@ int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a
     a.words = (a.NG + 31) / 32;
     a.rows_valid = G < kRows ? G : kRows;
     a.blocks_per_group = G / kRows > 0 ? G / kRows : 1;
+    a.gpb = G < kRows ? kRows / G : 1;
     a.row_tiles = (D + kRows - 1) / kRows;
     a.mask_bits = mask_bits;
     a.act_in = static_cast<const __nv_bfloat16*>(x_or_a);
