@@ -253,7 +253,8 @@ def run_ours(args):
         if qproj:
             binding.wide_qproj(ctx, x_in, w["w_q"], cfg.group, meta, y=y_out)
         elif oproj:
-            binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out)
+            binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out,
+                               flags=binding.FLAG_INPUT_MASKED if args.premasked else 0)
         else:
             binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out)
     calls = {"n": 0}
@@ -319,6 +320,12 @@ def run_ours(args):
         step()
     if ctx.status() != 0:
         raise RuntimeError("device status word set during warm-up")
+    if args.premasked and args.op == "oproj":
+        # the attention output as wide_attn leaves it: zeros for inactive (token, group) pairs
+        # (x and hence the mask are the same in every step)
+        m = (bits.view(torch.int32)[:, :, None] >> torch.arange(32, device=dev, dtype=torch.int32)) & 1
+        m = m.reshape(T, -1)[:, :NG].to(torch.bfloat16).repeat_interleave(cfg.group, dim=1)
+        d["attn_out"] = (d["attn_out"] * m).contiguous()
     run_step = rotating(lambda c: step(copy=c))
     for _ in range(n_copies):
         run_step()
@@ -692,6 +699,8 @@ def main():
     ap.add_argument("--group", type=int, default=0)
     ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn", "qproj"],
                     help="oproj, qproj and attn need a workload with an attention half")
+    ap.add_argument("--premasked", action="store_true",
+                    help="oproj: feed an attention output that already has zeros for inactive pairs")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")

@@ -75,6 +75,9 @@ extern "C" {
 #define WIDE_FLAG_SIMT 1u        /* use the plain CUDA-core kernels (any shape; the only path for fp32) */
 #define WIDE_FLAG_FORCE_PREFILL 2u /* tokens <= WIDE_DECODE_MAX_TOKENS would normally take the decode path */
 #define WIDE_FLAG_FORCE_DECODE 4u  /* take the union-streaming decode path (tokens <= WIDE_DECODE_MAX_TOKENS) */
+#define WIDE_FLAG_INPUT_MASKED 8u  /* wide_oproj: attn_out already holds exact zeros for every inactive
+                                      (token, group) pair, as wide_attn writes it; the prefill path then
+                                      skips its masking pass (and the token clustering that rides on it) */
 
 #define WIDE_DECODE_MAX_TOKENS 64
 #define WIDE_MAX_GROUPS 256
@@ -231,6 +234,8 @@ WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_
  * a = attention output flattened head-major [tokens, attn_dim], group g = channels [gG, (g+1)G).
  *   perm, counts: reserved (the current kernels do not read them; may be NULL).
  *   token_order, token_rank as for wide_ffn.
+ *   WIDE_FLAG_INPUT_MASKED: see the flag; with an input that is not masked the result is the
+ *       dense product for every token tile that uses the group at all.
  */
 WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
                int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,

@@ -299,7 +299,8 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
                                           out_dtype);
         case PATH_PREFILL_TC:
             return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits,
-                                                token_order, token_rank, y, out_dtype, workspace);
+                                                token_order, token_rank, y, out_dtype, workspace,
+                                                (flags & WIDE_FLAG_INPUT_MASKED) != 0);
         default:
             return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
                                                out_dtype, workspace);

@@ -105,7 +105,8 @@ int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const vo
 // `a_masked` is scratch [T, K] bf16.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                  int D, int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
-                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked);
+                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked,
+                                 bool input_masked);
 
 // tcgen05 decode path (bf16, T <= WIDE_DECODE_MAX_TOKENS).
 size_t wide_decode_workspace(int T, int D, int inner);

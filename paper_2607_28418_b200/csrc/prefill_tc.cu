@@ -1028,8 +1028,11 @@ int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const
 
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T, int D,
                                  int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
-                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked) {
+                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked,
+                                 bool input_masked) {
     if (T == 0) return WIDE_OK;
+    // an input that already has zeros for the inactive pairs is the GEMM operand as it stands
+    if (input_masked) return launch_down_auto(ctx, s, a, wo, mask_bits, T, D, K, G, y, out_dtype, nullptr);
     const int words = (K / G + 31) / 32;
     const long long total = static_cast<long long>(T) * (K / 8);
     long long blocks = (total + 255) / 256;

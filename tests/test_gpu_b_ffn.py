@@ -211,6 +211,20 @@ def test_oproj_prefill_tc(ctx, T, D, K, G, k):
     assert_close(y, ref, f"oproj prefill {T}x{D}x{K} G{G}")
 
 
+def test_oproj_prefill_with_an_input_that_is_already_masked(ctx):
+    """The output of wide_attn has zeros for inactive pairs; the O-projection then needs no masking pass."""
+    from paper_2607_28418_b200 import binding
+    T, D, K, G, k = 700, 512, 1024, 128, 3
+    rng = np.random.default_rng(8)
+    a = synth.make_activations(rng, T, K, "bf16", "random")
+    w_o = synth.make_weight(rng, D, K, 0.02, "bf16")
+    mask = synth.random_mask(9, T, K // G, k)
+    a_masked = (a * wo.expand_group_mask(mask, G)).astype(np.float32)
+    y = binding.wide_oproj(ctx, to_dev(a_masked, "bf16"), to_dev(w_o, "bf16"), G, bits_to_dev(wo.pack_mask_bits(mask)),
+                           meta_to_dev(wo.reorder(mask, 128)), flags=binding.FLAG_INPUT_MASKED)
+    assert_close(y, wo.oproj(a, w_o, mask, G), "oproj, masked input")
+
+
 @pytest.mark.parametrize("B", [1, 32])
 def test_oproj_decode(ctx, B):
     from paper_2607_28418_b200 import binding
