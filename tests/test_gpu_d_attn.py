@@ -116,3 +116,36 @@ def test_qproj_closed_cases(ctx):
     assert (y0 == 0).all().item()
     with pytest.raises(binding.WideError):
         binding.wide_qproj(ctx, xd, wd, 64, meta_to_dev(wo.reorder(np.ones((T, n_out // 64), dtype=bool), 128)))
+
+
+# ----------------------------------------------------------------------------- the attention half as a chain
+def test_attention_half_chain_stage_by_stage(ctx):
+    """route -> reorder -> routed Q projection -> masked attention -> O-projection on its already
+    masked input.  Every stage is compared with the oracle applied to what the stage received."""
+    from paper_2607_28418_b200 import binding
+    from tests.gpu_util import bits_to_host
+    T, D, H, hd, hpg = 640, 1024, 8, 128, 2
+    NG, G = H // hpg, hpg * hd
+    rng = np.random.default_rng(31)
+    x = synth.make_activations(rng, T, D, "bf16", "random")
+    w_r = synth.make_weight(rng, NG, D, 1.0 / np.sqrt(D), "bf16")
+    w_q = synth.make_weight(rng, H * hd, D, 1.0 / np.sqrt(D), "bf16")     # unit-variance queries
+    w_o = synth.make_weight(rng, D, H * hd, 0.02, "bf16")
+    kv = synth.make_attn_case(32, T, T, H, H, hd)
+    xd = to_dev(x, "bf16")
+    bits, _ = binding.wide_route(ctx, xd, to_dev(w_r, "bf16"), NG, 2)
+    mask = wo.mask_topk(wo.route_scores(x, w_r), 2)
+    assert (bits_to_host(bits) == wo.pack_mask_bits(mask)).all()
+    meta = binding.wide_reorder(ctx, bits, NG, 128)
+    assert (meta["perm"].cpu().numpy() == wo.reorder(mask, 128)["perm"]).all()
+    q = binding.wide_qproj(ctx, xd, to_dev(w_q, "bf16"), G, meta)
+    assert_close(q, wo.qproj(x, w_q, mask, G), "chain: qproj")
+    q_host = q.float().cpu().numpy()
+    o = binding.wide_attn(ctx, q, to_dev(kv["k"].reshape(T, -1), "bf16"), to_dev(kv["v"].reshape(T, -1), "bf16"), H, H, hpg, meta)
+    ref_o = wo.masked_attention(q_host.reshape(T, H, hd), kv["k"], kv["v"], mask, hpg)
+    assert_close(o.reshape(T, H, hd), ref_o, "chain: attention")
+    o_host = o.float().cpu().numpy()
+    y = binding.wide_oproj(ctx, o, to_dev(w_o, "bf16"), G, bits, meta, flags=binding.FLAG_INPUT_MASKED)
+    assert_close(y, wo.oproj(o_host, w_o, mask, G), "chain: oproj")
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
