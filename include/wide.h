@@ -244,8 +244,8 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
                size_t workspace_bytes, unsigned flags);
 
 /*
- * wide_attn -- Eq. 1 under the head-group mask, prefill form of Algorithm 4.  For every active
- * pair (token t, routing group g) and every query head h of g:
+ * wide_attn -- Eq. 1 under the head-group mask, Algorithm 4.  For every active pair (token t,
+ * routing group g) and every query head h of g:
  *     o[t, h, :] = sum_j softmax_j(scale * q[t, h, :] . k[j, h_kv, :]) v[j, h_kv, :]
  * over the keys j <= t + (tokens_k - tokens_q) when causal != 0, over all keys otherwise;
  * h_kv = h / (n_q_heads / n_kv_heads), routing group g = h / heads_per_group.  Inactive pairs,
@@ -253,10 +253,17 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
  *
  *   q   [tokens_q, n_q_heads * head_dim]  bf16, head-major (one sequence; tokens are positions)
  *   k,v [tokens_k, n_kv_heads * head_dim] bf16
- *   perm [n_groups, tokens_q], counts [n_groups]: outputs of wide_reorder for the attention mask
- *       [tokens_q, n_groups], n_groups = n_q_heads / heads_per_group <= WIDE_MAX_GROUPS
+ *   mask_bits [tokens_q, W]: the attention mask, n_groups = n_q_heads / heads_per_group
+ *       <= WIDE_MAX_GROUPS.  Read by the decode form only; may be NULL (prefill form then).
+ *   perm [n_groups, tokens_q], counts [n_groups]: outputs of wide_reorder for that mask.  Read by
+ *       the prefill form only; may be NULL when the decode form runs.
  *   scale: multiplies the logits (<= 0 selects 1/sqrt(head_dim))
  *   o   out [tokens_q, n_q_heads * head_dim] bf16, fully overwritten
+ * Prefill form (tcgen05): query tiles gathered through perm.  Decode form (the last paragraph of
+ * the paper's attention section: reordering bypassed, routing checked per block, online softmax
+ * split over the keys): taken when mask_bits is given and tokens_q * (n_q_heads / n_kv_heads) <= 8;
+ * K and V of a KV head none of whose query rows is active are not read.  WIDE_FLAG_FORCE_PREFILL /
+ * WIDE_FLAG_FORCE_DECODE override the choice.
  * All device pointers, 16-byte aligned, owned by the caller; nothing is allocated; work is
  * enqueued on `stream`.  Needs dtype bf16, head_dim 64 or 128, n_q_heads % n_kv_heads == 0,
  * n_q_heads % heads_per_group == 0.
@@ -265,8 +272,8 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
  */
 WIDE_API int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const void* v, int dtype,
               int tokens_q, int tokens_k, int n_q_heads, int n_kv_heads, int head_dim,
-              int heads_per_group, const int32_t* perm, const int32_t* counts, int causal, float scale,
-              void* o, unsigned flags);
+              int heads_per_group, const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
+              int causal, float scale, void* o, unsigned flags);
 
 /*
  * wide_qproj -- the query projection under the head-group mask (Section 3.1: only the active head

@@ -75,7 +75,8 @@ def load_library() -> ctypes.CDLL:
                                _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                _c_void_p, _c_size_t, _c_uint]
     lib.wide_attn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
-                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_int, ctypes.c_float, _c_void_p, _c_uint]
+                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_int, ctypes.c_float,
+                              _c_void_p, _c_uint]
     lib.wide_qproj.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_int,
                                _c_void_p, _c_void_p, _c_void_p, _c_uint]
     lib.wide_unpermute.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
@@ -308,16 +309,18 @@ def wide_oproj(ctx: Context, attn_out: torch.Tensor, w_o: torch.Tensor, group: i
 
 
 def wide_attn(ctx: Context, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, n_q_heads: int, n_kv_heads: int,
-              heads_per_group: int, meta: Dict[str, torch.Tensor], causal: bool = True, scale: float = 0.0,
-              flags: int = 0, o: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """q [T_q, H_q*d], k/v [T_k, H_kv*d] bf16; meta = wide_reorder outputs of the attention mask."""
+              heads_per_group: int, meta: Optional[Dict[str, torch.Tensor]], causal: bool = True, scale: float = 0.0,
+              flags: int = 0, o: Optional[torch.Tensor] = None, mask_bits: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [T_q, H_q*d], k/v [T_k, H_kv*d] bf16; meta = wide_reorder outputs of the attention mask
+    (prefill form), mask_bits = the mask itself (decode form, a handful of query tokens)."""
     Tq, Tk = q.shape[0], k.shape[0]
     head_dim = q.shape[1] // n_q_heads
     if o is None:
         o = torch.empty_like(q)
+    m = meta or {}
     rc = ctx.lib.wide_attn(ctx.handle, _stream(), _ptr(q), _ptr(k), _ptr(v), _dtype_code(q), Tq, Tk, n_q_heads,
-                           n_kv_heads, head_dim, heads_per_group, _ptr(meta["perm"]), _ptr(meta["counts"]),
-                           1 if causal else 0, float(scale), _ptr(o), flags)
+                           n_kv_heads, head_dim, heads_per_group, _ptr(mask_bits), _ptr(m.get("perm")),
+                           _ptr(m.get("counts")), 1 if causal else 0, float(scale), _ptr(o), flags)
     _check(rc, "wide_attn")
     return o
 

@@ -81,11 +81,15 @@ int wide_create(wide_ctx** out, int device) {
         return WIDE_ERR_CUDA;
     }
     ctx->d_tickets = nullptr;
-    if (cudaMalloc(&ctx->decode_acc, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess ||
+    ctx->attn_part = nullptr;
+    ctx->attn_part_bytes = 4u << 20;
+    if (cudaMalloc(&ctx->attn_part, ctx->attn_part_bytes) != cudaSuccess ||
+        cudaMalloc(&ctx->decode_acc, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess ||
         cudaMalloc(&ctx->d_tickets, 2048 * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->d_tickets, 0, 2048 * sizeof(unsigned)) != cudaSuccess ||
         cudaMemset(ctx->d_status, 0, 16 * sizeof(int)) != cudaSuccess ||
         cudaMemset(ctx->decode_acc, 0, ctx->decode_acc_floats * sizeof(float)) != cudaSuccess) {
+        cudaFree(ctx->attn_part);
         cudaFree(ctx->decode_acc);
         cudaFree(ctx->d_tickets);
         cudaFree(ctx->d_status);
@@ -162,6 +166,7 @@ int wide_launch_count(wide_ctx* ctx, unsigned long long* count) {
 int wide_destroy(wide_ctx* ctx) {
     if (!ctx) return WIDE_ERR_INVALID_ARG;
     free_profile(ctx);
+    cudaFree(ctx->attn_part);
     cudaFree(ctx->d_tickets);
     cudaFree(ctx->decode_acc);
     cudaFree(ctx->d_status);
@@ -309,20 +314,32 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
 
 int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const void* v, int dtype, int tokens_q,
               int tokens_k, int n_q_heads, int n_kv_heads, int head_dim, int heads_per_group,
-              const int32_t* perm, const int32_t* counts, int causal, float scale, void* o, unsigned flags) {
-    (void)flags;
-    if (!ctx || !q || !k || !v || !perm || !counts || !o) return WIDE_ERR_INVALID_ARG;
+              const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts, int causal, float scale, void* o,
+              unsigned flags) {
+    if (!ctx || !q || !k || !v || !o) return WIDE_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return WIDE_ERR_INVALID_ARG;
     if (tokens_q < 0 || tokens_k <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || heads_per_group <= 0)
         return WIDE_ERR_INVALID_ARG;
     if (n_q_heads % n_kv_heads != 0 || n_q_heads % heads_per_group != 0) return WIDE_ERR_INVALID_ARG;
-    if (dtype != WIDE_BF16 || (head_dim != 64 && head_dim != 128) || !ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (dtype != WIDE_BF16 || (head_dim != 64 && head_dim != 128)) return WIDE_ERR_UNSUPPORTED_SHAPE;
     if (n_q_heads / heads_per_group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
     if (!wide_aligned16(q) || !wide_aligned16(k) || !wide_aligned16(v) || !wide_aligned16(o)) return WIDE_ERR_ALIGNMENT;
     if (tokens_q == 0) return WIDE_OK;
     if (!(scale > 0.f)) scale = 1.0f / sqrtf(static_cast<float>(head_dim));
-    return wide_launch_attn_prefill_tc(ctx, static_cast<cudaStream_t>(stream), q, k, v, tokens_q, tokens_k, n_q_heads,
-                                       n_kv_heads, head_dim, heads_per_group, perm, counts, causal ? 1 : 0, scale, o);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // a handful of query rows per KV head: the split-key decode form, straight from the mask
+    const bool decode = mask_bits && !(flags & WIDE_FLAG_FORCE_PREFILL) &&
+                        wide_attn_decode_fits(tokens_q, n_q_heads, n_kv_heads);
+    if (decode || (flags & WIDE_FLAG_FORCE_DECODE)) {
+        if (!mask_bits) return WIDE_ERR_INVALID_ARG;
+        if (!wide_attn_decode_fits(tokens_q, n_q_heads, n_kv_heads)) return WIDE_ERR_UNSUPPORTED_SHAPE;
+        return wide_launch_attn_decode(ctx, s, q, k, v, mask_bits, tokens_q, tokens_k, n_q_heads, n_kv_heads, head_dim,
+                                       heads_per_group, causal ? 1 : 0, scale, o);
+    }
+    if (!perm || !counts) return WIDE_ERR_INVALID_ARG;
+    if (!ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    return wide_launch_attn_prefill_tc(ctx, s, q, k, v, tokens_q, tokens_k, n_q_heads, n_kv_heads, head_dim,
+                                       heads_per_group, perm, counts, causal ? 1 : 0, scale, o);
 }
 
 int wide_qproj(wide_ctx* ctx, void* stream, const void* x, const void* w, int dtype, int tokens, int hidden,

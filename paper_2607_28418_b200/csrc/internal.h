@@ -22,6 +22,8 @@ struct wide_ctx {
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
     unsigned* d_tickets;    // 2048 completion counters of the decode path; zero between calls
+    float* attn_part;       // partial (m, l, O) of the key slices of the decode attention
+    size_t attn_part_bytes;
     unsigned long long wait_ns;  // bound of every device-side wait
     void* encode_tiled;     // cuTensorMapEncodeTiled, resolved through the runtime
     unsigned long long launches;  // kernels launched by the library so far
@@ -129,3 +131,10 @@ int wide_launch_attn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* q, co
 // tcgen05 routed linear layer (GEMM-MN, bf16): y [T, Nout] bf16, zeros for inactive (token, group) pairs.
 int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w, int T, int D, int Nout,
                              int G, const int32_t* perm, const int32_t* counts, void* y);
+
+// Decode form of the masked attention (CUDA cores, split over the keys); needs
+// tokens_q * (n_q_heads / n_kv_heads) <= 8 (wide_attn_decode_fits).
+bool wide_attn_decode_fits(int Tq, int Hq, int Hkv);
+int wide_launch_attn_decode(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, const void* v,
+                            const uint32_t* mask_bits, int Tq, int Tk, int Hq, int Hkv, int head_dim, int hpg,
+                            int causal, float scale, void* o);

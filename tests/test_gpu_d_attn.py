@@ -149,3 +149,46 @@ def test_attention_half_chain_stage_by_stage(ctx):
     assert_close(y, wo.oproj(o_host, w_o, mask, G), "chain: oproj")
     torch.cuda.synchronize()
     assert ctx.status() == 0
+
+
+# ----------------------------------------------------------------------------- decode form (split over the keys)
+@pytest.mark.parametrize("t_q,t_k,h_q,h_kv,d,hpg", [
+    (1, 1000, 8, 8, 128, 2),       # one new token, MHA
+    (1, 4097, 32, 8, 128, 4),      # GQA 4:1, ragged key count
+    (2, 300, 8, 2, 64, 4),         # two tokens, head_dim 64
+    (4, 515, 4, 4, 128, 1),        # four tokens (speculative block), every head its own group
+    (1, 17, 2, 2, 128, 1),         # fewer keys than one chunk
+])
+@pytest.mark.parametrize("causal", [True, False])
+def test_attn_decode_matches_oracle(ctx, t_q, t_k, h_q, h_kv, d, hpg, causal):
+    from paper_2607_28418_b200 import binding
+    case = synth.make_attn_case(21, t_q, t_k, h_q, h_kv, d)
+    mask = synth.bernoulli_mask(22 + t_k, t_q, h_q // hpg, 0.5)
+    mask[0, 0] = True
+    o = binding.wide_attn(ctx, to_dev(case["q"].reshape(t_q, -1), "bf16"), to_dev(case["k"].reshape(t_k, -1), "bf16"),
+                          to_dev(case["v"].reshape(t_k, -1), "bf16"), h_q, h_kv, hpg, None, causal=causal,
+                          mask_bits=bits_to_dev(wo.pack_mask_bits(mask)))
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg, causal=causal)
+    got = o.reshape(t_q, h_q, d)
+    assert (got.float().cpu().numpy()[~np.repeat(mask, hpg, axis=1)] == 0.0).all()
+    assert_close(got, ref, "attn decode")
+
+
+def test_attn_decode_and_prefill_forms_agree(ctx):
+    from paper_2607_28418_b200 import binding
+    t_q, t_k, h_q, h_kv, d, hpg = 2, 700, 8, 4, 128, 2
+    case = synth.make_attn_case(23, t_q, t_k, h_q, h_kv, d)
+    mask = synth.bernoulli_mask(24, t_q, h_q // hpg, 0.6)
+    bits = bits_to_dev(wo.pack_mask_bits(mask))
+    meta = meta_to_dev(wo.reorder(mask, 128))
+    args = (to_dev(case["q"].reshape(t_q, -1), "bf16"), to_dev(case["k"].reshape(t_k, -1), "bf16"),
+            to_dev(case["v"].reshape(t_k, -1), "bf16"), h_q, h_kv, hpg)
+    a = binding.wide_attn(ctx, *args, meta, mask_bits=bits)                                    # decode form
+    b = binding.wide_attn(ctx, *args, meta, mask_bits=bits, flags=binding.FLAG_FORCE_PREFILL)  # tcgen05 form
+    ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg)
+    assert_close(a.reshape(t_q, h_q, d), ref, "decode form")
+    assert_close(b.reshape(t_q, h_q, d), ref, "prefill form")
+    with pytest.raises(binding.WideError):
+        binding.wide_attn(ctx, *args, None)                                                    # neither mask nor metadata
