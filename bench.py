@@ -527,9 +527,11 @@ def run_attn(args):
     H = cfg.attn_dim // hd
     hpg = cfg.attn_group // hd
     NG, k = cfg.attn_n_groups, cfg.attn_k
+    decode = T <= 8                       # --batch B: B new tokens against a resident K/V cache
+    Tk = args.kv_len if args.kv_len else (synth.CONFIGS[args.workload].tokens if decode else T)
     oc = synth.make_oproj_case(cfg, 1000 * rank)
-    ac = synth.make_attn_case(1000 * rank, T, T, H, H, hd)
-    host = {"x": oc["x"], "q": ac["q"].reshape(T, H * hd), "k": ac["k"].reshape(T, H * hd), "v": ac["v"].reshape(T, H * hd)}
+    ac = synth.make_attn_case(1000 * rank, T, Tk, H, H, hd)
+    host = {"x": oc["x"], "q": ac["q"].reshape(T, H * hd), "k": ac["k"].reshape(Tk, H * hd), "v": ac["v"].reshape(Tk, H * hd)}
     w_router = to_dev(oc["w_router_attn"], "bf16")
     pinned = {n: torch.from_numpy(synth.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).pin_memory() for n, a in host.items()}
     bufs = [{n: t.to(dev) for n, t in pinned.items()} for _ in range(2)]
@@ -540,11 +542,13 @@ def run_attn(args):
 
     def attn_only(slot=0):
         b = bufs[slot]
-        binding.wide_attn(ctx, b["q"], b["k"], b["v"], H, H, hpg, state["meta"], causal=True, o=obuf[slot])
+        binding.wide_attn(ctx, b["q"], b["k"], b["v"], H, H, hpg, state["meta"], causal=True, o=obuf[slot],
+                          mask_bits=bits if decode else None)
 
     def step(slot=0, kk=k):
         binding.wide_route(ctx, bufs[slot]["x"], w_router, NG, kk, mask_bits=bits)
-        state["meta"] = binding.wide_reorder(ctx, bits, NG, 128, out=state["meta"])
+        if not decode:
+            state["meta"] = binding.wide_reorder(ctx, bits, NG, 128, out=state["meta"])
         attn_only(slot)
 
     def sync_all():
@@ -611,6 +615,8 @@ def run_attn(args):
                 if i >= 2:
                     s_in.wait_event(ev["run"][b])
                 for n in pinned:
+                    if decode and n in ("k", "v"):
+                        continue                        # the K/V cache is resident; only the new tokens travel
                     bufs[b][n].copy_(pinned[n], non_blocking=True)
                 ev["in"][b].record()
             with torch.cuda.stream(s_run):
@@ -644,8 +650,19 @@ def run_attn(args):
     if rank == 0:
         # algorithmic FLOPs: every active (token t, head) pair does 4 * d * (t + 1) (QK^T and PV over its keys)
         mask = np.unpackbits(bits.cpu().numpy().view(np.uint8), axis=1, bitorder="little")[:, :NG].astype(bool)
-        flops = float((mask.sum(axis=1) * hpg * 4.0 * hd * (np.arange(T) + 1.0)).sum())
+        flops = float((mask.sum(axis=1) * hpg * 4.0 * hd * (np.arange(T) + 1.0 + (Tk - T))).sum())
         ach = flops / (attn_ms * 1e-3) / 1e12
+        if decode:
+            # algorithmic bytes: K and V rows of every KV head some active query row reads
+            heads_read = int(np.repeat(mask.any(axis=0), hpg).sum())
+            kv_bytes = 2.0 * heads_read * Tk * hd * 2
+            roof = {"kernel": "attn_decode", "bound": "hbm", "achieved": kv_bytes / (attn_ms * 1e-3) / 1e9,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "traffic": None, "peak_source": peaks["source"], "kv_heads_read": heads_read}
+        else:
+            roof = {"kernel": "attn_prefill", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                    "traffic": NCU_TRAFFIC_BYTES.get(("attn_prefill", cfg.name)), "peak_source": peaks["source"]}
         kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
                        "share": round(v["total_ms"] / max(sum(p["total_ms"] for p in prof.values()), 1e-9), 4)}
                    for n, v in prof.items()}
@@ -653,18 +670,16 @@ def run_attn(args):
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "op": "attn", "tokens_per_gpu": T, "heads": H, "head_dim": hd,
+            "config": {"workload": cfg.name, "op": "attn", "tokens_per_gpu": T, "keys": Tk, "heads": H, "head_dim": hd,
                        "heads_per_group": hpg, "n_groups": NG, "k": k, "causal": True, "router": cfg.router,
                        "parallelism": f"sequence-sharded x{world} (independent sequences), no collective",
-                       "l2": "q, k, v, o of one step are %.0f MB (larger than L2)" % (4 * T * H * hd * 2 / 1e6)},
+                       "l2": "q, k, v, o of one step are %.0f MB (larger than L2)" % ((2 * T + 2 * Tk) * H * hd * 2 / 1e6)},
             "e2e": {"value": aggregate(T, e2e_steps, ms_e2e, world), "unit": "tokens/s",
-                    "h2d_bytes_per_step": sum(t.numel() * 2 for t in pinned.values()),
+                    "h2d_bytes_per_step": sum(t.numel() * 2 for n, t in pinned.items() if not (decode and n in ("k", "v"))),
                     "d2h_bytes_per_step": o_host[0].numel() * 2},
             "launch": "one CUDA graph replay per step" if not args.no_graph else "direct launches",
             "gpu_launches": int(launches), "clocks": clocks,
-            "roofline": {"kernel": "attn_prefill", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                         "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                         "traffic": NCU_TRAFFIC_BYTES.get(("attn_prefill", cfg.name)), "peak_source": peaks["source"]},
+            "roofline": roof,
             "kernels": kernels,
             "attn": {"graph_ms": attn_ms, "active_gflop": flops / 1e9},
             "dense": {"ms_per_step": dense_ms, "speedup_vs_dense": (dense_ms / (ms_total / args.steps)) if dense_ms else None,
@@ -675,7 +690,8 @@ def run_attn(args):
             t0 = time.perf_counter()
             m_s = mask[:sample]
             from oracle import wide_oracle as wo
-            wo.masked_attention(ac["q"][:sample], ac["k"][:sample], ac["v"][:sample], m_s, hpg)
+            ks = Tk if decode else sample
+            wo.masked_attention(ac["q"][:sample], ac["k"][:ks], ac["v"][:ks], m_s, hpg)
             dt = time.perf_counter() - t0
             line["cpu_baseline"] = {"value": sample / dt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
                                     "sample": f"first {sample} of {T} positions, masked attention only, fp64 numpy ({dt:.1f} s)"}
@@ -701,6 +717,7 @@ def main():
                     help="oproj, qproj and attn need a workload with an attention half")
     ap.add_argument("--premasked", action="store_true",
                     help="oproj: feed an attention output that already has zeros for inactive pairs")
+    ap.add_argument("--kv-len", type=int, default=0, help="attn: number of keys (default: the workload's tokens)")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")

@@ -29,7 +29,7 @@ __device__ __forceinline__ float exp2_fast(float x) {
     return y;
 }
 
-template <int HD>
+template <int HD, int RT>   // RT: compile-time bound of the rows served (1, 2, 4 or 8)
 __global__ void __launch_bounds__(32 * kDecWarps)
 attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, const uint32_t* __restrict__ mask_bits, int words, int Tq,
@@ -37,10 +37,10 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
                    float* __restrict__ part) {
     constexpr int kDL = HD / 32;                  // output dimensions per lane
     constexpr int kVec = HD / 8;                  // 16-byte pieces of a key row
-    __shared__ float qs[kMaxRows][HD];
-    __shared__ float ps[kDecWarps][kMaxRows][32];
-    __shared__ float wm[kDecWarps][kMaxRows], wl[kDecWarps][kMaxRows];
-    __shared__ float wo[kDecWarps][kMaxRows][HD];
+    __shared__ float qs[RT][HD];
+    __shared__ float ps[kDecWarps][RT][32];
+    __shared__ float wm[kDecWarps][RT], wl[kDecWarps][RT];
+    __shared__ float wo[kDecWarps][RT][HD];
     __shared__ int s_any;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int split = blockIdx.x, hkv = blockIdx.y;
@@ -67,9 +67,9 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     __syncthreads();
 
     const int j0 = split * keys_per_split, j1 = min(Tk, j0 + keys_per_split);
-    float m[kMaxRows], l[kMaxRows], o[kMaxRows][kDL];
+    float m[RT], l[RT], o[RT][kDL];
 #pragma unroll
-    for (int r = 0; r < kMaxRows; ++r) {
+    for (int r = 0; r < RT; ++r) {
         m[r] = -CUDART_INF_F;
         l[r] = 0.f;
 #pragma unroll
@@ -84,9 +84,9 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
         const uint4* kp = reinterpret_cast<const uint4*>(k + static_cast<size_t>(valid ? j : j1 - 1) * ldk + static_cast<size_t>(hkv) * HD);
 #pragma unroll
         for (int i = 0; i < kVec; ++i) kr[i] = __ldg(kp + i);
-        float s[kMaxRows];
+        float s[RT];
 #pragma unroll
-        for (int r = 0; r < kMaxRows; ++r) {
+        for (int r = 0; r < RT; ++r) {
             s[r] = -CUDART_INF_F;
             if (r < R) {
                 float a = 0.f;
@@ -106,7 +106,7 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
         }
         // online softmax per row across the 32 keys of the chunk
 #pragma unroll
-        for (int r = 0; r < kMaxRows; ++r) {
+        for (int r = 0; r < RT; ++r) {
             if (r < R) {
                 float mx = s[r];
 #pragma unroll
@@ -126,28 +126,35 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
             }
         }
         __syncwarp();
-        // PV: the warp reads each V row of the chunk once, lane = kDL output dimensions
+        // PV: the warp reads each V row of the chunk once, lane = kDL output dimensions.  The rows
+        // are fetched in batches of kVB loads per lane before any is used (this phase is bound by
+        // load latency, not by instructions).
         const int nk = min(32, j1 - c0);
-#pragma unroll 4
-        for (int kk = 0; kk < nk; ++kk) {
-            const __nv_bfloat16* vp = v + static_cast<size_t>(c0 + kk) * ldk + static_cast<size_t>(hkv) * HD + lane * kDL;
-            float vv[kDL];
-            if (kDL == 4) {
-                const uint2 raw = __ldg(reinterpret_cast<const uint2*>(vp));
-                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                vv[0] = a.x; vv[1] = a.y; vv[kDL - 2] = b.x; vv[kDL - 1] = b.y;
-            } else {
-                const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(vp));
-                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw));
-                vv[0] = a.x; vv[1] = a.y;
+        constexpr int kVB = RT <= 2 ? 16 : 8;
+        for (int k0 = 0; k0 < nk; k0 += kVB) {
+            uint2 raw[kVB];
+#pragma unroll
+            for (int u = 0; u < kVB; ++u) {
+                const int kk = min(k0 + u, nk - 1);
+                const __nv_bfloat16* vp = v + static_cast<size_t>(c0 + kk) * ldk + static_cast<size_t>(hkv) * HD + lane * kDL;
+                if (kDL == 4) raw[u] = __ldg(reinterpret_cast<const uint2*>(vp));
+                else raw[u] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(vp)), 0u);
             }
 #pragma unroll
-            for (int r = 0; r < kMaxRows; ++r) {
-                if (r < R) {
-                    const float p = ps[warp][r][kk];
+            for (int u = 0; u < kVB; ++u) {
+                if (k0 + u < nk) {
+                    float vv[4];
+                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw[u].x));
+                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw[u].y));
+                    vv[0] = a.x; vv[1] = a.y; vv[2] = b.x; vv[3] = b.y;
 #pragma unroll
-                    for (int d = 0; d < kDL; ++d) o[r][d] = fmaf(p, vv[d], o[r][d]);
+                    for (int r = 0; r < RT; ++r) {
+                        if (r < R) {
+                            const float p = ps[warp][r][k0 + u];
+#pragma unroll
+                            for (int d = 0; d < kDL; ++d) o[r][d] = fmaf(p, vv[d], o[r][d]);
+                        }
+                    }
                 }
             }
         }
@@ -156,7 +163,7 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
     // merge the four warps, write this key slice's partial result
 #pragma unroll
-    for (int r = 0; r < kMaxRows; ++r) {
+    for (int r = 0; r < RT; ++r) {
         if (r < R) {
             if (lane == 0) { wm[warp][r] = m[r]; wl[warp][r] = l[r]; }
 #pragma unroll
@@ -218,8 +225,9 @@ int launch_attn_decode(wide_ctx* ctx, cudaStream_t s, const void* q, const void*
                        void* o) {
     const int rep = Hq / Hkv, R = Tq * rep;
     const int words = (Hq / hpg + 31) / 32;
-    // enough key slices to fill the GPU twice, at least 128 keys each, and the scratch slab must hold them
-    int n_splits = (2 * ctx->sm_count + Hkv - 1) / Hkv;
+    // enough key slices for about eight resident CTAs per SM (the kernel hides its load latency by
+    // occupancy), at least 128 keys each, and the scratch slab must hold them
+    int n_splits = (8 * ctx->sm_count + Hkv - 1) / Hkv;
     if (n_splits > (Tk + 127) / 128) n_splits = (Tk + 127) / 128;
     if (n_splits > kMaxSplits) n_splits = kMaxSplits;
     const size_t per_split = static_cast<size_t>(Hkv) * R * (HD + 2) * sizeof(float);
@@ -229,9 +237,18 @@ int launch_attn_decode(wide_ctx* ctx, cudaStream_t s, const void* q, const void*
     n_splits = (Tk + kps - 1) / kps;
     {
         WideLaunch l(ctx, s, "attn_decode");
-        attn_decode_kernel<HD><<<dim3(n_splits, Hkv), 32 * kDecWarps, 0, s>>>(
-            static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
-            mask_bits, words, Tq, Tk, Hq, Hkv, hpg, causal, scale * 1.4426950408889634f, kps, ctx->attn_part);
+        const dim3 grid(n_splits, Hkv);
+        const __nv_bfloat16 *qb = static_cast<const __nv_bfloat16*>(q), *kb = static_cast<const __nv_bfloat16*>(k),
+                            *vb = static_cast<const __nv_bfloat16*>(v);
+        const float sl = scale * 1.4426950408889634f;
+#define WIDE_DEC_CASE(rt) \
+    attn_decode_kernel<HD, rt><<<grid, 32 * kDecWarps, 0, s>>>(qb, kb, vb, mask_bits, words, Tq, Tk, Hq, Hkv, hpg, causal, sl, \
+                                                              kps, ctx->attn_part)
+        if (R <= 1) WIDE_DEC_CASE(1);
+        else if (R <= 2) WIDE_DEC_CASE(2);
+        else if (R <= 4) WIDE_DEC_CASE(4);
+        else WIDE_DEC_CASE(8);
+#undef WIDE_DEC_CASE
     }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     WideLaunch l(ctx, s, "attn_decode_merge");
