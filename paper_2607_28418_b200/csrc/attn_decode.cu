@@ -84,6 +84,19 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
         const uint4* kp = reinterpret_cast<const uint4*>(k + static_cast<size_t>(valid ? j : j1 - 1) * ldk + static_cast<size_t>(hkv) * HD);
 #pragma unroll
         for (int i = 0; i < kVec; ++i) kr[i] = __ldg(kp + i);
+        // with few query rows there are registers to spare: the chunk's V rows are requested now,
+        // together with the key rows, so that a chunk costs one load latency instead of two
+        constexpr bool kEarlyV = RT <= 2;
+        uint2 vr[kEarlyV ? 32 : 1];
+        const int nk = min(32, j1 - c0);
+        if (kEarlyV) {
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+                const __nv_bfloat16* vp = v + static_cast<size_t>(c0 + min(u, nk - 1)) * ldk + static_cast<size_t>(hkv) * HD + lane * kDL;
+                if (kDL == 4) vr[u] = __ldg(reinterpret_cast<const uint2*>(vp));
+                else vr[u] = make_uint2(__ldg(reinterpret_cast<const uint32_t*>(vp)), 0u);
+            }
+        }
         float s[RT];
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
@@ -129,9 +142,27 @@ attn_decode_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
         // PV: the warp reads each V row of the chunk once, lane = kDL output dimensions.  The rows
         // are fetched in batches of kVB loads per lane before any is used (this phase is bound by
         // load latency, not by instructions).
-        const int nk = min(32, j1 - c0);
-        constexpr int kVB = RT <= 2 ? 16 : 8;
-        for (int k0 = 0; k0 < nk; k0 += kVB) {
+        constexpr int kVB = 8;
+        if (kEarlyV) {
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+                if (u < nk) {
+                    float vv[4];
+                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vr[u].x));
+                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vr[u].y));
+                    vv[0] = a.x; vv[1] = a.y; vv[2] = b.x; vv[3] = b.y;
+#pragma unroll
+                    for (int r = 0; r < RT; ++r) {
+                        if (r < R) {
+                            const float p = ps[warp][r][u];
+#pragma unroll
+                            for (int d = 0; d < kDL; ++d) o[r][d] = fmaf(p, vv[d], o[r][d]);
+                        }
+                    }
+                }
+            }
+        }
+        for (int k0 = kEarlyV ? nk : 0; k0 < nk; k0 += kVB) {
             uint2 raw[kVB];
 #pragma unroll
             for (int u = 0; u < kVB; ++u) {
