@@ -6,14 +6,17 @@
  *   wide_reorder    per-group mask reordering + tile predicates   (Section 3.3, Eq. 6-8, Algorithm 1)
  *   wide_ffn        block-skipping SwiGLU FFN                     (Eq. 3; Algorithms 2 and 3)
  *   wide_oproj      head-group-masked attention output projection (Eq. 2; Eq. 10, Algorithm 3)
- *   wide_attn       head-group-masked causal attention, prefill   (Eq. 1; Algorithm 4)
+ *   wide_attn       head-group-masked causal attention            (Eq. 1; Algorithm 4: prefill and decode forms)
  *   wide_qproj      routed query projection, GEMM-MN              (Eq. 1 under the mask; Algorithm 2)
  *   wide_unpermute  the scatter epilogue as a standalone step     (Algorithm 2, epilogue)
  *
  * General rules
  *   - Every data pointer is a DEVICE pointer owned by the caller; the library never
  *     allocates, frees or keeps caller-visible memory.  Scratch memory is passed in as
- *     `workspace` (size from wide_workspace_bytes).
+ *     `workspace` (size from wide_workspace_bytes); a few small buffers (decode accumulators,
+ *     completion counters, the partial results of the decode attention) belong to the context
+ *     and are allocated once by wide_create, which is why one context must not run two calls
+ *     concurrently on different streams.
  *   - All work is enqueued on the caller's stream (`stream` is a cudaStream_t cast to
  *     void*); no call synchronises the host or reads results back, except wide_status.
  *   - Matrices are row-major and contiguous.  Base pointers must be 16-byte aligned.

@@ -1,22 +1,25 @@
-// Prefill path of wide_ffn / wide_oproj on the 5th-generation tensor cores (tcgen05 + TMEM),
-// operands staged by TMA (weights, hidden activation) or gathered with cp.async (token rows
-// selected through the reorder permutation).
+// Prefill path of wide_ffn / wide_oproj / wide_qproj (and the score GEMM of wide_route) on the
+// 5th-generation tensor cores (tcgen05 + TMEM), operands staged by TMA (weights, hidden
+// activation) or gathered with cp.async (token rows selected through the reorder permutation).
 //
-//   gateup_kernel  Algorithm 2 (GEMM-MN, N-axis): one work item = one active (token tile, group)
-//                  pair of the reordered mask.  A = 128 gathered rows of X, B = the group's rows of
-//                  W_gate and W_up side by side (one UMMA of N = 2*BN), fp32 accumulators in TMEM,
-//                  epilogue silu(gate)*up -> bf16, scattered through the permutation straight into
-//                  the token-major hidden activation H (rows past the group's count are dropped);
-//                  the same warps zero the group's inactive rows of H.
-//   down_kernel    Eq. 10 (K-axis) in owner-computes form: a CTA owns a 128-token x BN output tile
-//                  in original token order and walks the K-groups, skipping every group that no
-//                  token of the tile selected (block-level predicate on the unsorted mask);
-//                  inactive (token, group) pairs inside an active block are exact zeros of H.  No
-//                  atomics, deterministic, output written once.
+//   gateup_kernel   Algorithm 2 (GEMM-MN, N-axis): a work item is one or two consecutive 128-row
+//                   tiles of a group's sorted active rows times one block of the group's channels.
+//                   A = gathered rows of X, B = the group's rows of W_gate and W_up side by side
+//                   (one UMMA of N = 2*BN), fp32 accumulators in TMEM, epilogue silu(gate)*up ->
+//                   bf16, scattered through the permutation straight into the token-major hidden
+//                   activation H (rows past the group's count are dropped); the same warps zero
+//                   the group's inactive rows of H.  With kLinear the same kernel is the routed
+//                   linear layer of wide_qproj (one weight, plain store).
+//   down_kernel     Eq. 10 (K-axis) in owner-computes form: a CTA owns a 128-token x BN output tile
+//                   and walks the K-groups, skipping every group that no token of the tile selected
+//                   (block-level predicate on the mask of the tile's tokens); inactive (token,
+//                   group) pairs inside an active block are exact zeros of H.  No atomics,
+//                   deterministic, output written once.  Also the K-split score GEMM of the router.
+//   down256_kernel  the same product with 256-token tiles and column tiles of even widths.
 //
-// Both kernels are persistent (one CTA per SM) and warp-specialised: TMA producer, UMMA issuer,
-// (gather warps,) epilogue warps; a 4-stage shared-memory ring and two TMEM accumulator buffers
-// overlap loads, MMAs and epilogues.  Every mbarrier wait is bounded.
+// All are persistent (at most one CTA per SM) and warp-specialised: TMA producer, UMMA issuer,
+// (gather warps,) epilogue warps over a shared-memory ring; down_kernel double-buffers its TMEM
+// accumulator, the 256-row items of the other two fill TMEM.  Every mbarrier wait is bounded.
 #include <cuda.h>
 
 #include "internal.h"
