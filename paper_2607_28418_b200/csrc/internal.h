@@ -18,7 +18,8 @@ struct wide_ctx {
     int device;
     int sm_count;
     int* d_status;          // [0] device status word (WIDE_OK or WIDE_ERR_TIMEOUT), [1] reorder ticket,
-                            // [4..5] grid-barrier counters of the decode kernel (16 ints in all)
+                            // [4..5] grid-barrier counters of the decode kernel, [8..9] tile queue of the
+                            // 256-row down projection (16 ints in all)
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
     unsigned* d_tickets;    // 2048 completion counters of the decode path; zero between calls

@@ -322,7 +322,8 @@ __global__ void __launch_bounds__(192, 1)
 down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N,
                int K, int G, void* __restrict__ Y,
-               int out_bf16, int n_n, int box_n, int* __restrict__ status, unsigned long long wait_ns) {
+               int out_bf16, int n_n, int box_n, unsigned* __restrict__ queue, int* __restrict__ status,
+               unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStages2 * kStage2Bytes);
@@ -330,6 +331,13 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tfull = smem_u32(bars + 2 * kStages2), tempty = smem_u32(bars + 2 * kStages2 + 1);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages2 + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // Tiles are handed out by a global counter (tiles of a clustered mask differ in how many
+    // groups they skip, so a fixed assignment leaves SMs idle).  The producer warp fetches the next
+    // tile index and passes it to the UMMA warp and the four epilogue warps through a two-slot
+    // ring in shared memory: sq_full[slot] <- producer, sq_empty[slot] <- the five readers.
+    __shared__ int sq_tile[2];
+    __shared__ uint64_t sq_bars[4];
+    const uint32_t sq_full = smem_u32(sq_bars), sq_empty = smem_u32(sq_bars + 2);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
@@ -339,6 +347,10 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         mbar_init(tfull, 1);
         mbar_init(tempty, 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(sq_full + 8 * i, 1);
+            mbar_init(sq_empty + 8 * i, 5);
+        }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -361,6 +373,18 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto col0 = [&](int n) { return 16 * (n * q_base + min(n, q_rem)); };
     auto width = [&](int n) { return 16 * (q_base + (n < q_rem ? 1 : 0)); };
     const uint32_t stage_tx = kA2Bytes + static_cast<uint32_t>(box_n) * (kBK * 2);   // TMA always moves whole boxes
+    // a reader warp takes the tc-th tile of this CTA from the ring (-1: no more tiles, -2: gave up)
+    auto next_tile = [&](int tc) -> int {
+        const int slot = tc & 1;
+        int tile = -2;
+        if (lane == 0) {
+            if (mbar_wait(sq_full + 8 * slot, (tc >> 1) & 1, wait_ns, abort_flag)) {
+                tile = sq_tile[slot];
+                mbar_arrive(sq_empty + 8 * slot);
+            }
+        }
+        return __shfl_sync(0xffffffffu, tile, 0);
+    };
 
     // OR of the mask words of the tile's 256 tokens
     auto tile_mask = [&](int m, uint32_t (&act)[kMaskWords]) {
@@ -375,7 +399,23 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------------ TMA producer
         int it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int tc = 0; ok; ++tc) {
+            // fetch the next tile and publish it (the first one is this CTA's own index)
+            int tile = -1;
+            if (lane == 0) {
+                const int slot = tc & 1;
+                if (!mbar_wait(sq_empty + 8 * slot, ((tc >> 1) & 1) ^ 1u, wait_ns, abort_flag)) {
+                    ok = false;
+                } else {
+                    const unsigned got = tc == 0 ? blockIdx.x : gridDim.x + atomicAdd(queue, 1u);
+                    tile = got < static_cast<unsigned>(n_tiles) ? static_cast<int>(got) : -1;
+                    sq_tile[slot] = tile;
+                    mbar_arrive(sq_full + 8 * slot);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (!ok || tile < 0) break;
             const int m = tile % n_m, n = tile / n_m;
             uint32_t act[kMaskWords];
             tile_mask(m, act);
@@ -396,12 +436,21 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
-        if (!ok && lane == 0) { report_timeout(status); abort_grace(); }
+        if (lane == 0) {
+            // the CTA that finishes last puts the counters back to zero for the next launch
+            if (ok && atomicAdd(queue + 1, 1u) + 1u == gridDim.x) {
+                queue[0] = 0u;
+                queue[1] = 0u;
+            }
+            if (!ok) { report_timeout(status); abort_grace(); }
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ UMMA issuer
-        int it = 0, tc = 0;
+        int it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
+        for (int tc = 0; ok; ++tc) {
+            const int tile = next_tile(tc);
+            if (tile < 0) { ok = tile == -1; break; }
             const int m = tile % n_m;
             const uint32_t idesc = umma_idesc_bf16(kBM, width(tile / n_m));
             uint32_t act[kMaskWords];
@@ -441,9 +490,10 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;
-        int tc = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tc) {
+        for (int tc = 0; ok; ++tc) {
+            const int tile = next_tile(tc);
+            if (tile < 0) { ok = tile == -1; break; }
             const int m = tile % n_m, n = tile / n_m;
             uint32_t act[kMaskWords];
             tile_mask(m, act);
@@ -980,7 +1030,8 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
     down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
-                                             n_n, wmax, ctx->d_status, ctx->wait_ns);
+                                             n_n, wmax, reinterpret_cast<unsigned*>(ctx->d_status) + 8, ctx->d_status,
+                                             ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
