@@ -328,18 +328,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             // P = exp2(S*c - m) as bf16 into the operand layout, row sum
             float rs4[4] = {0.f, 0.f, 0.f, 0.f};
             uint8_t* prow = p_s + b * kPBytes + r * 128;
+            // sixteen scores at a time, each step over all sixteen before the next (arguments, then
+            // exponentials, then sums and packing): the steps of one score depend on each other, so
+            // score-by-score code runs at the sum of the instruction latencies
 #pragma unroll
-            for (int c0 = 0; c0 < kKV; c0 += 8) {
-                uint32_t pk[4];
+            for (int c0 = 0; c0 < kKV; c0 += 16) {
+                float x[16];
 #pragma unroll
-                for (int i = 0; i < 8; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(v[c0 + i]), scale_log2e, -m_use));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(v[c0 + i + 1]), scale_log2e, -m_use));
-                    rs4[(i >> 1) & 3] += p0 + p1;
-                    pk[i >> 1] = pack2(p0, p1);
+                for (int i = 0; i < 16; ++i) x[i] = fmaf(__uint_as_float(v[c0 + i]), scale_log2e, -m_use);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) x[i] = fast_exp2(x[i]);
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                    rs4[0] += x[i];
+                    rs4[1] += x[i + 1];
+                    rs4[2] += x[i + 2];
+                    rs4[3] += x[i + 3];
                 }
+                uint32_t pk[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[i] = pack2(x[2 * i], x[2 * i + 1]);
                 *reinterpret_cast<uint4*>(prow + (c0 / kBK) * kBlk + ((((c0 % kBK) / 8) ^ (r & 7)) << 4)) =
                     make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4*>(prow + (c0 / kBK) * kBlk + (((((c0 + 8) % kBK) / 8) ^ (r & 7)) << 4)) =
+                    make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
             lrow = fmaf(lrow, alpha, (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
             tc_fence_before_sync();
