@@ -138,3 +138,9 @@ def test_llama13b_layer_attention_and_qproj(ctx):
     assert (gq[~wo.expand_group_mask(mask[rows], cfg.attn_group)] == 0.0).all()
     assert np.abs(gq - ref).max() <= REL_TOL * np.abs(ref).max()
     assert ctx.status() == 0
+
+
+def test_prefill_four_times_the_largest_config(ctx):
+    """T = 16384 on the 8B shape: index arithmetic past the configs' sizes (perm of 1.8 M entries,
+    H of 235 M elements), several waves of tiles in every kernel."""
+    _chain(ctx, synth.CONFIGS["llama8b_prefill"].with_(tokens=16384), 3, n_sample=40)
