@@ -376,6 +376,221 @@ void launch_select_band(cudaStream_t s, int T, const float* sc32, int ksplit, in
         sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores);
 }
 
+// ---------------------------------------------------------------------------- fast pair-argmax path (bf16)
+// Eq. 4 with the bottleneck product on the tensor cores: u = x W1 comes from the same K-split
+// score GEMM as the top-k form (W1 transposed once per call, its rank <= 32 columns are the
+// "groups"), with the same rigorous bound on its error.  The logits l = u W2 are then formed in
+// fp32 per token and a pair is decided when its margin |l0 - l1| exceeds everything the errors of
+// u and of the fp32 product can add up to.  A pair that is too close to call (about one in 140
+// with Gaussian weights) is marked and decided by a second kernel from
+//     l0 - l1 = x . d_g,   d_g = W1 (W2[:, 2g] - W2[:, 2g+1])   (d_g in fp64, once per call),
+// one fp64 dot product of length D per marked pair.  fp64 FMAs are scarce on this part (a few per
+// clock and SM), which is why they are kept for the marked pairs.  If even that dot product is
+// within 2^-36 of zero relative to ||x|| ||d_g|| (an exact tie, in practice), the token is redone the
+// long way, u = x W1 and l = u W2 in fp64, which is the definition.
+constexpr int kPairMaxRank = 32;
+
+__global__ void __launch_bounds__(256)
+transpose_w1_kernel(const __nv_bfloat16* __restrict__ w1, int D, int rank, int NG, __nv_bfloat16* __restrict__ w1t,
+                    float* __restrict__ dn2) {
+    for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < NG; g += gridDim.x * blockDim.x) dn2[g] = 0.f;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < static_cast<long long>(D) * rank;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int c = static_cast<int>(i / D), d = static_cast<int>(i % D);
+        w1t[i] = w1[static_cast<size_t>(d) * rank + c];
+    }
+}
+
+// d64[g][i] = sum_c W1[i][c] (W2[c][2g] - W2[c][2g+1]) in fp64; dn2[g] += sum_i d^2 (fp32, rounded up).
+// Block = 128 rows i x 32 groups.
+__global__ void __launch_bounds__(128)
+pair_delta_kernel(const __nv_bfloat16* __restrict__ w1, const __nv_bfloat16* __restrict__ w2, int D, int rank, int NG,
+                  double* __restrict__ d64, float* __restrict__ dn2) {
+    __shared__ double delta[kPairMaxRank][32];
+    __shared__ float sq[32];
+    const int tid = threadIdx.x, g0 = blockIdx.y * 32, i = blockIdx.x * 128 + tid;
+    for (int e = tid; e < rank * 32; e += 128) {
+        const int c = e / 32, g = g0 + e % 32;
+        delta[c][e % 32] = g < NG ? static_cast<double>(__bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g])) -
+                                        static_cast<double>(__bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g + 1]))
+                                  : 0.0;
+    }
+    if (tid < 32) sq[tid] = 0.f;
+    __syncthreads();
+    double w[kPairMaxRank];
+#pragma unroll
+    for (int c = 0; c < kPairMaxRank; ++c)
+        w[c] = (c < rank && i < D) ? static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])) : 0.0;
+    for (int gg = 0; gg < 32 && g0 + gg < NG; ++gg) {
+        double a = 0.0;
+#pragma unroll
+        for (int c = 0; c < kPairMaxRank; ++c)
+            if (c < rank) a = fma(w[c], delta[c][gg], a);
+        if (i < D) d64[static_cast<size_t>(g0 + gg) * D + i] = a;
+        float q = static_cast<float>(a);
+        q = q * q * 1.0001f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+        if ((tid & 31) == 0) atomicAdd(&sq[gg], q);
+    }
+    __syncthreads();
+    if (tid < 32 && g0 + tid < NG) atomicAdd(dn2 + g0 + tid, sq[tid]);
+}
+
+// One warp per token.  Lane c holds u_c (c < rank); lane l decides the groups l, l + 32, ...
+__global__ void __launch_bounds__(128)
+pair_band_kernel(const float* __restrict__ u_slabs, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
+                 const __nv_bfloat16* __restrict__ w2, const float* __restrict__ wnorm, int T, int NG, int D, int rank,
+                 uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out, uint32_t* __restrict__ close_bits) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const int words = (NG + 31) >> 5;
+    const size_t slab = static_cast<size_t>(T) * ld;
+    float u = 0.f;
+    if (lane < rank)
+        for (int ks = 0; ks < nsplit; ++ks) u += __ldg(u_slabs + ks * slab + static_cast<size_t>(t) * ld + lane);
+    // ||x_t||
+    float xsq = 0.f;
+    const uint4* xv = reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * D);
+    for (int i = lane; i < D / 8; i += 32) {
+        const uint4 a = __ldg(xv + i);
+        const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(ah[e]);
+            xsq = fmaf(f.x, f.x, fmaf(f.y, f.y, xsq));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
+    // error bound of u_c (see the top-k form), then of the fp32 product below
+    const float steps = static_cast<float>((D + nsplit - 1) / nsplit + nsplit);
+    const float eu = lane < rank ? kAccumErr * steps * sqrtf(xsq) * 1.0001f * __ldg(wnorm + lane) : 0.f;
+    const float au = fabsf(u);
+    if (lane == 0) close_bits[static_cast<size_t>(t) * 32 + 31] = __float_as_uint(sqrtf(xsq) * 1.0001f);
+    for (int j = 0; j < words; ++j) {
+        const int g = 32 * j + lane;
+        float l0 = 0.f, l1 = 0.f, band = 0.f, mag = 0.f;
+        for (int c = 0; c < rank; ++c) {
+            const float uc = __shfl_sync(0xffffffffu, u, c), ec = __shfl_sync(0xffffffffu, eu, c);
+            const float ac = __shfl_sync(0xffffffffu, au, c);
+            if (g < NG) {
+                const float a0 = __bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g]);
+                const float a1 = __bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g + 1]);
+                l0 = fmaf(uc, a0, l0);
+                l1 = fmaf(uc, a1, l1);
+                const float aa = fabsf(a0) + fabsf(a1);
+                band = fmaf(ec, aa, band);
+                mag = fmaf(ac, aa, mag);
+            }
+        }
+        // fp32 rounding of the two sums and of their difference: (rank + 2) * 2^-24 * sum |u||a|
+        band = (band + static_cast<float>(rank + 2) * kAccumErr * mag) * 1.001f;
+        const bool sel = g < NG && l0 >= l1;
+        const bool close = g < NG && fabsf(l0 - l1) <= band;
+        const unsigned word = __ballot_sync(0xffffffffu, sel), cword = __ballot_sync(0xffffffffu, close);
+        if (lane == 0) {
+            mask_bits[static_cast<size_t>(t) * words + j] = word;
+            close_bits[static_cast<size_t>(t) * 32 + j] = cword;
+        }
+        if (scores_out && g < NG) {
+            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = l0;
+            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = l1;
+        }
+    }
+}
+
+// The marked pairs, exactly.  One block per token (most have nothing marked and leave at once).
+__global__ void __launch_bounds__(128)
+pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w1,
+                  const __nv_bfloat16* __restrict__ w2, const double* __restrict__ d64, const float* __restrict__ dn2,
+                  int T, int D, int rank, int NG, const uint32_t* __restrict__ close_bits,
+                  uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out) {
+    __shared__ double s_part[4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int words = (NG + 31) >> 5;
+    for (int t = blockIdx.x; t < T; t += gridDim.x) {
+        const uint32_t cw = close_bits[static_cast<size_t>(t) * 32 + lane];   // words [0, W) marks, word 31 ||x||
+        if (!__any_sync(0xffffffffu, lane < words && cw != 0u)) continue;      // the same in all four warps
+        const __nv_bfloat16* xr = x + static_cast<size_t>(t) * D;
+        const float xnorm = __uint_as_float(__shfl_sync(0xffffffffu, cw, 31));
+        bool long_way = false;
+        for (int j = 0; j < words; ++j) {
+            uint32_t bits = __shfl_sync(0xffffffffu, cw, j);
+            uint32_t word = mask_bits[static_cast<size_t>(t) * words + j];
+            while (bits) {
+                const int b = __ffs(bits) - 1;
+                bits &= bits - 1;
+                const int g = 32 * j + b;
+                const double* dr = d64 + static_cast<size_t>(g) * D;
+                // eight consecutive elements per thread and step: one 16-byte load of x, four of d_g
+                double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+#pragma unroll 4
+                for (int i = threadIdx.x * 8; i < D; i += 1024) {
+                    const uint4 xa = *reinterpret_cast<const uint4*>(xr + i);
+                    const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xa);
+                    const double2* dv = reinterpret_cast<const double2*>(dr + i);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __bfloat1622float2(xh[e]);
+                        const double2 d = dv[e];
+                        acc[2 * e] = fma(static_cast<double>(f.x), d.x, acc[2 * e]);
+                        acc[2 * e + 1] = fma(static_cast<double>(f.y), d.y, acc[2 * e + 1]);
+                    }
+                }
+                double m = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+                if (lane == 0) s_part[warp] = m;
+                __syncthreads();
+                m = (s_part[0] + s_part[1]) + (s_part[2] + s_part[3]);
+                __syncthreads();
+                if (fabs(m) <= 1.4551915e-11 * static_cast<double>(xnorm * sqrtf(dn2[g]) * 1.001f)) long_way = true;   // 2^-36
+                word = m >= 0.0 ? (word | (1u << b)) : (word & ~(1u << b));
+                if (scores_out && threadIdx.x == 0) {
+                    // keep the pair's mean, set its difference to the exact one
+                    float* sp = scores_out + static_cast<size_t>(t) * 2 * NG + 2 * g;
+                    const float mid = 0.5f * (sp[0] + sp[1]);
+                    sp[0] = mid + 0.5f * static_cast<float>(m);
+                    sp[1] = mid - 0.5f * static_cast<float>(m);
+                }
+            }
+            if (threadIdx.x == 0) mask_bits[static_cast<size_t>(t) * words + j] = word;
+        }
+        if (long_way && warp == 0) {
+            // the definition: u = x W1, l = u W2, all in fp64
+            double uu = 0.0;   // lane c ends up with u_c
+            for (int c = 0; c < rank; ++c) {
+                double a = 0.0;
+                for (int i = lane; i < D; i += 32)
+                    a = fma(static_cast<double>(__bfloat162float(xr[i])),
+                            static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])), a);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                if (lane == c) uu = a;
+            }
+            for (int j = 0; j < words; ++j) {
+                const int g = 32 * j + lane;
+                double l0 = 0.0, l1 = 0.0;
+                for (int c = 0; c < rank; ++c) {
+                    const double uc = __shfl_sync(0xffffffffu, uu, c);
+                    if (g < NG) {
+                        l0 = fma(uc, static_cast<double>(__bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g])), l0);
+                        l1 = fma(uc, static_cast<double>(__bfloat162float(w2[static_cast<size_t>(c) * 2 * NG + 2 * g + 1])), l1);
+                    }
+                }
+                const unsigned word = __ballot_sync(0xffffffffu, g < NG && l0 >= l1);
+                if (lane == 0) mask_bits[static_cast<size_t>(t) * words + j] = word;
+                if (scores_out && g < NG) {
+                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = static_cast<float>(l0);
+                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = static_cast<float>(l1);
+                }
+            }
+        }
+    }
+}
+
 template <typename TA, typename TB>
 void launch_gemm_f64(wide_ctx* ctx, cudaStream_t s, const TA* A, const TB* B, double* C, int M, int N, int K,
                      long long sbk, long long sbn) {
@@ -423,6 +638,52 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
 #undef WIDE_SEL_CASE
             default: return WIDE_ERR_UNSUPPORTED_SHAPE;
         }
+        return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+    }
+    if (mode == WIDE_ROUTE_PAIR_ARGMAX && dtype == WIDE_BF16 && D % 64 == 0 && D <= 16384 && ctx->encode_tiled &&
+        !(flags & WIDE_FLAG_SIMT) && rank <= kPairMaxRank && rank % 8 == 0 &&
+        static_cast<size_t>(T) * rank * sizeof(double) >= static_cast<size_t>(rank) * D * 2 &&
+        static_cast<size_t>(T) * 2048 >= static_cast<size_t>(NG) * D * sizeof(double)) {
+        // workspace: [0] u slabs (fp32 [ks][T, 32]) | [1] W1^T (bf16 [rank, D]) | [2] marked pairs (bits [T, W])
+        //            | [3] d_g (fp64 [NG, D]) | tail: column norms of W1 (256 floats at most) and ||d_g||^2
+        const size_t off1 = wide_align_up(static_cast<size_t>(T) * 2 * NG * sizeof(double), 256);
+        const size_t off2 = off1 + wide_align_up(static_cast<size_t>(T) * rank * sizeof(double), 256);
+        const size_t off3 = off2 + wide_align_up(static_cast<size_t>(T) * 128, 256);
+        const size_t total = wide_route_workspace(T, NG, rank);
+        char* wsb = static_cast<char*>(ws);
+        float* slabs = static_cast<float*>(ws);
+        __nv_bfloat16* w1t = reinterpret_cast<__nv_bfloat16*>(wsb + off1);
+        uint32_t* close_bits = reinterpret_cast<uint32_t*>(wsb + off2);
+        double* d64 = reinterpret_cast<double*>(wsb + off3);
+        float* wn = reinterpret_cast<float*>(wsb + total - 1024);      // 32 floats used
+        float* dn2 = wn + 64;                                           // NG <= 192 floats fit behind them
+        if (NG > 192) return WIDE_ERR_UNSUPPORTED_SHAPE;
+        const int ld = 32;
+        int max_split = static_cast<int>(off1 / (static_cast<size_t>(T) * ld * sizeof(float)));
+        if (max_split > kMaxSlabs) max_split = kMaxSlabs;
+        if (max_split < 1) max_split = 1;
+        const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+        const __nv_bfloat16* w1b = static_cast<const __nv_bfloat16*>(w_router);
+        const __nv_bfloat16* w2b = static_cast<const __nv_bfloat16*>(w2);
+        {
+            WideLaunch l(ctx, s, "route_pair_transpose");
+            transpose_w1_kernel<<<64, 256, 0, s>>>(w1b, D, rank, NG, w1t, dn2);
+        }
+        {
+            WideLaunch l(ctx, s, "route_pair_delta");
+            pair_delta_kernel<<<dim3((D + 127) / 128, (NG + 31) / 32), 128, 0, s>>>(w1b, w2b, D, rank, NG, d64, dn2);
+        }
+        int ksplit = 1;
+        const int rc = wide_launch_scores_tc(ctx, s, x, w1t, T, rank, ld, D, slabs, wn, max_split, &ksplit);
+        if (rc != WIDE_OK) return rc;
+        {
+            WideLaunch l(ctx, s, "route_pair_band");
+            pair_band_kernel<<<(T + 3) / 4, 128, 0, s>>>(slabs, ksplit, ld, xb, w2b, wn, T, NG, D, rank, mask_bits, scores,
+                                                          close_bits);
+        }
+        WideLaunch l(ctx, s, "route_pair_exact");
+        const int grid = T < 16 * ctx->sm_count ? T : 16 * ctx->sm_count;
+        pair_exact_kernel<<<grid, 128, 0, s>>>(xb, w1b, w2b, d64, dn2, T, D, rank, NG, close_bits, mask_bits, scores);
         return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
     }
     double* sc = static_cast<double*>(ws);

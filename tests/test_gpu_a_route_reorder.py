@@ -96,6 +96,47 @@ def test_route_pair_argmax_bit_exact(ctx, dtype):
     np.testing.assert_allclose(scores.cpu().numpy(), logits.reshape(cfg.tokens, -1), rtol=1e-5, atol=1e-5)
 
 
+def test_route_pair_argmax_layer_size_and_near_ties(ctx):
+    """The tensor-core form of Eq. 4 at a layer's size: pairs whose logits tie exactly, differ by one
+    bf16 ulp of one weight, or differ only by rounding noise are all decided as fp64 decides them."""
+    from paper_2607_28418_b200 import binding
+    T, D, NG, rank = 1024, 2048, 86, 16
+    rng = np.random.default_rng(11)
+    x = synth.round_to_bf16(rng.standard_normal((T, D)).astype(np.float32))
+    x[3] = 0.0                                                      # every pair ties
+    w1 = synth.round_to_bf16((rng.standard_normal((D, rank)) / np.sqrt(D)).astype(np.float32))
+    w2 = synth.round_to_bf16((rng.standard_normal((rank, NG, 2)) / np.sqrt(rank)).astype(np.float32))
+    w2[:, 0::5, 1] = w2[:, 0::5, 0]                                 # exact ties for every token
+    for g in range(1, NG, 5):                                       # one ulp apart in one row
+        c = int(rng.integers(0, rank))
+        w2[:, g, 1] = w2[:, g, 0]
+        w2[c, g, 1] = synth.round_to_bf16(np.array([w2[c, g, 0] * (1 + 2.0 ** -7)], dtype=np.float32))[0]
+    w2 = synth.round_to_bf16(w2).reshape(rank, 2 * NG)
+    logits = wo.route_logits_pair(x, w1, w2)
+    ref = wo.pack_mask_bits(wo.mask_pair_argmax(logits))
+    xd, w1d, w2d = to_dev(x, "bf16"), to_dev(w1, "bf16"), to_dev(w2, "bf16")
+    bits, scores = binding.wide_route(ctx, xd, w1d, NG, mode=binding.ROUTE_PAIR_ARGMAX, w2=w2d, rank=rank,
+                                      want_scores=True)
+    assert (bits_to_host(bits) == ref).all()
+    np.testing.assert_allclose(scores.cpu().numpy(), logits.reshape(T, -1), rtol=2e-3, atol=2e-3)
+    bits2, _ = binding.wide_route(ctx, xd, w1d, NG, mode=binding.ROUTE_PAIR_ARGMAX, w2=w2d, rank=rank,
+                                  flags=binding.FLAG_SIMT)
+    assert torch.equal(bits, bits2)
+
+
+def test_route_pair_argmax_integer_ties(ctx):
+    from paper_2607_28418_b200 import binding
+    T, D, NG, rank = 256, 256, 40, 8
+    rng = np.random.default_rng(3)
+    x = synth.round_to_bf16(rng.integers(-2, 3, size=(T, D)).astype(np.float32))
+    w1 = synth.round_to_bf16(rng.integers(-1, 2, size=(D, rank)).astype(np.float32))
+    w2 = synth.round_to_bf16(rng.integers(-1, 2, size=(rank, 2 * NG)).astype(np.float32))
+    ref = wo.pack_mask_bits(wo.mask_pair_argmax(wo.route_logits_pair(x, w1, w2)))
+    bits, _ = binding.wide_route(ctx, to_dev(x, "bf16"), to_dev(w1, "bf16"), NG, mode=binding.ROUTE_PAIR_ARGMAX,
+                                 w2=to_dev(w2, "bf16"), rank=rank)
+    assert (bits_to_host(bits) == ref).all()
+
+
 def test_route_argument_errors(ctx):
     from paper_2607_28418_b200 import binding
     x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
