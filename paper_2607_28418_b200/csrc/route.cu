@@ -641,7 +641,7 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
         return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
     }
     if (mode == WIDE_ROUTE_PAIR_ARGMAX && dtype == WIDE_BF16 && D % 64 == 0 && D <= 16384 && ctx->encode_tiled &&
-        !(flags & WIDE_FLAG_SIMT) && rank <= kPairMaxRank && rank % 8 == 0 &&
+        !(flags & WIDE_FLAG_SIMT) && rank <= kPairMaxRank && rank % 8 == 0 && NG <= 192 &&
         static_cast<size_t>(T) * rank * sizeof(double) >= static_cast<size_t>(rank) * D * 2 &&
         static_cast<size_t>(T) * 2048 >= static_cast<size_t>(NG) * D * sizeof(double)) {
         // workspace: [0] u slabs (fp32 [ks][T, 32]) | [1] W1^T (bf16 [rank, D]) | [2] marked pairs (bits [T, W])
@@ -656,8 +656,7 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
         uint32_t* close_bits = reinterpret_cast<uint32_t*>(wsb + off2);
         double* d64 = reinterpret_cast<double*>(wsb + off3);
         float* wn = reinterpret_cast<float*>(wsb + total - 1024);      // 32 floats used
-        float* dn2 = wn + 64;                                           // NG <= 192 floats fit behind them
-        if (NG > 192) return WIDE_ERR_UNSUPPORTED_SHAPE;
+        float* dn2 = wn + 64;                                           // NG <= 192 floats behind them
         const int ld = 32;
         int max_split = static_cast<int>(off1 / (static_cast<size_t>(T) * ld * sizeof(float)));
         if (max_split > kMaxSlabs) max_split = kMaxSlabs;
