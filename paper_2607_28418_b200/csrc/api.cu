@@ -334,7 +334,7 @@ int wide_attn(wide_ctx* ctx, void* stream, const void* q, const void* k, const v
         if (!mask_bits) return WIDE_ERR_INVALID_ARG;
         if (!wide_attn_decode_fits(tokens_q, n_q_heads, n_kv_heads)) return WIDE_ERR_UNSUPPORTED_SHAPE;
         return wide_launch_attn_decode(ctx, s, q, k, v, mask_bits, tokens_q, tokens_k, n_q_heads, n_kv_heads, head_dim,
-                                       heads_per_group, causal ? 1 : 0, scale, o);
+                                       heads_per_group, causal ? 1 : 0, scale, o, flags);
     }
     if (!perm || !counts) return WIDE_ERR_INVALID_ARG;
     if (!ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;

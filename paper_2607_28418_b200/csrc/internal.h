@@ -138,4 +138,4 @@ int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const
 bool wide_attn_decode_fits(int Tq, int Hq, int Hkv);
 int wide_launch_attn_decode(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, const void* v,
                             const uint32_t* mask_bits, int Tq, int Tk, int Hq, int Hkv, int head_dim, int hpg,
-                            int causal, float scale, void* o);
+                            int causal, float scale, void* o, unsigned flags);

@@ -158,16 +158,21 @@ def test_attention_half_chain_stage_by_stage(ctx):
     (2, 300, 8, 2, 64, 4),         # two tokens, head_dim 64
     (4, 515, 4, 4, 128, 1),        # four tokens (speculative block), every head its own group
     (1, 17, 2, 2, 128, 1),         # fewer keys than one chunk
+    (1, 20011, 8, 8, 128, 2),      # long cache: every warp goes round its ring stage several times
+    (2, 9001, 8, 2, 64, 4),        # eight query rows per KV head, head_dim 64, many tiles
 ])
 @pytest.mark.parametrize("causal", [True, False])
-def test_attn_decode_matches_oracle(ctx, t_q, t_k, h_q, h_kv, d, hpg, causal):
+@pytest.mark.parametrize("plain_loads", [False, True])
+def test_attn_decode_matches_oracle(ctx, t_q, t_k, h_q, h_kv, d, hpg, causal, plain_loads):
+    """Both decode kernels: K and V through the TMA ring (default) and by plain loads (WIDE_FLAG_SIMT)."""
     from paper_2607_28418_b200 import binding
     case = synth.make_attn_case(21, t_q, t_k, h_q, h_kv, d)
     mask = synth.bernoulli_mask(22 + t_k, t_q, h_q // hpg, 0.5)
     mask[0, 0] = True
     o = binding.wide_attn(ctx, to_dev(case["q"].reshape(t_q, -1), "bf16"), to_dev(case["k"].reshape(t_k, -1), "bf16"),
                           to_dev(case["v"].reshape(t_k, -1), "bf16"), h_q, h_kv, hpg, None, causal=causal,
-                          mask_bits=bits_to_dev(wo.pack_mask_bits(mask)))
+                          mask_bits=bits_to_dev(wo.pack_mask_bits(mask)),
+                          flags=binding.FLAG_SIMT if plain_loads else 0)
     torch.cuda.synchronize()
     assert ctx.status() == 0
     ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg, causal=causal)
