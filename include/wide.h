@@ -197,8 +197,11 @@ WIDE_API int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int d
  *       tokens with the same mask next to each other, so that token tiles taken in this order share
  *       their active groups: token_order = the tokens in a STABLE sort by key(t), token_rank its
  *       inverse (token_rank[token_order[p]] = p), with
- *           key(t) = h >> 24,  h = 0x811C9DC5;  for each mask word w of token t:  h = (h ^ w) * 0x01000193
- *       (32-bit wrap-around).  The prefill FFN / O-projection keep their intermediate rows in this
+ *           n_groups <= 32:  key(t) = mask word 0 of token t & 0xFF  (the decisions for groups 0..7:
+ *                            a tile of the sorted order agrees on the leading ones)
+ *           n_groups  > 32:  key(t) = h >> 24,  h = 0x811C9DC5;  for each mask word w of token t:
+ *                            h = (h ^ w) * 0x01000193  (32-bit wrap-around)
+ *       The prefill FFN / O-projection keep their intermediate rows in this
  *       order and walk token tiles in it; a (tile, group) block is skipped when no token of the tile
  *       selected the group.
  * tile_m must be a power of two >= 16.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE.
@@ -265,7 +268,8 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
  * Prefill form (tcgen05): query tiles gathered through perm.  Decode form (the last paragraph of
  * the paper's attention section: reordering bypassed, routing checked per block, online softmax
  * split over the keys): taken when mask_bits is given and tokens_q * (n_q_heads / n_kv_heads) <= 8;
- * K and V of a KV head none of whose query rows is active are not read.  WIDE_FLAG_FORCE_PREFILL /
+ * K and V of a KV head none of whose query rows is active are not read; the decode form brings K and
+ * V in by TMA (n_kv_heads <= 256), or by plain loads with WIDE_FLAG_SIMT.  WIDE_FLAG_FORCE_PREFILL /
  * WIDE_FLAG_FORCE_DECODE override the choice.
  * All device pointers, 16-byte aligned, owned by the caller; nothing is allocated; work is
  * enqueued on `stream`.  Needs dtype bf16, head_dim 64 or 128, n_q_heads % n_kv_heads == 0,

@@ -114,9 +114,12 @@ def unpack_mask_bits(bits: np.ndarray, n_groups: int) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------- token clustering
-def mask_key(words_row) -> int:
-    """Clustering key of one token: top 8 bits of an FNV-1a style hash over its packed mask words
-    (the definition stated in the library header; 32-bit wrap-around arithmetic)."""
+def mask_key(words_row, n_groups: int) -> int:
+    """Clustering key of one token (the definition stated in the library header): with at most 32
+    groups the decisions for groups 0..7 as an integer (bit g = group g); with more groups the top
+    8 bits of an FNV-1a style hash over its packed mask words (32-bit wrap-around arithmetic)."""
+    if n_groups <= 32:
+        return int(words_row[0]) & 0xFF
     h = 0x811C9DC5
     for w in words_row:
         h = ((h ^ int(w)) * 0x01000193) & 0xFFFFFFFF
@@ -129,7 +132,7 @@ def cluster_tokens(mask: np.ndarray) -> Dict[str, np.ndarray]:
     with identical masks are neighbours.  token_rank is the inverse of token_order."""
     bits = pack_mask_bits(mask)
     T = bits.shape[0]
-    keys = [mask_key(bits[t]) for t in range(T)]
+    keys = [mask_key(bits[t], mask.shape[1]) for t in range(T)]
     order = sorted(range(T), key=lambda t: (keys[t], t))
     rank = [0] * T
     for p, t in enumerate(order):

@@ -268,7 +268,6 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
     const int q = warp & 3;
     const int e = (warp - 2) * 32 + lane;  // 0..127, unique per epilogue thread
     const PassGeom g = geom_of(mode, a, n_union);
-    const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
     const int nb4 = (a.B + 3) / 4;  // 16-byte pieces of a row that hold real tokens
     {
         // Warm L2 with the accumulator rows this CTA will add to (they may have been evicted since

@@ -12,9 +12,13 @@ __device__ void build_metadata(const int32_t* counts, int NG, int tile_m, int n_
                                int32_t* __restrict__ union_list, int32_t* __restrict__ n_union,
                                int32_t* __restrict__ offsets);
 
-// Token clustering key: 8 bits of an FNV-1a style hash over the token's mask words.  Tokens with
-// the same mask get the same key.
-__device__ __forceinline__ unsigned mask_key(const uint32_t* __restrict__ row, int words) {
+// Token clustering key, 8 bits.  Up to 32 groups: the decisions for groups 0..7 themselves, so that
+// in sorted order a tile of tokens agrees on the leading decisions and the groups it agrees to skip
+// drop out of the tile's K loop even when every token has a mask of its own.  More groups: the top
+// byte of an FNV-1a style hash over the token's mask words (only equal masks can then share a tile
+// on purpose).  Tokens with the same mask get the same key either way.
+__device__ __forceinline__ unsigned mask_key(const uint32_t* __restrict__ row, int words, int NG) {
+    if (NG <= 32) return row[0] & 0xFFu;
     uint32_t h = 0x811C9DC5u;
     for (int w = 0; w < words; ++w) h = (h ^ row[w]) * 0x01000193u;
     return h >> 24;
@@ -24,7 +28,7 @@ __device__ __forceinline__ unsigned mask_key(const uint32_t* __restrict__ row, i
 // order[p] = token at clustered position p, rank[t] = position of token t.  Tokens that share a
 // mask end up next to each other, so token tiles taken in this order use few groups when the
 // router's decisions cluster.
-__device__ void cluster_tokens(const uint32_t* __restrict__ mask_bits, int T, int words, int32_t* __restrict__ order,
+__device__ void cluster_tokens(const uint32_t* __restrict__ mask_bits, int T, int words, int NG, int32_t* __restrict__ order,
                                int32_t* __restrict__ rank) {
     constexpr int nwarps = kPartThreads / 32;
     __shared__ unsigned s_next[256];                // next free position of every bucket
@@ -32,7 +36,7 @@ __device__ void cluster_tokens(const uint32_t* __restrict__ mask_bits, int T, in
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid < 256) s_next[tid] = 0u;
     __syncthreads();
-    for (int t = tid; t < T; t += kPartThreads) atomicAdd(&s_next[mask_key(mask_bits + static_cast<size_t>(t) * words, words)], 1u);
+    for (int t = tid; t < T; t += kPartThreads) atomicAdd(&s_next[mask_key(mask_bits + static_cast<size_t>(t) * words, words, NG)], 1u);
     __syncthreads();
     if (warp == 0) {
         // exclusive prefix over the 256 buckets: 8 per lane
@@ -52,7 +56,7 @@ __device__ void cluster_tokens(const uint32_t* __restrict__ mask_bits, int T, in
     __syncthreads();
     for (int c0 = 0; c0 < T; c0 += kPartThreads) {
         const int t = c0 + tid;
-        const unsigned key = t < T ? mask_key(mask_bits + static_cast<size_t>(t) * words, words) : 0xFFFFFFFFu;
+        const unsigned key = t < T ? mask_key(mask_bits + static_cast<size_t>(t) * words, words, NG) : 0xFFFFFFFFu;
         for (int i = tid; i < nwarps * 256; i += kPartThreads) (&s_wcnt[0][0])[i] = 0;
         __syncthreads();
         const unsigned peers = __match_any_sync(0xffffffffu, key);
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(kPartThreads) partition_kernel(const uint32_t*
     __shared__ int s_total;
     __shared__ int s_last;
     if (static_cast<int>(blockIdx.x) == NG) {  // the extra CTA clusters the tokens
-        cluster_tokens(mask_bits, T, words, token_order, token_rank);
+        cluster_tokens(mask_bits, T, words, NG, token_order, token_rank);
         return;
     }
     const int g = blockIdx.x;

@@ -221,25 +221,44 @@ def test_cluster_tokens_permutation_grouping_and_stability():
     assert sorted(order.tolist()) == list(range(T))
     assert (rank[order] == np.arange(T)).all() and (order[rank] == np.arange(T)).all()
     bits = wo.pack_mask_bits(mask)
-    keys = np.array([wo.mask_key(bits[t]) for t in range(T)])
+    keys = np.array([wo.mask_key(bits[t], NG) for t in range(T)])
     assert ((0 <= keys) & (keys < 256)).all()
     assert (np.diff(keys[order]) >= 0).all()                        # sorted by key
     for p in range(T - 1):                                           # stable inside a key
         if keys[order[p]] == keys[order[p + 1]]:
             assert order[p] < order[p + 1]
     # identical masks are neighbours unless two prototypes collide on the 8-bit key
-    proto_keys = {wo.mask_key(wo.pack_mask_bits(protos[i:i + 1])[0]) for i in range(5)}
+    proto_keys = {wo.mask_key(wo.pack_mask_bits(protos[i:i + 1])[0], NG) for i in range(5)}
     if len(proto_keys) == 5:
         runs = 1 + int((np.diff(which[order]) != 0).sum())
         assert runs == len(set(which.tolist()))
 
 
 def test_mask_key_is_the_header_hash():
-    # two worked values of h = (h ^ w) * 0x01000193 from h0 = 0x811C9DC5, top byte
-    assert wo.mask_key([0]) == ((0x811C9DC5 * 0x01000193) & 0xFFFFFFFF) >> 24
+    # more than 32 groups: two worked values of h = (h ^ w) * 0x01000193 from h0 = 0x811C9DC5, top byte
+    assert wo.mask_key([0, 0], 40) == ((((0x811C9DC5 * 0x01000193) & 0xFFFFFFFF) * 0x01000193) & 0xFFFFFFFF) >> 24
     h = ((0x811C9DC5 ^ 0xFFFFFFFF) * 0x01000193) & 0xFFFFFFFF
     h = ((h ^ 0x1) * 0x01000193) & 0xFFFFFFFF
-    assert wo.mask_key([0xFFFFFFFF, 1]) == h >> 24
+    assert wo.mask_key([0xFFFFFFFF, 1], 33) == h >> 24
+    # up to 32 groups: the decisions for groups 0..7 themselves
+    assert wo.mask_key([0b1_0110_0101], 10) == 0b0110_0101
+    assert wo.mask_key([0xFFFFFF00], 32) == 0
+
+
+def test_cluster_tokens_few_groups_tiles_agree_on_leading_decisions():
+    """With a handful of groups and a mask of its own per token, tiles of the clustered order still
+    skip blocks: the sorted order is lexicographic in the decisions for groups 7..0, so 32 tiles of
+    128 tokens agree on about five of them."""
+    T, NG, k = 4096, 10, 5
+    rng = np.random.default_rng(5)
+    mask = wo.mask_topk(rng.standard_normal((T, NG)), k)
+    order = wo.cluster_tokens(mask)["token_order"]
+    def active_blocks(m):
+        return sum(int(m[i:i + 128].any(axis=0).sum()) for i in range(0, T, 128))
+    assert active_blocks(mask) == 32 * NG                     # token order: nothing to skip
+    assert active_blocks(mask[order]) <= 0.87 * 32 * NG       # clustered order: about one block in six drops out
+    keys = np.array([wo.mask_key(b, NG) for b in wo.pack_mask_bits(mask)])
+    assert (np.diff(keys[order]) >= 0).all()
 
 
 # ----------------------------------------------------------------------------- gather / scatter
