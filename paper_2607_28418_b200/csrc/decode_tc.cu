@@ -16,7 +16,7 @@
 //                 (a ticket counter tells) turns it into h = M ? silu(gate) * up : 0 (bf16) and
 //                 re-zeroes the accumulator.
 //       (O-proj)  instead: a_masked = M ? attn_out : 0
-//   grid barrier  -- while waiting, each CTA's ring is already filled with its first W_down tiles
+//   grid barrier  -- while waiting, each CTA has its first two W_down tiles on order (not the whole ring)
 //   pass 2        W_down (or W_o): 128-row tiles x the columns of groups in U, same scheme; the CTA
 //                 that adds the last partial of a row tile converts it to the output dtype and
 //                 re-zeroes the accumulator.
@@ -517,11 +517,15 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
                 if (lane == 0) {
                     ok = produce_pass(MODE_GATEUP, a, &tmG, &tmU, &tmX, P, s_union, n_union, -1, 0);
                     if (ok) {
-                        // fill the ring with this CTA's first W_down tiles while the others finish
+                        // Ask for this CTA's first two W_down tiles while the others finish.  Only two:
+                        // the CTAs that finish pass 1 last go through a chain of dependent L2 round
+                        // trips (fence, ticket, sums, fence, barrier), and each of those takes about
+                        // 3 us while every SM has a full ring of weight tiles on order, about 1 us
+                        // when the memory system is quiet.
                         const PassGeom g2 = geom_of(MODE_DOWN, a, n_union);
                         const int mine = max(0, min((static_cast<int>(blockIdx.x) + 1) * g2.L, g2.total) -
                                                     min(static_cast<int>(blockIdx.x) * g2.L, g2.total));
-                        pre = min(P.nstages, mine);
+                        pre = min(min(P.nstages, 2), mine);
                         ok = produce_pass(MODE_DOWN, a, &tmWd, &tmWd, &tmH, P, s_union, n_union, pre, 0);
                     }
                 }
