@@ -10,7 +10,7 @@ import torch
 
 from oracle import wide_oracle as wo
 from paper_2607_28418_b200 import synth
-from tests.gpu_util import REL_TOL, bits_to_host, to_dev
+from tests.gpu_util import REL_TOL, bits_to_dev, bits_to_host, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -138,6 +138,29 @@ def test_llama13b_layer_attention_and_qproj(ctx):
     assert (gq[~wo.expand_group_mask(mask[rows], cfg.attn_group)] == 0.0).all()
     assert np.abs(gq - ref).max() <= REL_TOL * np.abs(ref).max()
     assert ctx.status() == 0
+
+
+def test_llama13b_layer_attention_decode_long_cache(ctx):
+    """The decode form at the size the benchmark times: one new token against a cache of 32 768
+    keys, 40 heads of 128, five of ten head groups active (both kernels: TMA ring and plain loads).
+    Every head is checked: the oracle's cost is one row of scores per head."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.CONFIGS["llama13b_layer"]
+    hd, Tk = 128, 32768
+    H, hpg, NG = cfg.attn_dim // hd, cfg.attn_group // hd, cfg.attn_n_groups
+    ac = synth.make_attn_case(4, 1, Tk, H, H, hd)
+    mask = synth.random_mask(9, 1, NG, cfg.attn_k)
+    bits = bits_to_dev(wo.pack_mask_bits(mask))
+    qd, kd, vd = (to_dev(ac[n].reshape(-1, H * hd), "bf16") for n in ("q", "k", "v"))
+    ref = wo.masked_attention(ac["q"], ac["k"], ac["v"], mask, hpg)
+    head_mask = np.repeat(mask, hpg, axis=1)
+    for flags in (0, binding.FLAG_SIMT):
+        o = binding.wide_attn(ctx, qd, kd, vd, H, H, hpg, None, causal=True, mask_bits=bits, flags=flags)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        got = o.float().cpu().numpy().reshape(1, H, hd)
+        assert (got[~head_mask] == 0.0).all()
+        assert np.abs(got - ref).max() <= REL_TOL * np.abs(ref).max()
 
 
 def test_prefill_four_times_the_largest_config(ctx):
