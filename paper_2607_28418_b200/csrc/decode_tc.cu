@@ -13,16 +13,16 @@
 //                 through a ring of 8 to 10 stages (>= 128 KB in flight per SM), tcgen05 accumulates in
 //                 TMEM, the epilogue adds each partial tile into an L2-resident fp32 accumulator
 //                 with 16-byte red.add.  The CTA that adds the last partial of a 128-channel block
-//                 (a ticket counter tells) turns it into h = M ? silu(gate) * up : 0 (bf16) and
-//                 re-zeroes the accumulator.
+//                 (a ticket counter tells) turns it into h = M ? silu(gate) * up : 0 (bf16).
 //       (O-proj)  instead: a_masked = M ? attn_out : 0
 //   grid barrier  -- while waiting, each CTA has its first two W_down tiles on order (not the whole ring)
 //   pass 2        W_down (or W_o): 128-row tiles x the columns of groups in U, same scheme; the CTA
-//                 that adds the last partial of a row tile converts it to the output dtype and
-//                 re-zeroes the accumulator.
+//                 that adds the last partial of a row tile converts it to the output dtype.
+//   Clearing the accumulators is nobody's critical path: the epilogue warps clear the output sums
+//   at the start of pass 1 and the gate / up sums at the start of pass 2, a share per CTA.
 //
-// The fp32 accumulators, ticket counters and barrier words belong to the context and are zero
-// between calls.  One context must not run two decode calls concurrently.
+// The fp32 accumulators, ticket counters and barrier words belong to the context; counters, barrier
+// words and the gate / up sums are zero between calls.  One context must not run two decode calls concurrently.
 #include <cuda.h>
 
 #include "internal.h"
@@ -54,9 +54,9 @@ struct DecodeArgs {
     int row_tiles;         // pass 2: ceil(D / 128)
     const uint32_t* mask_bits;
     const __nv_bfloat16* act_in;  // O-proj: attention output [B, inner]
-    float* gate;           // [inner, NT] fp32 (token fastest), zero on entry and on exit
+    float* gate;           // [inner, NT] fp32 (token fastest), zero on entry; cleared again during pass 2
     float* up;
-    float* yacc;           // [D, NT]
+    float* yacc;           // [D, NT], cleared during pass 1 (or the masking phase)
     __nv_bfloat16* h;      // [64, inner] bf16 scratch (caller workspace)
     void* y;
     int out_bf16;
@@ -270,6 +270,22 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
     const PassGeom g = geom_of(mode, a, n_union);
     const int nb4 = (a.B + 3) / 4;  // 16-byte pieces of a row that hold real tokens
     {
+        // The accumulators of the OTHER pass are idle now: put this CTA's share of them back to zero
+        // (pass 1 clears the output sums that pass 2 will add to, pass 2 clears the gate / up sums for
+        // the next call; the grid barrier between the passes orders both against their use).
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (mode == MODE_GATEUP) {
+            float4* p = reinterpret_cast<float4*>(a.yacc);
+            const int n = a.D * (a.NT / 4);
+            for (int i = blockIdx.x * 128 + e; i < n; i += gridDim.x * 128) p[i] = z;
+        } else if (a.is_ffn) {
+            float4* pg = reinterpret_cast<float4*>(a.gate);
+            float4* pu = reinterpret_cast<float4*>(a.up);
+            const int n = a.inner * (a.NT / 4);
+            for (int i = blockIdx.x * 128 + e; i < n; i += gridDim.x * 128) { pg[i] = z; pu[i] = z; }
+        }
+    }
+    {
         // Warm L2 with the accumulator rows this CTA will add to (they may have been evicted since
         // the previous call zeroed them), so the red.adds at the end of the pass hit L2.
         Share pre(blockIdx.x, g.total, g.L, g.spb);
@@ -353,7 +369,7 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
         if (*s_flag) {
             constexpr int kB4 = 8;  // 16-byte pieces per round: 2 * kB4 loads in flight per thread
             if (mode == MODE_GATEUP) {
-                // h[b, ch] for the 128 (or G) channels of this block; re-zero gate / up
+                // h[b, ch] for the 128 (or G) channels of this block
                 // which tokens execute which group of the tile: thread e looks at token e % 64 for
                 // the group of the tile half e / 64 (one group per tile: both halves see the same)
                 const int vslot = a.gpb > 1 ? slot_blk * a.gpb + (e >> 6) : slot_blk / a.blocks_per_group;
@@ -368,8 +384,10 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
                 const unsigned long long tokmask =
                     static_cast<unsigned long long>(s_tokmask[mh]) | (static_cast<unsigned long long>(s_tokmask[mh + 1]) << 32);
                 if (ch_valid) {
-                    float4* gp = reinterpret_cast<float4*>(a.gate + static_cast<size_t>(ch) * a.NT);
-                    float4* up = reinterpret_cast<float4*>(a.up + static_cast<size_t>(ch) * a.NT);
+                    const float4* gp = reinterpret_cast<const float4*>(a.gate + static_cast<size_t>(ch) * a.NT);
+                    const float4* up = reinterpret_cast<const float4*>(a.up + static_cast<size_t>(ch) * a.NT);
+                    __nv_bfloat16* hp = a.h + ch;                  // token b of this channel: hp[b * inner]
+                    unsigned long long tm = tokmask;
                     for (int b0 = 0; b0 < nb4; b0 += kB4) {
                         float4 gv[kB4], uv[kB4];
 #pragma unroll
@@ -382,17 +400,17 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
 #pragma unroll
                         for (int j = 0; j < kB4; ++j) {
                             if (b0 + j < nb4) {
-                                gp[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                up[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 const float gs[4] = {gv[j].x, gv[j].y, gv[j].z, gv[j].w};
                                 const float us[4] = {uv[j].x, uv[j].y, uv[j].z, uv[j].w};
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
                                     const int b = 4 * (b0 + j) + i;
                                     if (b < a.B) {
-                                        const float v = ((tokmask >> b) & 1ull) ? gs[i] / (1.f + __expf(-gs[i])) * us[i] : 0.f;
-                                        a.h[static_cast<size_t>(b) * a.inner + ch] = __float2bfloat16_rn(v);
+                                        const float v = (tm & 1ull) ? __fdividef(gs[i], 1.f + __expf(-gs[i])) * us[i] : 0.f;
+                                        *hp = __float2bfloat16_rn(v);
                                     }
+                                    hp += a.inner;
+                                    tm >>= 1;
                                 }
                             }
                         }
@@ -410,7 +428,6 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
 #pragma unroll
                         for (int j = 0; j < kB4; ++j) {
                             if (b0 + j < nb4) {
-                                yp[b0 + j] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 const float vs[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
@@ -538,6 +555,11 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
             const int vec_per_row = a.inner / 8, vec_per_group = a.G / 8;
             const uint4* src = reinterpret_cast<const uint4*>(a.act_in);
             uint4* dst = reinterpret_cast<uint4*>(a.h);
+            {
+                float4* p = reinterpret_cast<float4*>(a.yacc);   // the output sums, cleared before pass 2 adds to them
+                const long long n = static_cast<long long>(a.D) * (a.NT / 4);
+                for (long long i = gtid; i < n; i += gthreads) p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
             for (long long i = gtid; i < static_cast<long long>(a.B) * vec_per_row; i += gthreads) {
                 const int t = static_cast<int>(i / vec_per_row);
                 const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
@@ -593,7 +615,10 @@ constexpr int kSmemD = kRingBytesD + (2 * kMaxStagesD + 4) * 8 + 16 + 1024;
 int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a, const void* wg, const void* wu,
                   const void* wd, int B, int D, int inner, int G, const uint32_t* mask_bits, void* y, int out_dtype,
                   void* ws) {
-    if (static_cast<size_t>(kMaxNT) * (2 * static_cast<size_t>(inner) + D) > ctx->decode_acc_floats)
+    // The output sums sit at a fixed place (they are left as they are after a call and cleared at the
+    // start of the next one, whatever its shape); the gate / up sums follow and are zero between calls.
+    constexpr size_t kYaccFloats = static_cast<size_t>(kMaxNT) * 16384;
+    if (D > 16384 || kYaccFloats + static_cast<size_t>(kMaxNT) * 2 * static_cast<size_t>(inner) > ctx->decode_acc_floats)
         return WIDE_ERR_UNSUPPORTED_SHAPE;
     DecodeArgs a{};
     a.is_ffn = is_ffn ? 1 : 0;
@@ -610,9 +635,9 @@ int launch_decode(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* x_or_a
     a.row_tiles = (D + kRows - 1) / kRows;
     a.mask_bits = mask_bits;
     a.act_in = static_cast<const __nv_bfloat16*>(x_or_a);
-    a.gate = ctx->decode_acc;
-    a.up = ctx->decode_acc + static_cast<size_t>(kMaxNT) * inner;
-    a.yacc = ctx->decode_acc + 2 * static_cast<size_t>(kMaxNT) * inner;
+    a.yacc = ctx->decode_acc;
+    a.gate = ctx->decode_acc + kYaccFloats;
+    a.up = a.gate + static_cast<size_t>(kMaxNT) * inner;
     a.h = static_cast<__nv_bfloat16*>(ws);
     a.y = y;
     a.out_bf16 = out_dtype == WIDE_BF16 ? 1 : 0;
