@@ -387,7 +387,7 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
                     const float4* gp = reinterpret_cast<const float4*>(a.gate + static_cast<size_t>(ch) * a.NT);
                     const float4* up = reinterpret_cast<const float4*>(a.up + static_cast<size_t>(ch) * a.NT);
                     __nv_bfloat16* hp = a.h + ch;                  // token b of this channel: hp[b * inner]
-                    unsigned long long tm = tokmask;
+                    const unsigned long long tm = tokmask;
                     for (int b0 = 0; b0 < nb4; b0 += kB4) {
                         float4 gv[kB4], uv[kB4];
 #pragma unroll
@@ -400,18 +400,20 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
 #pragma unroll
                         for (int j = 0; j < kB4; ++j) {
                             if (b0 + j < nb4) {
-                                const float gs[4] = {gv[j].x, gv[j].y, gv[j].z, gv[j].w};
-                                const float us[4] = {uv[j].x, uv[j].y, uv[j].z, uv[j].w};
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    const int b = 4 * (b0 + j) + i;
-                                    if (b < a.B) {
-                                        const float v = (tm & 1ull) ? __fdividef(gs[i], 1.f + __expf(-gs[i])) * us[i] : 0.f;
-                                        *hp = __float2bfloat16_rn(v);
-                                    }
-                                    hp += a.inner;
-                                    tm >>= 1;
-                                }
+                                // four tokens at a time, no branches: rows of h past the batch (up to
+                                // the next multiple of four) are scratch and get zeros (their sums are zero)
+                                const float e0 = __expf(-gv[j].x), e1 = __expf(-gv[j].y);
+                                const float e2 = __expf(-gv[j].z), e3 = __expf(-gv[j].w);
+                                const float r0 = __fdividef(gv[j].x, 1.f + e0) * uv[j].x;
+                                const float r1 = __fdividef(gv[j].y, 1.f + e1) * uv[j].y;
+                                const float r2 = __fdividef(gv[j].z, 1.f + e2) * uv[j].z;
+                                const float r3 = __fdividef(gv[j].w, 1.f + e3) * uv[j].w;
+                                const unsigned m4 = static_cast<unsigned>(tm >> (4 * (b0 + j))) & 15u;
+                                __nv_bfloat16* hq = hp + static_cast<size_t>(4 * (b0 + j)) * a.inner;
+                                hq[0] = __float2bfloat16_rn((m4 & 1u) ? r0 : 0.f);
+                                hq[a.inner] = __float2bfloat16_rn((m4 & 2u) ? r1 : 0.f);
+                                hq[2 * static_cast<size_t>(a.inner)] = __float2bfloat16_rn((m4 & 4u) ? r2 : 0.f);
+                                hq[3 * static_cast<size_t>(a.inner)] = __float2bfloat16_rn((m4 & 8u) ? r3 : 0.f);
                             }
                         }
                     }
