@@ -128,20 +128,21 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// All CTAs of the (co-resident) grid meet here; used once per launch.  bar[0] counts arrivals,
-// bar[1] departures: the CTA that leaves last puts both back to zero for the next launch, so the
-// kernel can be replayed from a CUDA graph without host-side state.  Returns false if the wait
-// expired.
+// All CTAs of the (co-resident) grid meet here; used once per launch.  bar[0] counts arrivals
+// (a fire-and-forget red after a fence; thread 0 then polls with acquire loads), bar[1] departures:
+// the CTA that leaves last puts both back to zero for the next launch, so the kernel can be replayed
+// from a CUDA graph without host-side state.  Returns false if the wait expired.
 __device__ bool grid_barrier(unsigned* bar, unsigned long long wait_ns, volatile int* abort_flag, int* status) {
+    __shared__ int s_passed;
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(bar, 1u);
+        // arrive without waiting for the counter's old value: one round trip less on the critical path
+        asm volatile("red.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
         bool passed = true;
         if (!*abort_flag) {
             const uint64_t start = globaltimer_ns();
             while (ld_acquire_u32(bar) < gridDim.x) {
-                __nanosleep(20);
                 if (globaltimer_ns() - start > wait_ns) {
                     *abort_flag = 1;
                     atomicExch(status, WIDE_ERR_TIMEOUT);
@@ -152,13 +153,14 @@ __device__ bool grid_barrier(unsigned* bar, unsigned long long wait_ns, volatile
         } else {
             passed = false;
         }
-        __threadfence();
-        if (passed && atomicAdd(bar + 1, 1u) + 1u == gridDim.x) {
-            bar[0] = 0u;
-            bar[1] = 0u;
-        }
+        s_passed = passed;
     }
     __syncthreads();
+    // departures are counted off the critical path, by a thread that has nothing to do for a while
+    if (threadIdx.x == kThreadsD - 1 && s_passed && atomicAdd(bar + 1, 1u) + 1u == gridDim.x) {
+        bar[0] = 0u;
+        bar[1] = 0u;
+    }
     return *abort_flag == 0;
 }
 
