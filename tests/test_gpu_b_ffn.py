@@ -183,6 +183,24 @@ def test_decode_clustered_union_and_zero_cases(ctx):
     assert_close(y1, ref, "decode dense fp32 out")
 
 
+def test_decode_calls_of_different_shapes_share_one_context(ctx):
+    """The decode kernels keep fp32 sums, counters and a barrier in buffers owned by the context
+    (cleared by the kernels themselves, not by the host).  A sequence of calls whose shapes place
+    those sums differently -- small then large batch, narrow then wide layer, FFN then O-projection
+    and back -- must leave every call with clean sums."""
+    from paper_2607_28418_b200 import binding
+    seq = [("ffn", 5, 512, 2048, 128), ("ffn", 64, 1024, 4096, 128), ("oproj", 32, 512, 1024, 512),
+           ("ffn", 3, 1024, 2048, 64), ("oproj", 1, 1024, 512, 256), ("ffn", 64, 512, 2048, 256),
+           ("ffn", 16, 1024, 4096, 128)]
+    for i, (kind, B, D, inner, G) in enumerate(seq):
+        if kind == "ffn":
+            cfg = synth.WideConfig("t", tokens=B, hidden=D, d_ff=inner, group=G, k=max(1, inner // G // 2))
+            y, ref, _ = _run_ffn(ctx, cfg, 40 + i, binding.FLAG_NONE, with_meta=False)
+        else:
+            y, ref = _run_oproj(ctx, B, D, inner, G, 1, binding.FLAG_NONE, seed=40 + i)
+        assert_close(y, ref, f"call {i}: {kind} B{B} D{D} inner{inner} G{G}")
+
+
 # ----------------------------------------------------------------------------- O-projection
 def _run_oproj(ctx, T, D, K, G, k, flags, dtype="bf16", seed=0):
     from paper_2607_28418_b200 import binding
