@@ -339,14 +339,15 @@ attn_decode_ring_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 
     if (warp == kRingConsumers) {
         if (lane == 0) {
+            const uint64_t stream_policy = l2_policy_evict_first();   // K and V are read once
             for (int t = 0; t < ntiles; ++t) {
                 const int st = t % kRingStages;
                 const uint32_t ph = (t / kRingStages) & 1;
                 if (!mbar_wait(empty + 8 * st, ph ^ 1u, wait_ns, &s_abort)) break;
                 mbar_arrive_expect_tx(full + 8 * st, 2 * kTileBytes);
                 const uint32_t dst = smem_u32(ring + st * 2 * kTileBytes);
-                tma_load_2d(dst, &tmK, hkv * HD, j0 + t * kRingKeys, full + 8 * st);
-                tma_load_2d(dst + kTileBytes, &tmV, hkv * HD, j0 + t * kRingKeys, full + 8 * st);
+                tma_load_2d_hint(dst, &tmK, hkv * HD, j0 + t * kRingKeys, full + 8 * st, stream_policy);
+                tma_load_2d_hint(dst + kTileBytes, &tmV, hkv * HD, j0 + t * kRingKeys, full + 8 * st, stream_policy);
                 s_issued = t + 1;
             }
         }

@@ -193,6 +193,7 @@ __device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* t
     const int ksub = a.G / kBKD;
     const int rows_valid = mode == MODE_GATEUP ? a.rows_valid : kRows;
     const uint32_t act_tx = static_cast<uint32_t>(a.NT * kBKD * 2);
+    const uint64_t stream_policy = l2_policy_evict_first();   // weight tiles are read once
     Share sh(blockIdx.x, g.total, g.L, g.spb);
     Segment sg;
     int step = 0;
@@ -224,7 +225,7 @@ __device__ bool produce_pass(int mode, const DecodeArgs& a, const CUtensorMap* t
                 if (!mbar_wait(P.empty + 8 * s, ph ^ 1u, a.wait_ns, P.abort_flag)) return false;
                 mbar_arrive_expect_tx(P.full + 8 * s, stage_tx);
                 for (int j = 0; j < nbox; ++j)
-                    tma_load_2d(dst + j * rows_valid * (kBKD * 2), tw, col, row0[j], P.full + 8 * s);
+                    tma_load_2d_hint(dst + j * rows_valid * (kBKD * 2), tw, col, row0[j], P.full + 8 * s, stream_policy);
             }
             if (weights_only_steps < 0) tma_load_2d(dst + kWBytes, tmAct, col, 0, P.full + 8 * s);
         }
