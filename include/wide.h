@@ -269,7 +269,8 @@ WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const
  * the paper's attention section: reordering bypassed, routing checked per block, online softmax
  * split over the keys): taken when mask_bits is given and tokens_q * (n_q_heads / n_kv_heads) <= 8;
  * K and V of a KV head none of whose query rows is active are not read; the decode form brings K and
- * V in by TMA (n_kv_heads <= 256), or by plain loads with WIDE_FLAG_SIMT.  WIDE_FLAG_FORCE_PREFILL /
+ * V in by TMA (n_kv_heads <= 256; CUDA cores for one query row per KV head, warp-level tensor-core
+ * instructions for two to eight), or by plain loads with WIDE_FLAG_SIMT.  WIDE_FLAG_FORCE_PREFILL /
  * WIDE_FLAG_FORCE_DECODE override the choice.
  * All device pointers, 16-byte aligned, owned by the caller; nothing is allocated; work is
  * enqueued on `stream`.  Needs dtype bf16, head_dim 64 or 128, n_q_heads % n_kv_heads == 0,

@@ -23,7 +23,7 @@ namespace {
 
 constexpr int kMaxRows = 8;      // query rows per KV head served by one CTA
 constexpr int kDecWarps = 4;
-constexpr int kMaxSplits = 32;
+constexpr int kMaxSplits = 128;
 
 __device__ __forceinline__ float exp2_fast(float x) {
     float y;
@@ -484,41 +484,318 @@ attn_decode_ring_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The ring kernel for more than one query row per KV head (grouped-query attention, or a few new
+// tokens at once).  With R rows every key costs 2 * R * HD multiply-adds, which the CUDA cores cannot
+// issue at the rate HBM delivers the keys; the rows are therefore padded to the 16 rows of a
+// warp-level tensor-core instruction (mma.sync m16n8k16, bf16 in, fp32 out -- with at most eight real
+// rows there is no shape here for the 64-row tcgen05 instructions).  Same CTA layout as above: one
+// producer thread, four consumer warps, a stage of 32 keys per warp.  K and V tiles are laid down by
+// TMA in the 128-byte swizzle, [64-column half][32 keys][128 B], so that ldmatrix reads them without
+// bank conflicts: K as it lies (the B operand of S = Q K^T), V transposed on the way in (the B operand
+// of O += P V).  The score fragments are turned into the probabilities' A fragments in registers.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// d (16x8, fp32) += a (16x16, bf16, row-major) * b (16x8, bf16, column-major); rows 8..15 of a are zero
+// here, so the two accumulators of those rows (x2, x3) stay zero and are shared by all tiles.
+__device__ __forceinline__ void mma_16816(float& d0, float& d1, float& x2, float& x3, uint32_t a0, uint32_t a2, uint32_t b0,
+                                          uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d0), "+f"(d1), "+f"(x2), "+f"(x3)
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kRingThreads, 2)
+attn_decode_ring_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                            const __nv_bfloat16* __restrict__ q, const uint32_t* __restrict__ mask_bits, int words, int Tq,
+                            int Tk, int Hq, int Hkv, int hpg, int causal, float scale_log2e, int max_splits,
+                            float* __restrict__ part, int* __restrict__ hdr, int* status, unsigned long long wait_ns) {
+    using namespace wptx;
+    constexpr int kHalves = HD / 64;               // 64-column halves of a K or V tile
+    constexpr int kHalfBytes = kRingKeys * 128;    // 32 keys x 128 B
+    constexpr int kTileBytes = kHalves * kHalfBytes;
+    constexpr int kKS = HD / 16;                   // k-steps of S = Q K^T
+    constexpr int kNT = HD / 8;                    // 8-column tiles of O
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float wm[kRingConsumers][8], wl[kRingConsumers][8];
+    __shared__ uint8_t s_heads[256];
+    __shared__ int s_nact;
+    __shared__ int s_abort;
+    __shared__ int s_issued;
+    __shared__ __align__(8) uint64_t s_bars[2 * kRingStages];
+    uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rep = Hq / Hkv;
+    const int R = Tq * rep;                        // <= 8
+    const int delta = Tk - Tq;
+    const size_t ldq = static_cast<size_t>(Hq) * HD;
+    const uint32_t full = smem_u32(s_bars), empty = smem_u32(s_bars + kRingStages);
+
+    if (tid == 0) {
+        for (int st = 0; st < kRingStages; ++st) {
+            mbar_init(full + 8 * st, 1);
+            mbar_init(empty + 8 * st, 1);
+        }
+        s_abort = 0;
+        s_issued = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmK);
+        prefetch_tmap(&tmV);
+    }
+    if (warp == 0) {
+        int pos = 0;   // the KV heads that some row reads, ascending
+        for (int h0 = 0; h0 < Hkv; h0 += 32) {
+            const int hkv = h0 + lane;
+            bool any = false;
+            if (hkv < Hkv)
+                for (int r = 0; r < R; ++r) any = any || wide_mask_bit(mask_bits, words, r / rep, (hkv * rep + r % rep) / hpg);
+            const unsigned vote = __ballot_sync(0xffffffffu, any);
+            if (any) s_heads[pos + __popc(vote & ((1u << lane) - 1u))] = static_cast<uint8_t>(hkv);
+            pos += __popc(vote);
+        }
+        if (lane == 0) s_nact = pos;
+    }
+    __syncthreads();
+    const int n_act = s_nact;
+    if (n_act == 0) {
+        if (blockIdx.x == 0 && tid == 0) hdr[0] = 1;
+        return;
+    }
+    int n_splits = min(min(static_cast<int>(gridDim.x) / n_act, (Tk + kRingKeys - 1) / kRingKeys), max_splits);
+    if (n_splits < 1) n_splits = 1;
+    const int kps = ((Tk + n_splits - 1) / n_splits + kRingKeys - 1) / kRingKeys * kRingKeys;
+    n_splits = (Tk + kps - 1) / kps;          // no empty slice
+    if (blockIdx.x == 0 && tid == 0) hdr[0] = n_splits;
+    if (static_cast<int>(gridDim.x) < n_act) {
+        if (blockIdx.x == 0 && tid == 0) atomicExch(status, WIDE_ERR_UNSUPPORTED_SHAPE);
+        return;
+    }
+    if (static_cast<int>(blockIdx.x) >= n_act * n_splits) return;
+    const int hkv = s_heads[blockIdx.x / n_splits], split = blockIdx.x % n_splits;
+    const int j0 = split * kps, j1 = min(Tk, j0 + kps);
+    const int ntiles = (j1 - j0 + kRingKeys - 1) / kRingKeys;
+
+    // this thread's query row (fragment row lane / 4) and its A fragments: a0 = columns 16 ks + 2 (lane % 4) + {0, 1},
+    // a2 = the same + 8
+    const int qr = lane >> 2, qc = (lane & 3) * 2;
+    const bool row_ok = qr < R;
+    uint32_t qa0[kKS], qa2[kKS];
+    {
+        const int t = row_ok ? qr / rep : 0, h = hkv * rep + (row_ok ? qr % rep : 0);
+        const __nv_bfloat16* qp = q + t * ldq + static_cast<size_t>(h) * HD + qc;
+#pragma unroll
+        for (int ks = 0; ks < kKS; ++ks) {
+            qa0[ks] = row_ok ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
+            qa2[ks] = row_ok ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
+        }
+    }
+    const int lim = causal ? (row_ok ? qr / rep : 0) + delta : Tk - 1;   // last key this row may see
+    float m = -CUDART_INF_F, l = 0.f, x2 = 0.f, x3 = 0.f;
+    float o[kNT][2];
+#pragma unroll
+    for (int nt = 0; nt < kNT; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; }
+
+    if (warp == kRingConsumers) {
+        if (lane == 0) {
+            const uint64_t stream_policy = l2_policy_evict_first();   // K and V are read once
+            for (int t = 0; t < ntiles; ++t) {
+                const int st = t % kRingStages;
+                const uint32_t ph = (t / kRingStages) & 1;
+                if (!mbar_wait(empty + 8 * st, ph ^ 1u, wait_ns, &s_abort)) break;
+                mbar_arrive_expect_tx(full + 8 * st, 2 * kTileBytes);
+                const uint32_t dst = smem_u32(ring + st * 2 * kTileBytes);
+#pragma unroll
+                for (int hb = 0; hb < kHalves; ++hb) {
+                    tma_load_2d_hint(dst + hb * kHalfBytes, &tmK, hkv * HD + 64 * hb, j0 + t * kRingKeys, full + 8 * st, stream_policy);
+                    tma_load_2d_hint(dst + kTileBytes + hb * kHalfBytes, &tmV, hkv * HD + 64 * hb, j0 + t * kRingKeys, full + 8 * st,
+                                     stream_policy);
+                }
+                s_issued = t + 1;
+            }
+        }
+    } else {
+        // ldmatrix row addresses of this lane: matrix lane / 8 of an x4 load, row lane % 8
+        const int lrow = lane & 7, lmat = lane >> 3;
+        for (int t = warp; t < ntiles; t += kRingConsumers) {
+            const int st = t % kRingStages;
+            const uint32_t ph = (t / kRingStages) & 1;
+            if (!mbar_wait(full + 8 * st, ph, wait_ns, &s_abort)) break;
+            const uint32_t kt = smem_u32(ring + st * 2 * kTileBytes), vt = kt + kTileBytes;
+            const int c0 = j0 + t * kRingKeys;
+            // S = Q K^T: four 8-key tiles, kKS k-steps.  One x4 load = (k-step ks, columns +0 / +8) and (ks + 1, +0 / +8)
+            float sc[4][2];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                sc[nt][0] = 0.f; sc[nt][1] = 0.f;
+                const int krow = 8 * nt + lrow;
+#pragma unroll
+                for (int ks = 0; ks < kKS; ks += 2) {
+                    const int h0 = 16 * (ks + (lmat >> 1)) + 8 * (lmat & 1);           // first column of this lane's matrix
+                    const uint32_t addr = kt + (h0 >> 6) * kHalfBytes + krow * 128 + ((((h0 & 63) >> 3) ^ (krow & 7)) << 4);
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(addr, b0, b1, b2, b3);
+                    mma_16816(sc[nt][0], sc[nt][1], x2, x3, qa0[ks], qa2[ks], b0, b1);
+                    mma_16816(sc[nt][0], sc[nt][1], x2, x3, qa0[ks + 1], qa2[ks + 1], b2, b3);
+                }
+            }
+            // online softmax of this thread's row over the tile's 32 keys (the row is spread over 4 lanes)
+            float mx = -CUDART_INF_F;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int j = c0 + 8 * nt + qc + e;
+                    sc[nt][e] = (j < j1 && j <= lim) ? sc[nt][e] * scale_log2e : -CUDART_INF_F;
+                    mx = fmaxf(mx, sc[nt][e]);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m, mx);
+            const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
+            const float alpha = exp2_fast(m - m_use);
+            float sum = 0.f;
+            uint32_t pa[4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const float p0 = exp2_fast(sc[nt][0] - m_use), p1 = exp2_fast(sc[nt][1] - m_use);
+                sum += p0 + p1;
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                pa[nt] = *reinterpret_cast<const uint32_t*>(&pk);
+            }
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            l = fmaf(l, alpha, sum);
+            m = m_new;
+#pragma unroll
+            for (int nt = 0; nt < kNT; ++nt) { o[nt][0] *= alpha; o[nt][1] *= alpha; }
+            // O += P V: two k-steps of 16 keys; one transposed x4 load = (column tile nt, keys +0 / +8) and (nt + 1, ...)
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                const int vrow = 16 * kk + 8 * (lmat & 1) + lrow;
+#pragma unroll
+                for (int nt = 0; nt < kNT; nt += 2) {
+                    const int ch = nt + (lmat >> 1);                                   // 8-column chunk of the head dimension
+                    const uint32_t addr = vt + (ch >> 3) * kHalfBytes + vrow * 128 + (((ch & 7) ^ (vrow & 7)) << 4);
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                    mma_16816(o[nt][0], o[nt][1], x2, x3, pa[2 * kk], pa[2 * kk + 1], b0, b1);
+                    mma_16816(o[nt + 1][0], o[nt + 1][1], x2, x3, pa[2 * kk], pa[2 * kk + 1], b2, b3);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + 8 * st);
+        }
+    }
+    __syncthreads();   // every tile that was requested has been consumed (or the wait ran out): the ring is free
+    if (s_abort) {
+        if (tid == 0) {
+            atomicExch(status, WIDE_ERR_TIMEOUT);
+            volatile int never = 0;
+            for (int t = max(0, s_issued - kRingStages); t < s_issued; ++t)
+                mbar_wait(full + 8 * (t % kRingStages), (t / kRingStages) & 1, wait_ns, &never);
+        }
+        return;
+    }
+
+    // merge the four warps (their partial O goes through the ring's memory), write this slice's partial
+    float* wo = reinterpret_cast<float*>(ring);   // [kRingConsumers][8][HD]
+    if (warp < kRingConsumers && row_ok) {
+        if ((lane & 3) == 0) { wm[warp][qr] = m; wl[warp][qr] = l; }
+#pragma unroll
+        for (int nt = 0; nt < kNT; ++nt) {
+            wo[(warp * 8 + qr) * HD + 8 * nt + qc] = o[nt][0];
+            wo[(warp * 8 + qr) * HD + 8 * nt + qc + 1] = o[nt][1];
+        }
+    }
+    __syncthreads();
+    float* dst = part + (static_cast<size_t>(split) * Hkv + hkv) * R * (HD + 2);
+    for (int i = tid; i < R * HD; i += kRingThreads) {
+        const int r = i / HD, d = i % HD;
+        float mm = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kRingConsumers; ++w) mm = fmaxf(mm, wm[w][r]);
+        const float m_use = mm == -CUDART_INF_F ? 0.f : mm;
+        float acc = 0.f, ll = 0.f;
+#pragma unroll
+        for (int w = 0; w < kRingConsumers; ++w) {
+            const float al = exp2_fast(wm[w][r] - m_use);
+            acc = fmaf(wo[(w * 8 + r) * HD + d], al, acc);
+            ll = fmaf(wl[w][r], al, ll);
+        }
+        dst[r * (HD + 2) + 2 + d] = acc;
+        if (d == 0) {
+            dst[r * (HD + 2)] = mm;
+            dst[r * (HD + 2) + 1] = ll;
+        }
+    }
+}
+
 // One CTA per (token, query head): merge the key slices, normalise, write bf16; zeros for an
 // inactive (token, group) pair or a query that saw no key.
 template <int HD>
-__global__ void __launch_bounds__(HD)
+__global__ void __launch_bounds__(4 * HD)
 attn_decode_merge_kernel(const float* __restrict__ part, const uint32_t* __restrict__ mask_bits, int words, int Tq,
                          int Hq, int Hkv, int hpg, int n_splits_host, const int* __restrict__ hdr,
                          __nv_bfloat16* __restrict__ o) {
+    // 4 * HD threads: thread (quarter qt, dimension d) takes the slices qt, qt + 4, ...; all of its loads
+    // (at most kMaxSplits / 4) are requested before anything is used, so the kernel costs about one
+    // load latency whatever the number of slices.
+    constexpr int kPer = kMaxSplits / 4;
     const int n_splits = hdr ? *hdr : n_splits_host;
-    const int t = blockIdx.x / Hq, h = blockIdx.x % Hq, d = threadIdx.x;
+    const int t = blockIdx.x / Hq, h = blockIdx.x % Hq;
+    const int qt = threadIdx.x / HD, d = threadIdx.x % HD;
     const int rep = Hq / Hkv, R = Tq * rep;
     const int hkv = h / rep, r = t * rep + h % rep;
     __shared__ float s_m[kMaxSplits], s_w[kMaxSplits];
-    float out = 0.f;
-    if (wide_mask_bit(mask_bits, words, t, h / hpg)) {   // the same for the whole CTA
+    __shared__ float s_acc[4][HD], s_ll[4];
+    const bool on = wide_mask_bit(mask_bits, words, t, h / hpg);   // the same for the whole CTA
+    if (on) {
         const size_t stride = static_cast<size_t>(Hkv) * R * (HD + 2);
         const float* p0 = part + (static_cast<size_t>(hkv) * R + r) * (HD + 2);
-        // the slices' (m, l) first, all at once, so that the sums below wait for one load latency
-        for (int s = d; s < n_splits; s += HD) {
-            s_m[s] = __ldcg(p0 + s * stride);
-            s_w[s] = __ldcg(p0 + s * stride + 1);
+        for (int sp = threadIdx.x; sp < n_splits; sp += 4 * HD) {
+            s_m[sp] = __ldcg(p0 + sp * stride);
+            s_w[sp] = __ldcg(p0 + sp * stride + 1);
+        }
+        float vals[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int sp = qt + 4 * i;
+            vals[i] = sp < n_splits ? __ldcg(p0 + sp * stride + 2 + d) : 0.f;
         }
         __syncthreads();
         float mm = -CUDART_INF_F;
-        for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, s_m[s]);
+        for (int sp = 0; sp < n_splits; ++sp) mm = fmaxf(mm, s_m[sp]);
         const float m_use = mm == -CUDART_INF_F ? 0.f : mm;
         float acc = 0.f, ll = 0.f;
-#pragma unroll 16
-        for (int s = 0; s < n_splits; ++s) {
-            const float a = exp2_fast(s_m[s] - m_use);
-            acc = fmaf(__ldcg(p0 + s * stride + 2 + d), a, acc);
-            ll = fmaf(s_w[s], a, ll);
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+            const int sp = qt + 4 * i;
+            if (sp < n_splits) {
+                const float a = exp2_fast(s_m[sp] - m_use);
+                acc = fmaf(vals[i], a, acc);
+                ll = fmaf(s_w[sp], a, ll);
+            }
         }
-        out = ll > 0.f ? acc / ll : 0.f;
+        s_acc[qt][d] = acc;
+        if (d == 0) s_ll[qt] = ll;
+        __syncthreads();
     }
-    o[(static_cast<size_t>(t) * Hq + h) * HD + d] = __float2bfloat16_rn(out);
+    if (qt == 0) {
+        float out = 0.f;
+        if (on) {
+            const float acc = (s_acc[0][d] + s_acc[1][d]) + (s_acc[2][d] + s_acc[3][d]);
+            const float ll = (s_ll[0] + s_ll[1]) + (s_ll[2] + s_ll[3]);
+            out = ll > 0.f ? acc / ll : 0.f;
+        }
+        o[(static_cast<size_t>(t) * Hq + h) * HD + d] = __float2bfloat16_rn(out);
+    }
 }
 
 template <int HD>
@@ -556,7 +833,7 @@ int launch_attn_decode(wide_ctx* ctx, cudaStream_t s, const void* q, const void*
     }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     WideLaunch l(ctx, s, "attn_decode_merge");
-    attn_decode_merge_kernel<HD><<<Tq * Hq, HD, 0, s>>>(ctx->attn_part, mask_bits, words, Tq, Hq, Hkv, hpg, n_splits,
+    attn_decode_merge_kernel<HD><<<Tq * Hq, 4 * HD, 0, s>>>(ctx->attn_part, mask_bits, words, Tq, Hq, Hkv, hpg, n_splits,
                                                          nullptr, static_cast<__nv_bfloat16*>(o));
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
@@ -598,6 +875,32 @@ int launch_attn_decode_ring(wide_ctx* ctx, cudaStream_t s, const void* q, const 
     if (max_splits < 1) return WIDE_ERR_UNSUPPORTED_SHAPE;
     int* hdr = reinterpret_cast<int*>(reinterpret_cast<char*>(ctx->attn_part) + slab);
     int grid = 0;   // as many CTAs as are resident at once (set per instantiation below); never fewer than KV heads
+    if (R >= 2) {
+        // several query rows per KV head: the tensor-core form (tiles in the 128-byte swizzle)
+        CUtensorMap smK, smV;
+        if (!wide_make_tmap_bf16(ctx, &smK, k, static_cast<uint64_t>(Tk), static_cast<uint64_t>(Hkv) * HD, kRingKeys) ||
+            !wide_make_tmap_bf16(ctx, &smV, v, static_cast<uint64_t>(Tk), static_cast<uint64_t>(Hkv) * HD, kRingKeys))
+            return WIDE_ERR_CUDA;
+        constexpr int kSmemM = kRingStages * 2 * kRingKeys * HD * 2 + 1024;
+        WIDE_CUDA_CHECK(cudaFuncSetAttribute(attn_decode_ring_mma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kSmemM));
+        int per_sm = 0;
+        WIDE_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attn_decode_ring_mma_kernel<HD>, kRingThreads,
+                                                                      kSmemM));
+        grid = (per_sm > 0 ? per_sm : 1) * ctx->sm_count;
+        if (grid < Hkv) grid = Hkv;
+        {
+            WideLaunch l(ctx, s, "attn_decode");
+            attn_decode_ring_mma_kernel<HD><<<grid, kRingThreads, kSmemM, s>>>(
+                smK, smV, static_cast<const __nv_bfloat16*>(q), mask_bits, words, Tq, Tk, Hq, Hkv, hpg, causal,
+                scale * 1.4426950408889634f, max_splits, ctx->attn_part, hdr, ctx->d_status, ctx->wait_ns);
+        }
+        if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
+        WideLaunch l(ctx, s, "attn_decode_merge");
+        attn_decode_merge_kernel<HD><<<Tq * Hq, 4 * HD, 0, s>>>(ctx->attn_part, mask_bits, words, Tq, Hq, Hkv, hpg, 0, hdr,
+                                                             static_cast<__nv_bfloat16*>(o));
+        return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+    }
     constexpr int kSmem = kRingStages * 2 * kRingKeys * HD * 2 + 128;
     const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
     const float sl = scale * 1.4426950408889634f;
@@ -624,7 +927,7 @@ int launch_attn_decode_ring(wide_ctx* ctx, cudaStream_t s, const void* q, const 
     }
     if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
     WideLaunch l(ctx, s, "attn_decode_merge");
-    attn_decode_merge_kernel<HD><<<Tq * Hq, HD, 0, s>>>(ctx->attn_part, mask_bits, words, Tq, Hq, Hkv, hpg, 0, hdr,
+    attn_decode_merge_kernel<HD><<<Tq * Hq, 4 * HD, 0, s>>>(ctx->attn_part, mask_bits, words, Tq, Hq, Hkv, hpg, 0, hdr,
                                                          static_cast<__nv_bfloat16*>(o));
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
