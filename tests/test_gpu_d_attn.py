@@ -160,6 +160,8 @@ def test_attention_half_chain_stage_by_stage(ctx):
     (1, 17, 2, 2, 128, 1),         # fewer keys than one chunk
     (1, 20011, 8, 8, 128, 2),      # long cache: every warp goes round its ring stage several times
     (2, 9001, 8, 2, 64, 4),        # eight query rows per KV head, head_dim 64, many tiles
+    (1, 40000, 8, 2, 128, 4),      # grouped-query decode, long cache: every warp reuses its stage several times
+    (2, 30011, 8, 4, 64, 2),       # four rows per KV head, head_dim 64, long cache, ragged tail
 ])
 @pytest.mark.parametrize("causal", [True, False])
 @pytest.mark.parametrize("plain_loads", [False, True])
