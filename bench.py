@@ -527,13 +527,14 @@ def run_attn(args):
     ctx = binding.Context(local)
     T, hd = cfg.tokens, 128
     H = cfg.attn_dim // hd
+    Hkv = cfg.kv_heads or H                # grouped-query attention when fewer
     hpg = cfg.attn_group // hd
     NG, k = cfg.attn_n_groups, cfg.attn_k
     decode = T <= 8                       # --batch B: B new tokens against a resident K/V cache
     Tk = args.kv_len if args.kv_len else (synth.CONFIGS[args.workload].tokens if decode else T)
     oc = synth.make_oproj_case(cfg, 1000 * rank)
-    ac = synth.make_attn_case(1000 * rank, T, Tk, H, H, hd)
-    host = {"x": oc["x"], "q": ac["q"].reshape(T, H * hd), "k": ac["k"].reshape(Tk, H * hd), "v": ac["v"].reshape(Tk, H * hd)}
+    ac = synth.make_attn_case(1000 * rank, T, Tk, H, Hkv, hd)
+    host = {"x": oc["x"], "q": ac["q"].reshape(T, H * hd), "k": ac["k"].reshape(Tk, Hkv * hd), "v": ac["v"].reshape(Tk, Hkv * hd)}
     w_router = to_dev(oc["w_router_attn"], "bf16")
     pinned = {n: torch.from_numpy(synth.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).pin_memory() for n, a in host.items()}
     bufs = [{n: t.to(dev) for n, t in pinned.items()} for _ in range(2)]
@@ -544,7 +545,7 @@ def run_attn(args):
 
     def attn_only(slot=0):
         b = bufs[slot]
-        binding.wide_attn(ctx, b["q"], b["k"], b["v"], H, H, hpg, state["meta"], causal=True, o=obuf[slot],
+        binding.wide_attn(ctx, b["q"], b["k"], b["v"], H, Hkv, hpg, state["meta"], causal=True, o=obuf[slot],
                           mask_bits=bits if decode else None)
 
     def step(slot=0, kk=k):
@@ -656,7 +657,7 @@ def run_attn(args):
         ach = flops / (attn_ms * 1e-3) / 1e12
         if decode:
             # algorithmic bytes: K and V rows of every KV head some active query row reads
-            heads_read = int(np.repeat(mask.any(axis=0), hpg).sum())
+            heads_read = int(np.repeat(mask.any(axis=0), hpg).reshape(Hkv, H // Hkv).any(axis=1).sum())   # KV heads
             kv_bytes = 2.0 * heads_read * Tk * hd * 2
             roof = {"kernel": "attn_decode", "bound": "hbm", "achieved": kv_bytes / (attn_ms * 1e-3) / 1e9,
                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -672,10 +673,10 @@ def run_attn(args):
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "op": "attn", "tokens_per_gpu": T, "keys": Tk, "heads": H, "head_dim": hd,
+            "config": {"workload": cfg.name, "op": "attn", "tokens_per_gpu": T, "keys": Tk, "heads": H, "kv_heads": Hkv, "head_dim": hd,
                        "heads_per_group": hpg, "n_groups": NG, "k": k, "causal": True, "router": cfg.router,
                        "parallelism": f"sequence-sharded x{world} (independent sequences), no collective",
-                       "l2": "q, k, v, o of one step are %.0f MB (larger than L2)" % ((2 * T + 2 * Tk) * H * hd * 2 / 1e6)},
+                       "l2": "q, k, v, o of one step are %.0f MB" % ((2 * T * H + 2 * Tk * Hkv) * hd * 2 / 1e6)},
             "e2e": {"value": aggregate(T, e2e_steps, ms_e2e, world), "unit": "tokens/s",
                     "h2d_bytes_per_step": sum(t.numel() * 2 for n, t in pinned.items() if not (decode and n in ("k", "v"))),
                     "d2h_bytes_per_step": o_host[0].numel() * 2},

@@ -68,6 +68,7 @@ class WideConfig:
     attn_dim: int = 0      # H * d
     attn_group: int = 0    # heads_per_group * d
     attn_k: int = 0
+    kv_heads: int = 0      # KV heads of 128 (0: as many as query heads)
 
     @property
     def n_groups(self) -> int:
@@ -96,6 +97,10 @@ CONFIGS: Dict[str, WideConfig] = {
     # Llama-2-13B-shaped layer: head-group masked O-projection + FFN.
     "llama13b_layer": WideConfig("llama13b_layer", tokens=4096, hidden=5120, d_ff=13824,
                                  group=128, k=54, attn_dim=5120, attn_group=512, attn_k=5),
+    # Llama-3-8B-shaped layer: grouped-query attention (32 query heads on 8 KV heads of 128; a routing
+    # group = the 4 query heads of one KV head) + the 8B FFN.
+    "llama8b_layer": WideConfig("llama8b_layer", tokens=4096, hidden=4096, d_ff=14336,
+                                group=128, k=56, attn_dim=4096, attn_group=512, attn_k=4, kv_heads=8),
 }
 
 
