@@ -27,7 +27,8 @@
 // active query position of the tile (+ delta = T_k - T_q); only tiles that straddle a row's limit
 // evaluate element-wise predicates.
 //
-// Outputs of inactive (token, group) pairs are zeroed by a small kernel of its own.
+// Outputs of inactive (token, group) pairs are exact zeros, written by the CTAs of the tiles that hold no
+// (or not only) active rows before they do anything else.
 // Every mbarrier wait is bounded.
 #include <cuda.h>
 #include <math_constants.h>
@@ -80,22 +81,6 @@ constexpr int attn_smem_bytes() {
     return (HD / kBK) * kBlk + 4 * (HD / kBK) * kBlk + 2 * (kKV / kBK) * kBlk + 256 + 1024;
 }
 
-// o[row, heads of g, :] = 0 for every inactive (row, g) pair: sorted positions [counts[g], T_q).
-__global__ void __launch_bounds__(256)
-attn_zero_kernel(const int32_t* __restrict__ perm, const int32_t* __restrict__ counts, int Tq, int NG, int ppr,
-                 size_t ldq, __nv_bfloat16* __restrict__ o) {
-    // ppr = 16-byte pieces per (row, group); blockIdx.y = group
-    const int g = blockIdx.y;
-    const int c = counts[g];
-    const long long total = static_cast<long long>(Tq - c) * ppr;
-    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
-         i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int j = c + static_cast<int>(i / ppr), piece = static_cast<int>(i % ppr);
-        const int row = perm[static_cast<size_t>(g) * Tq + j];
-        reinterpret_cast<uint4*>(o + row * ldq + static_cast<size_t>(g) * ppr * 8)[piece] = make_uint4(0u, 0u, 0u, 0u);
-    }
-}
-
 // q [T_q, H_q*HD], o likewise; K/V come through the tensor maps ([T_k, H_kv*HD], box 64 x 128).
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -117,10 +102,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
     const int g = h / hpg;
     const int hkv = h / (Hq / Hkv);
     const int c = counts[g];
-    if (m * kQ >= c) return;   // block-level predicate: no active row in this tile
-    const int n_valid = min(kQ, c - m * kQ);
-    const int delta = Tk - Tq;
     const int32_t* rows = perm + static_cast<size_t>(g) * Tq + m * kQ;
+    // Block-level predicate: sorted positions >= counts[g] are the tokens that skip this head group, and
+    // their outputs are exact zeros.  A tile with no active row only writes those zeros (such tiles
+    // come first in the launch order and are gone at once); the tile that holds the boundary writes them
+    // for its inactive tail before it starts.
+    const int n_valid = max(0, min(kQ, c - m * kQ));
+    {
+        const int n_rows = min(kQ, Tq - m * kQ);
+        constexpr int kPieces = HD / 8;
+        for (int i = n_valid * kPieces + tid; i < n_rows * kPieces; i += kThreads) {
+            const int row = rows[i / kPieces];
+            reinterpret_cast<uint4*>(o + row * ldq + static_cast<size_t>(h) * HD)[i % kPieces] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    if (n_valid == 0) return;
+    const int delta = Tk - Tq;
     // key range: up to the largest active query position of the tile
     int j_max = Tk;
     if (causal) j_max = min(Tk, delta + 1 + rows[n_valid - 1]);
@@ -435,12 +432,6 @@ int launch_attn(wide_ctx* ctx, cudaStream_t s, const void* q, const void* k, con
     constexpr int smem = attn_smem_bytes<HD>();
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(attn_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     const int n_main = ((Tq + kQ - 1) / kQ) * Hq;
-    const int NG = Hq / hpg, ppr = hpg * HD / 8;
-    {
-        WideLaunch l(ctx, s, "attn_zero");
-        attn_zero_kernel<<<dim3(32, NG), 256, 0, s>>>(perm, counts, Tq, NG, ppr, static_cast<size_t>(Hq) * HD,
-                                                      static_cast<__nv_bfloat16*>(o));
-    }
     WideLaunch l(ctx, s, "attn_prefill");
     attn_kernel<HD><<<n_main, kThreads, smem, s>>>(
         tmK, tmV, static_cast<const __nv_bfloat16*>(q), perm, counts, Tq, Tk, Hq, Hkv, hpg, causal,
