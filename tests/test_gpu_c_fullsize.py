@@ -140,6 +140,46 @@ def test_llama13b_layer_attention_and_qproj(ctx):
     assert ctx.status() == 0
 
 
+def test_llama8b_layer_grouped_query_attention(ctx):
+    """Grouped-query attention at the 8B layer's full size: 32 query heads on 8 KV heads of 128, one
+    causal sequence of 4096 positions, 8 routing groups of 4 query heads, 4 active per token.  Prefill
+    form on three whole heads, decode form (one new token against the same 4096 keys) on every head."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.CONFIGS["llama8b_layer"]
+    T, hd = cfg.tokens, 128
+    H, Hkv, hpg, NG = cfg.attn_dim // hd, cfg.kv_heads, cfg.attn_group // hd, cfg.attn_n_groups
+    rep = H // Hkv
+    case = synth.make_oproj_case(cfg, 0)
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router_attn"]), cfg.attn_k)
+    bits = bits_to_dev(wo.pack_mask_bits(mask))
+    meta = binding.wide_reorder(ctx, bits, NG, 128)
+    ac = synth.make_attn_case(0, T, T, H, Hkv, hd)
+    qd, kd, vd = to_dev(ac["q"].reshape(T, -1), "bf16"), to_dev(ac["k"].reshape(T, -1), "bf16"), to_dev(ac["v"].reshape(T, -1), "bf16")
+    o = binding.wide_attn(ctx, qd, kd, vd, H, Hkv, hpg, meta)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    got = o.float().cpu().numpy().reshape(T, H, hd)
+    head_mask = np.repeat(mask, hpg, axis=1)
+    assert (got[~head_mask] == 0.0).all()
+    for h in (0, 13, 31):
+        g, kv = h // hpg, h // rep
+        ref = wo.masked_attention(ac["q"][:, h:h + 1], ac["k"][:, kv:kv + 1], ac["v"][:, kv:kv + 1], mask[:, g:g + 1], 1)
+        err = np.abs(got[:, h] - ref[:, 0]).max()
+        assert err <= REL_TOL * np.abs(ref).max(), f"head {h}: {err:.3e}"
+    # decode form: the last position as a new token against the whole cache
+    q1 = to_dev(ac["q"][T - 1:T].reshape(1, -1), "bf16")
+    m1 = mask[T - 1:T]
+    o1 = binding.wide_attn(ctx, q1, kd, vd, H, Hkv, hpg, None, causal=True, mask_bits=bits_to_dev(wo.pack_mask_bits(m1)))
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    ref1 = wo.masked_attention(ac["q"][T - 1:T], ac["k"], ac["v"], m1, hpg)
+    g1 = o1.float().cpu().numpy().reshape(1, H, hd)
+    assert (g1[~np.repeat(m1, hpg, axis=1)] == 0.0).all()
+    assert np.abs(g1 - ref1).max() <= REL_TOL * np.abs(ref1).max()
+    # and it is what the prefill form gave for that position
+    assert np.abs(g1[0] - got[T - 1]).max() <= REL_TOL * np.abs(ref1).max()
+
+
 def test_llama13b_layer_attention_decode_long_cache(ctx):
     """The decode form at the size the benchmark times: one new token against a cache of 32 768
     keys, 40 heads of 128, five of ten head groups active (both kernels: TMA ring and plain loads).
