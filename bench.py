@@ -31,14 +31,56 @@ from paper_2607_28418_b200 import synth  # noqa: E402
 
 METRIC = "masked-layer tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries
-# (profiles/), keyed by (kernel, workload); None until captured.
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the part's data-sheet figures (dense)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries,
+# keyed by (kernel, workload) -> (bytes, the summary under profiles/ it was read from).
 NCU_TRAFFIC_BYTES = {
-    ("prefill_gateup", "llama7b_prefill"): 355.4e6,
-    ("prefill_down", "llama7b_prefill"): 140.1e6,
+    ("prefill_gateup", "llama7b_prefill"): (355.4e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
+    ("prefill_down", "llama7b_prefill"): (140.1e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
     # decode: captured at batch 8 (union 111 groups, 357.3 MB); traffic is proportional to the union
-    ("decode_ffn_fused", "llama8b_decode"): 357.3e6 / 111,
+    ("decode_ffn_fused", "llama8b_decode"): (357.3e6 / 111, "profiles/decode_llama8b_batch8_fused_kernel.md"),
 }
+
+
+def ncu_traffic(kernel, workload, scale=1.0):
+    """(traffic bytes per launch or None, source file or None)."""
+    hit = NCU_TRAFFIC_BYTES.get((kernel, workload))
+    return (hit[0] * scale, hit[1]) if hit else (None, None)
+
+
+def roofline_record(kernel, bound, achieved, peaks, traffic=None, traffic_source=None, **extra):
+    """One roofline object: the fraction against the measured peak of this machine (the headline
+    `frac`) and against the part's nominal figure."""
+    key, unit = ("hbm_gbs", "GB/s") if bound == "hbm" else ("bf16_tflops", "TFLOP/s")
+    rec = {"kernel": kernel, "bound": bound, "achieved": achieved, "peak": peaks[key], "unit": unit,
+           "frac": achieved / peaks[key], "frac_measured": achieved / peaks[key],
+           "peak_nominal": NOMINAL_PEAKS[key], "frac_nominal": achieved / NOMINAL_PEAKS[key],
+           "traffic": traffic, "traffic_source": traffic_source, "peak_source": peaks["source"]}
+    rec.update(extra)
+    return rec
+
+
+def weight_copies(cfg, n_mats, flush_l2):
+    """Decode steps rotate over this many identical copies of the weights (> 4x L2 in all), so every
+    step streams its weights from HBM; prefill weights are larger than L2 by themselves."""
+    if cfg.tokens > 64 or flush_l2:
+        return 1
+    return max(2, -(-(640 << 20) // (n_mats * cfg.d_ff * cfg.hidden * 2)))
+
+
+def config_record(cfg, op, world, flush_l2=False):
+    """The workload description both arms print (same keys, same values).  `cfg` describes the
+    operation timed: for the attention-half operations d_ff / group / k are the attention
+    dimension, its group size and its budget."""
+    n_mats = 3 if op == "ffn" else 1
+    weights_mb = n_mats * cfg.d_ff * cfg.hidden * 2 / 1e6
+    n_copies = weight_copies(cfg, n_mats, flush_l2)
+    l2 = ("flushed between steps" if flush_l2 else
+          "weights rotate over %d copies (%.0f MB), every step streams from HBM" % (n_copies, n_copies * weights_mb)
+          if n_copies > 1 else "inputs larger than L2 (weights %.0f MB)" % weights_mb)
+    return {"workload": cfg.name, "op": op, "tokens_per_gpu": cfg.tokens, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
+            "group": cfg.group, "n_groups": cfg.n_groups, "k": cfg.k, "router": cfg.router,
+            "parallelism": f"token-sharded x{world}, weights replicated, no collective", "l2": l2}
 
 
 def load_peaks():
@@ -176,20 +218,131 @@ def run_reference(args):
     case = synth.make_ffn_case(cfg, 0, tokens=min(cfg.tokens, args.oracle_tokens))
     sample = min(cfg.tokens, args.oracle_tokens)
     steps = max(1, args.steps)
-    value, ms = time_oracle(case, cfg, sample, steps, min(args.warmup, 1))
+    warmup = max(3, args.warmup)
+    value, ms = time_oracle(case, cfg, sample, steps, warmup)
     cores = blas_threads()
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
-        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "tokens": cfg.tokens, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
-                   "group": cfg.group, "k": cfg.k, "router": cfg.router},
+        "config": config_record(cfg, args.op, world, args.flush_l2),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                          "sample": f"each step = the first {sample} of {cfg.tokens} tokens through route, top-k, "
                                    "reorder and the masked FFN in fp64 numpy"},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------- extra records
+def graph_of(torch, fn):
+    """Capture one call of fn (library calls only enqueue kernels on the current stream)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g.replay
+
+
+def event_ms(torch, fn, reps):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def sustained_record(torch, run_step, ms_hint, tokens, flops_ffn, peaks, gpu_index, seconds=2.0):
+    """The same step graph replayed back to back for `seconds`: what the path does once the part
+    has settled under its power cap, with the median SM clock seen meanwhile.  The fraction counts
+    the FFN's active FLOPs against the whole step (routing included), so it is a lower bound."""
+    reps = max(10, int(seconds / (ms_hint * 1e-3)))
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    ms = event_ms(torch, run_step, reps)
+    clocks = sampler.stop()
+    tfl = flops_ffn / (ms * 1e-3) / 1e12
+    peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    return {"seconds": round(reps * ms * 1e-3, 3), "replays": reps, "ms_per_step": ms, "value": tokens / (ms * 1e-3),
+            "unit": "tokens/s", "clocks": clocks, "ffn_active_tflops_over_step": tfl, "peak_sustained": peak,
+            "frac_of_sustained_peak": tfl / peak, "frac_of_nominal_peak": tfl / NOMINAL_PEAKS["bf16_tflops"]}
+
+
+def cublas_dense_context(torch, d, reps=10):
+    """Context only, not on the path: the dense SwiGLU FFN of the same shape through torch.matmul
+    (cuBLAS), the paper's own dense baseline for its kernel speed-ups."""
+    x, wg, wu, wd = d["x"], d["w_gate"], d["w_up"], d["w_down"]
+
+    def dense():
+        return (torch.nn.functional.silu(x @ wg.t()) * (x @ wu.t())) @ wd.t()
+    for _ in range(3):
+        dense()
+    ms = event_ms(torch, dense, reps)
+    return {"ms": ms, "what": "silu(x Wg^T) * (x Wu^T) then Wd^T through torch.matmul (cuBLAS), bf16; "
+                              "off the path, quoted beside the speed-up over our own dense run",
+            "dense_tflops": 6.0 * x.shape[0] * wg.shape[0] * x.shape[1] / (ms * 1e-3) / 1e12}
+
+
+def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 32, 64), replays=300):
+    """Llama-3-8B-shaped decode FFN (hidden 4096, d_ff 14336, 112 groups of 128, top-56, random
+    router) at each batch size: the FFN call replayed as a graph over two rotating copies of the
+    weights (704 MB > 4x L2, so every replay streams from HBM), and the whole step (route + FFN)."""
+    cfg = synth.CONFIGS["llama8b_decode"].with_(tokens=64)
+    case = synth.make_ffn_case(cfg, 0)
+    d = {k: binding.upload(v, "bf16") for k, v in case.items()}
+    wsets = [{k: d[k] for k in ("w_gate", "w_up", "w_down")}]
+    wsets.append({k: v.clone() for k, v in wsets[0].items()})
+    per_group = cfg.group * cfg.hidden * 2
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    out = []
+    for B in batches:
+        x = d["x"][:B].contiguous()
+        bits = torch.empty((B, (cfg.n_groups + 31) // 32), dtype=torch.int32, device=x.device)
+        y = torch.empty((B, cfg.hidden), dtype=torch.bfloat16, device=x.device)
+        binding.wide_route(ctx, x, d["w_router"], cfg.n_groups, cfg.k, mask_bits=bits)
+
+        def ffn(c):
+            w = wsets[c]
+            binding.wide_ffn(ctx, x, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, None, y=y)
+
+        def whole(c):
+            binding.wide_route(ctx, x, d["w_router"], cfg.n_groups, cfg.k, mask_bits=bits)
+            ffn(c)
+        for c in range(2):
+            ffn(c)
+        g_ffn = [graph_of(torch, lambda c=c: ffn(c)) for c in range(2)]
+        g_all = [graph_of(torch, lambda c=c: whole(c)) for c in range(2)]
+        state = {"i": 0}
+
+        def rot(graphs):
+            def run():
+                graphs[state["i"] & 1]()
+                state["i"] += 1
+            return run
+        event_ms(torch, rot(g_ffn), 6)
+        ffn_ms = event_ms(torch, rot(g_ffn), replays)
+        step_ms = event_ms(torch, rot(g_all), replays)
+        union_words = np.bitwise_or.reduce(bits.cpu().numpy().view(np.uint32), axis=0)
+        n_union = sum(bin(int(w)).count("1") for w in union_words)
+        gbs = 3.0 * n_union * per_group / (ffn_ms * 1e-3) / 1e9
+        out.append({"batch": B, "ffn_ms": ffn_ms, "step_ms": step_ms, "n_union": n_union, "achieved_gbs": gbs,
+                    "frac": gbs / peaks["hbm_gbs"], "frac_nominal": gbs / NOMINAL_PEAKS["hbm_gbs"],
+                    "tokens_per_s": B / (step_ms * 1e-3)})
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during the decode sweep")
+    clocks = sampler.stop()
+    return {"workload": "llama8b_decode", "router": "random", "k": cfg.k, "n_groups": cfg.n_groups,
+            "bytes": "union groups x 3 x group x hidden x 2 B (gate, up, down weights)", "peak": peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "replays": replays, "clocks": clocks, "points": out}
 
 
 # ------------------------------------------------------------------------------- our arm
@@ -240,10 +393,7 @@ def run_ours(args):
     # Decode: successive steps stand for successive layers of a model, each with its own weights.
     # The FFN weights rotate over several identical copies (> 4x L2 in total), so every step streams
     # its weights from HBM although the launches run back to back without an L2 flush in between.
-    n_copies = 1
-    if decode and not args.flush_l2:
-        per_copy = (1 if oproj else 3) * cfg.d_ff * cfg.hidden * 2
-        n_copies = max(2, -(-(640 << 20) // per_copy))
+    n_copies = weight_copies(cfg, 1 if oproj else 3, args.flush_l2)
     wkeys = ("w_q",) if qproj else ("w_o",) if oproj else ("w_gate", "w_up", "w_down")
     wsets = [{k: d[k] for k in wkeys}]
     for _ in range(n_copies - 1):
@@ -425,6 +575,15 @@ def run_ours(args):
                 dense_ms += timed(run_dense, 1) / dense_steps
         step()
 
+    # ---- extra records of the default single-GPU run: seconds-long replay, cuBLAS context, decode sweep
+    sustained = cublas = decode_rec = None
+    if world == 1 and not decode and not args.no_extras:
+        sustained = sustained_record(torch, run_step, ms_total / args.steps, T, flops_ffn_active(cfg, oproj), peaks, local)
+        if not oproj:
+            cublas = cublas_dense_context(torch, d)
+            if cfg.name == "llama7b_prefill":
+                decode_rec = decode_sweep(torch, binding, ctx, peaks, local)
+
     # ---- roofline of the dominant kernel (largest share of the timed region)
     kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
                    "share": round(v["total_ms"] / max(sum(p["total_ms"] for p in prof.values()), 1e-9), 4)}
@@ -443,17 +602,12 @@ def run_ours(args):
             per_group = cfg.group * cfg.hidden * 2
             bytes_alg = (1.0 if oproj else 3.0) * n_union * per_group   # weights of the groups in the union
             ach = bytes_alg / avg_s / 1e9
-            roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"],
-                        "traffic": (NCU_TRAFFIC_BYTES[(dom, cfg.name)] * n_union
-                                    if (dom, cfg.name) in NCU_TRAFFIC_BYTES else None),
-                        "peak_source": peaks["source"], "n_union": n_union}
+            tr, src = ncu_traffic(dom, cfg.name, n_union)
+            roofline = roofline_record(dom, "hbm", ach, peaks, tr, src, n_union=n_union)
         else:
             flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd}.get(dom, 2.0 * tkgd if oproj else 6.0 * tkgd)
-            ach = flops_alg / avg_s / 1e12
-            roofline = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                        "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                        "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.name)), "peak_source": peaks["source"]}
+            tr, src = ncu_traffic(dom, cfg.name)
+            roofline = roofline_record(dom, "tensor", flops_alg / avg_s / 1e12, peaks, tr, src)
 
     line = None
     if rank == 0:
@@ -463,13 +617,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "op": args.op, "tokens_per_gpu": T, "hidden": cfg.hidden, "d_ff": cfg.d_ff,
-                       "group": cfg.group, "n_groups": NG, "k": cfg.k, "router": cfg.router,
-                       "parallelism": f"token-sharded x{world}, weights replicated, no collective",
-                       "l2": "flushed between steps" if flush is not None else
-                             ("weights rotate over %d copies (%.0f MB), every step streams from HBM"
-                              % (n_copies, n_copies * 3 * cfg.d_ff * cfg.hidden * 2 / 1e6)) if n_copies > 1 else
-                             "inputs larger than L2 (weights %.0f MB)" % (3 * cfg.d_ff * cfg.hidden * 2 / 1e6)},
+            "config": config_record(cfg, args.op, world, args.flush_l2),
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": x_host.numel() * 2,
                     "d2h_bytes_per_step": y_host[0].numel() * 2,
                     "note": "activations cross PCIe every step (pinned host memory, copies of neighbouring "
@@ -486,6 +634,13 @@ def run_ours(args):
             "dense": {"ms_per_step": dense_ms, "speedup_vs_dense": (dense_ms / ms_step) if dense_ms else None,
                       "ideal": NG / cfg.k if cfg.k else None},
         }
+        if sustained:
+            line["sustained"] = sustained
+        if cublas:
+            cublas["speedup_of_masked_step_over_cublas_dense_ffn"] = cublas["ms"] / ms_step
+            line["cublas_dense_context"] = cublas
+        if decode_rec:
+            line["decode"] = decode_rec
         if world == 1 and not args.no_cpu_baseline and not oproj:
             sample = min(T, args.oracle_tokens)
             _, ms1 = time_oracle(case, cfg, sample, 1, 0)
@@ -659,13 +814,10 @@ def run_attn(args):
             # algorithmic bytes: K and V rows of every KV head some active query row reads
             heads_read = int(np.repeat(mask.any(axis=0), hpg).reshape(Hkv, H // Hkv).any(axis=1).sum())   # KV heads
             kv_bytes = 2.0 * heads_read * Tk * hd * 2
-            roof = {"kernel": "attn_decode", "bound": "hbm", "achieved": kv_bytes / (attn_ms * 1e-3) / 1e9,
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                    "traffic": None, "peak_source": peaks["source"], "kv_heads_read": heads_read}
+            roof = roofline_record("attn_decode", "hbm", kv_bytes / (attn_ms * 1e-3) / 1e9, peaks, kv_heads_read=heads_read)
         else:
-            roof = {"kernel": "attn_prefill", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                    "traffic": NCU_TRAFFIC_BYTES.get(("attn_prefill", cfg.name)), "peak_source": peaks["source"]}
+            tr, src = ncu_traffic("attn_prefill", cfg.name)
+            roof = roofline_record("attn_prefill", "tensor", ach, peaks, tr, src)
         kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
                        "share": round(v["total_ms"] / max(sum(p["total_ms"] for p in prof.values()), 1e-9), 4)}
                    for n, v in prof.items()}
@@ -725,6 +877,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of replaying a graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the seconds-long replay, the cuBLAS context row and the decode batch sweep")
     ap.add_argument("--oracle-tokens", type=int, default=4096, help="tokens of the workload the CPU oracle runs")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -96,7 +96,10 @@ WIDE_API int wide_destroy(wide_ctx* ctx);
 
 /* Synchronise `stream`, read the device status word into *status (WIDE_OK or
  * WIDE_ERR_TIMEOUT) and clear it; after a timeout the context's internal buffers are reset.
- * The only call that blocks the host. */
+ * The only call that blocks the host.
+ * After a device-side wait has expired the context's counters and accumulators are in an
+ * undefined state: until wide_status has been called, every decode-path call on the context
+ * finds the status word set when its kernel starts and returns without touching its outputs. */
 WIDE_API int wide_status(wide_ctx* ctx, void* stream, int* status);
 
 /* Override the bound of every device-side wait (nanoseconds; default 2e9). */
@@ -140,8 +143,10 @@ WIDE_API size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, 
  *
  * The selection equals the one taken on fp64 sums of the exact input products, so it does not
  * depend on summation order.  (bf16, TOPK, hidden % 64 == 0: scores come from the tensor cores in
- * fp32 and every group closer to the selection boundary than a proven error bound is re-scored
- * exactly in fp64; other cases, and WIDE_FLAG_SIMT, compute all scores in fp64.)
+ * fp32 and every group closer to the selection boundary than an error bound is re-scored exactly
+ * in fp64.  The bound assumes that the tensor-core accumulator loses at most 2^-23 of the running
+ * sum per accumulated element; the parity tests check the measured error against it.  Other
+ * cases, and WIDE_FLAG_SIMT, compute all scores in fp64.)
  *   x          [tokens, hidden]  dtype
  *   mask_bits  out uint32 [tokens, W]
  *   scores     out fp32 [tokens, n_groups] (TOPK) or [tokens, 2*n_groups] (PAIR), may be NULL
@@ -167,7 +172,9 @@ WIDE_API int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, i
  *     holds those 2 MiB until the process exits.
  *   - The first call on a device looks up the array's device address; it must be made with
  *     ctx's device current (else WIDE_ERR_INVALID_ARG) and should come before any stream
- *     capture.  Later calls reuse the cached address.
+ *     capture.  Later calls reuse the cached address.  The cache is written without a lock: host
+ *     threads that make that first call on one device at the same time all store the same
+ *     value, which is harmless.
  *   - All calls on a device share the one array.  Nothing in it needs clearing between calls
  *     (each call overwrites what it reads), but two calls that overlap on the GPU -- different
  *     streams, or different contexts of the same device -- race on it: serialise them.

@@ -181,9 +181,6 @@ class Context:
         _check(self.lib.wide_launch_count(self.handle, ctypes.byref(v)), "wide_launch_count")
         return int(v.value)
 
-    def set_wait_limit_ns(self, ns: int):
-        _check(self.lib.wide_set_wait_limit_ns(self.handle, ns), "wide_set_wait_limit_ns")
-
 
 def upload(a, dtype: str, device: Optional[torch.device] = None) -> torch.Tensor:
     """Host float32 array -> CUDA tensor of the workload dtype ("bf16": the values must already be

@@ -463,6 +463,9 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_consta
     __shared__ int s_nunion;
     __shared__ int s_flag;
     __shared__ unsigned s_tokmask[4];
+    // A wait that expired in an earlier kernel leaves the context's counters and sums dirty until
+    // wide_status resets them: with the status word set, this call does nothing at all.
+    if (*reinterpret_cast<volatile int*>(a.status) != WIDE_OK) return;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kRingBytesD);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStagesD + 4);

@@ -113,8 +113,11 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 // Cauchy-Schwarz bound on the sum of absolute products).  A group whose fp32 score is further
 // than 2*eps_t from the selection boundary keeps its fp32 decision; the few groups inside that
 // band get their score recomputed exactly in fp64, and the band is re-ranked on those exact
-// values.  The result equals the fp64 decision of the slow path.
-constexpr float kAccumErr = 5.9604645e-8f;  // 2^-24 per accumulated element
+// values.  The result equals the fp64 decision of the slow path provided the accumulator loses at
+// most 2^-23 of the running sum per step: the tensor core's accumulation order and rounding are
+// not specified (it may truncate where an FMA chain rounds to nearest, 2^-24), so the bound takes
+// the truncation figure; the measured error is two orders of magnitude below it.
+constexpr float kAccumErr = 1.1920929e-7f;  // 2^-23 per accumulated element
 
 constexpr int kSelTokens = 2;  // tokens per CTA in select_band_kernel (two warps each)
 constexpr int kBatch = 8;      // 16-byte loads in flight per lane and operand

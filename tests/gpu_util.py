@@ -44,3 +44,29 @@ def meta_to_dev(meta: dict) -> dict:
         "token_order": torch.from_numpy(meta["token_order"]).cuda(),
         "token_rank": torch.from_numpy(meta["token_rank"]).cuda(),
     }
+
+
+def ffn_ref_rows(case: dict, mask: np.ndarray, group: int, chunk: int = 1024) -> np.ndarray:
+    """The oracle's FFN over EVERY token row, computed a block of rows at a time (an output row
+    depends only on its own token and mask row, Eq. 3) so that the fp64 hidden activation of one
+    block, not of the whole batch, is alive at any moment."""
+    from oracle import wide_oracle as wo
+    T = case["x"].shape[0]
+    out = np.empty((T, case["w_down"].shape[0]), dtype=np.float64)
+    for r0 in range(0, T, chunk):
+        r1 = min(T, r0 + chunk)
+        out[r0:r1] = wo.ffn(case["x"][r0:r1], case["w_gate"], case["w_up"], case["w_down"], mask[r0:r1], group)
+    return out
+
+
+def assert_all_rows_close(y_gpu: torch.Tensor, y_ref: np.ndarray, what: str, rel: float = REL_TOL) -> float:
+    """Element-by-element comparison of the whole output: max|err| <= rel * max|ref|."""
+    got = y_gpu.float().cpu().numpy()
+    assert got.shape == y_ref.shape, f"{what}: shape {got.shape} vs {y_ref.shape}"
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    scale = float(np.abs(y_ref).max())
+    err = 0.0
+    for r0 in range(0, got.shape[0], 2048):       # blockwise: no second full-size fp64 temporary
+        err = max(err, float(np.abs(got[r0:r0 + 2048].astype(np.float64) - y_ref[r0:r0 + 2048]).max()))
+    assert err <= rel * scale + 1e-30, f"{what}: max|err| {err:.4e} > {rel} * max|ref| {scale:.4e}"
+    return err / scale if scale > 0 else 0.0

@@ -39,3 +39,30 @@ def test_expired_wait_sets_status_and_context_survives():
         assert ctx.status() == 0
     finally:
         ctx.close()
+
+
+def test_decode_calls_are_no_ops_until_the_status_is_read():
+    """After a wait has expired the decode path's counters and sums may be dirty; until
+    wide_status resets them a decode call must leave its output alone instead of adding to them."""
+    from paper_2607_28418_b200 import binding
+    ctx = binding.Context(0)
+    try:
+        cfg = synth.WideConfig("dirty", tokens=8, hidden=512, d_ff=1024, group=128, k=4)
+        case = synth.make_ffn_case(cfg, 6)
+        dev = {k: to_dev(v, cfg.dtype) for k, v in case.items()}
+        mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router"]), cfg.k)
+        bits = torch.from_numpy(wo.pack_mask_bits(mask).view(np.int32)).cuda()
+        ctx.set_wait_limit_ns(2_000_000)
+        ctx.selftest_wait()                                     # sets the status word, never read here
+        y = torch.full((8, 512), 7.0, dtype=torch.bfloat16, device="cuda")
+        binding.wide_ffn(ctx, dev["x"], dev["w_gate"], dev["w_up"], dev["w_down"], cfg.group, bits, None, y=y)
+        torch.cuda.synchronize()
+        assert (y == 7.0).all().item()                          # nothing was written
+        assert ctx.status() == binding.ERR_TIMEOUT
+        ctx.set_wait_limit_ns(2_000_000_000)
+        binding.wide_ffn(ctx, dev["x"], dev["w_gate"], dev["w_up"], dev["w_down"], cfg.group, bits, None, y=y)
+        ref = wo.ffn(case["x"], case["w_gate"], case["w_up"], case["w_down"], mask, cfg.group)
+        assert np.abs(y.float().cpu().numpy() - ref).max() <= 2e-2 * np.abs(ref).max()
+        assert ctx.status() == 0
+    finally:
+        ctx.close()

@@ -107,21 +107,24 @@ def test_constant_weight_closed_form():
         np.testing.assert_allclose(y[t], np.full(D, (t + 1) * G * h * w), rtol=1e-12)
 
 
-def test_n_axis_and_k_axis_gather_formulations_agree():
-    """Appendix A describes the same result as per-token gathers of the selected weight
-    groups (N-axis for gate/up, K-axis for down).  Written here from that description."""
+def test_per_token_selected_group_sums_agree():
+    """Appendix A states the pruned FFN per token: a token that selected R groups computes gate
+    and up only for the R*G channels of those groups and reduces the down projection over the
+    same channels.  Written here as plain loops over tokens, selected groups and channels."""
     x, wg, wu, wd = _tiny(7, T=7, D=6, NG=5, G=4)
-    R, G = 2, 4
-    mask = synth.random_mask(8, 7, 5, R)
-    sel = np.stack([np.nonzero(mask[t])[0] for t in range(7)])           # [M, R] group indices
-    chan = (sel[:, :, None] * G + np.arange(G)[None, None, :]).reshape(7, R * G)  # [M, R*G]
-    # N-axis: token-specific rows of gate / up, one dot product per selected channel
-    gate_sub = np.einsum("mk,mnk->mn", x, wg[chan])
-    up_sub = np.einsum("mk,mnk->mn", x, wu[chan])
-    h_sub = gate_sub / (1 + np.exp(-gate_sub)) * up_sub                  # [M, R*G]
-    # K-axis: the down projection reduces over the same selected channels only
-    wd_sub = np.transpose(wd[:, chan], (1, 0, 2))                         # [M, N, R*G]
-    y_ref = np.einsum("mk,mnk->mn", h_sub, wd_sub)
+    G = 4
+    mask = synth.random_mask(8, 7, 5, 2)
+    y_ref = np.zeros((7, wd.shape[0]))
+    for t in range(7):
+        for g in range(5):
+            if not mask[t, g]:
+                continue
+            for c in range(g * G, (g + 1) * G):
+                gate = sum(float(x[t, i]) * float(wg[c, i]) for i in range(6))
+                up = sum(float(x[t, i]) * float(wu[c, i]) for i in range(6))
+                h = gate / (1.0 + math.exp(-gate)) * up
+                for n in range(wd.shape[0]):
+                    y_ref[t, n] += h * float(wd[n, c])
     np.testing.assert_allclose(wo.ffn(x, wg, wu, wd, mask, G), y_ref, rtol=1e-12, atol=1e-14)
 
 

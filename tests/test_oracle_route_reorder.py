@@ -288,3 +288,21 @@ def test_gather_then_unpermute_masks_groupwise():
                 assert (blk == dense[t, g * G:(g + 1) * G]).all()
             else:
                 assert (blk == 0).all()
+
+
+def test_packed_layout_matches_hand_worked_fixture():
+    """gather_packed and unpermute each against a layout worked out by hand (Algorithm 2's scatter
+    epilogue): a mistake both functions share, e.g. in the row order of the packed buffer, would
+    survive the round-trip tests above but not this one."""
+    fx = _read_fixture(os.path.join(GOLDEN, "packed_hand_worked.txt"))
+    mask = np.array(fx["mask"], dtype=bool)
+    r = wo.reorder(mask, 2)
+    assert r["perm"].tolist() == fx["perm"]
+    assert r["counts"].tolist() == fx["counts"][0]
+    assert r["offsets"].tolist() == fx["offsets"][0]
+    dense = np.array(fx["dense"], dtype=np.float32)
+    packed = wo.gather_packed(dense, r["perm"], r["counts"], r["offsets"], 2)
+    assert packed.tolist() == fx["packed"]
+    back = wo.unpermute(np.array(fx["packed"], dtype=np.float32), np.array(fx["perm"], dtype=np.int32),
+                        np.array(fx["counts"][0]), np.array(fx["offsets"][0]), 5, 2)
+    assert back.tolist() == fx["scattered"]
