@@ -399,14 +399,19 @@ def run_ours(args):
     for _ in range(n_copies - 1):
         wsets.append({k: d[k].clone() for k in wkeys})
 
+    kflags = {"auto": 0, "group": binding.FLAG_KAXIS_GROUP, "owner": binding.FLAG_KAXIS_OWNER}[args.kaxis]
+    if args.reduce_bf16:
+        kflags |= binding.FLAG_REDUCE_BF16
+
     def main_op(x_in, w, y_out):
         if qproj:
             binding.wide_qproj(ctx, x_in, w["w_q"], cfg.group, meta, y=y_out)
         elif oproj:
             binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out,
-                               flags=binding.FLAG_INPUT_MASKED if args.premasked else 0)
+                               flags=(binding.FLAG_INPUT_MASKED if args.premasked else 0) | (0 if decode else kflags))
         else:
-            binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out)
+            binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out,
+                             flags=0 if decode else kflags)
     calls = {"n": 0}
 
     def step(k=cfg.k, slot=0, copy=None):
@@ -605,7 +610,7 @@ def run_ours(args):
             tr, src = ncu_traffic(dom, cfg.name, n_union)
             roofline = roofline_record(dom, "hbm", ach, peaks, tr, src, n_union=n_union)
         else:
-            flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd}.get(dom, 2.0 * tkgd if oproj else 6.0 * tkgd)
+            flops_alg = {"prefill_gateup": 4.0 * tkgd, "prefill_down": 2.0 * tkgd, "prefill_down_group": 2.0 * tkgd}.get(dom, 2.0 * tkgd if oproj else 6.0 * tkgd)
             tr, src = ncu_traffic(dom, cfg.name)
             roofline = roofline_record(dom, "tensor", flops_alg / avg_s / 1e12, peaks, tr, src)
 
@@ -872,6 +877,10 @@ def main():
                     help="oproj, qproj and attn need a workload with an attention half")
     ap.add_argument("--premasked", action="store_true",
                     help="oproj: feed an attention output that already has zeros for inactive pairs")
+    ap.add_argument("--kaxis", default="auto", choices=["auto", "group", "owner"],
+                    help="prefill K-axis kernel (down / output projection): per-group scatter-reduce, owner-computes, "
+                         "or the library's own choice")
+    ap.add_argument("--reduce-bf16", action="store_true", help="per-group K-axis kernel: add partial sums in bf16")
     ap.add_argument("--kv-len", type=int, default=0, help="attn: number of keys (default: the workload's tokens)")
     ap.add_argument("--flush-l2", action="store_true")
     ap.add_argument("--no-dense", action="store_true")

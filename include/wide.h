@@ -82,6 +82,16 @@ extern "C" {
                                       (token, group) pair, as wide_attn writes it; the prefill path then
                                       skips its masking pass (and the token clustering that rides on it) */
 
+#define WIDE_FLAG_KAXIS_GROUP 16u   /* wide_ffn / wide_oproj prefill: run the K-axis product in its per-group
+                                      form (Algorithm 3: only the active (tile, group) blocks, partial sums
+                                      reduced into the output), whatever the group size and active fraction */
+#define WIDE_FLAG_KAXIS_OWNER 32u   /* ... in its owner-computes form (a token tile walks all groups its
+                                      tokens use; no reduction traffic).  Default: chosen on the device from
+                                      the mask, see wide_oproj */
+#define WIDE_FLAG_REDUCE_BF16 64u   /* per-group form with a bf16 output: add the partial sums (one per active
+                                      group of a token) in bf16 straight into the output instead of in fp32
+                                      scratch; halves the reduction traffic.  Default when n_groups <= 16 */
+
 #define WIDE_DECODE_MAX_TOKENS 64
 #define WIDE_MAX_GROUPS 256
 
@@ -245,10 +255,21 @@ WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_
 /*
  * wide_oproj -- Eq. 2 / Eq. 10:  y[t,:] = sum_{g : M[t,g]=1} a[t, gG:(g+1)G] Wo[:, gG:(g+1)G]^T,
  * a = attention output flattened head-major [tokens, attn_dim], group g = channels [gG, (g+1)G).
- *   perm, counts: reserved (the current kernels do not read them; may be NULL).
- *   token_order, token_rank as for wide_ffn.
- *   WIDE_FLAG_INPUT_MASKED: see the flag; with an input that is not masked the result is the
- *       dense product for every token tile that uses the group at all.
+ *   perm, counts: outputs of wide_reorder for this mask, or both NULL.  The prefill path has two
+ *       K-axis kernels.  Per-group (Algorithm 3): for every active (128-row tile of a group's sorted
+ *       active rows, group) block, the block's partial product is reduced into y -- the FLOPs are
+ *       the active ones, the price is tokens * k * hidden partial sums through the L2 reduction
+ *       units.  Owner-computes: a token tile walks the groups any of its tokens uses -- no reduction
+ *       traffic, but nothing is skipped when every token has a mask of its own.  With perm / counts
+ *       given and group >= 256 (group >= 128 with WIDE_FLAG_REDUCE_BF16) the kernels choose between
+ *       the two on the device from the padded active fraction (no host read-back: the kernel that
+ *       is not chosen returns at once); without them, or with a smaller group, owner-computes runs.  WIDE_FLAG_KAXIS_GROUP /
+ *       WIDE_FLAG_KAXIS_OWNER override the choice, for wide_ffn's down projection as well.
+ *       The per-group kernel sums in fp32 (in y itself when out_dtype is fp32, else in scratch that
+ *       is converted at the end), or in bf16 straight into y when n_groups <= 16 or with
+ *       WIDE_FLAG_REDUCE_BF16.
+ *   token_order, token_rank as for wide_ffn (owner-computes kernel only).
+ *   WIDE_FLAG_INPUT_MASKED: see the flag.
  */
 WIDE_API int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
                int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,

@@ -31,6 +31,11 @@ size_t inner_scratch(int dtype, int tokens, int hidden, int inner) {
     return a > b ? a : b;
 }
 
+// fp32 sums [tokens, hidden] of the per-group K-axis kernel, behind the inner scratch
+size_t acc_scratch(int tokens, int hidden) {
+    return wide_align_up(static_cast<size_t>(tokens) * hidden * sizeof(float), 256);
+}
+
 }  // namespace
 
 extern "C" {
@@ -204,7 +209,7 @@ size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, int inner
     switch (op) {
         case WIDE_OP_ROUTE: return wide_route_workspace(tokens, n_groups, 64);
         case WIDE_OP_FFN:
-        case WIDE_OP_OPROJ: return inner_scratch(dtype, tokens, hidden, inner);
+        case WIDE_OP_OPROJ: return inner_scratch(dtype, tokens, hidden, inner) + acc_scratch(tokens, hidden);
         default: return 0;
     }
 }
@@ -263,7 +268,10 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
     if (!wide_aligned16(x) || !wide_aligned16(w_gate) || !wide_aligned16(w_up) || !wide_aligned16(w_down) ||
         !wide_aligned16(y) || !wide_aligned16(workspace))
         return WIDE_ERR_ALIGNMENT;
-    if (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, d_ff)) return WIDE_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, d_ff) + acc_scratch(tokens, hidden))
+        return WIDE_ERR_WORKSPACE;
+    if ((flags & WIDE_FLAG_KAXIS_GROUP) && (flags & WIDE_FLAG_KAXIS_OWNER)) return WIDE_ERR_INVALID_ARG;
+    void* acc = static_cast<uint8_t*>(workspace) + inner_scratch(dtype, tokens, hidden, d_ff);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (path) {
         case PATH_SIMT:
@@ -271,7 +279,7 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
                                         out_dtype, workspace);
         case PATH_PREFILL_TC:
             return wide_launch_ffn_prefill_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
-                                              perm, counts, token_order, token_rank, y, out_dtype, workspace);
+                                              perm, counts, token_order, token_rank, y, out_dtype, workspace, acc, flags);
         default:
             return wide_launch_ffn_decode_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
                                              y, out_dtype, workspace);
@@ -283,8 +291,9 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
                const int32_t* perm, const int32_t* counts, const int32_t* token_order,
                const int32_t* token_rank, void* y, int out_dtype, void* workspace,
                size_t workspace_bytes, unsigned flags) {
-    (void)perm; (void)counts;
     if ((token_order == nullptr) != (token_rank == nullptr)) return WIDE_ERR_INVALID_ARG;
+    if ((perm == nullptr) != (counts == nullptr)) return WIDE_ERR_INVALID_ARG;
+    if ((flags & WIDE_FLAG_KAXIS_GROUP) && ((flags & WIDE_FLAG_KAXIS_OWNER) || !perm)) return WIDE_ERR_INVALID_ARG;
     if (!ctx || !attn_out || !w_o || !mask_bits || !y) return WIDE_ERR_INVALID_ARG;
     if (!valid_dtype(dtype) || !valid_dtype(out_dtype)) return WIDE_ERR_INVALID_ARG;
     if (tokens < 0 || hidden <= 0 || attn_dim <= 0 || group <= 0 || attn_dim % group != 0) return WIDE_ERR_INVALID_ARG;
@@ -295,17 +304,17 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
     if (!wide_aligned16(attn_out) || !wide_aligned16(w_o) || !wide_aligned16(y) || !wide_aligned16(workspace))
         return WIDE_ERR_ALIGNMENT;
     if (path != PATH_SIMT &&
-        (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, attn_dim)))
+        (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, attn_dim) + acc_scratch(tokens, hidden)))
         return WIDE_ERR_WORKSPACE;
+    void* acc = workspace ? static_cast<uint8_t*>(workspace) + inner_scratch(dtype, tokens, hidden, attn_dim) : nullptr;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (path) {
         case PATH_SIMT:
             return wide_launch_oproj_simt(ctx, s, attn_out, w_o, dtype, tokens, hidden, attn_dim, group, mask_bits, y,
                                           out_dtype);
         case PATH_PREFILL_TC:
-            return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits,
-                                                token_order, token_rank, y, out_dtype, workspace,
-                                                (flags & WIDE_FLAG_INPUT_MASKED) != 0);
+            return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, perm,
+                                                counts, token_order, token_rank, y, out_dtype, workspace, acc, flags);
         default:
             return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
                                                out_dtype, workspace);

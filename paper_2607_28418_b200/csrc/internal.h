@@ -76,6 +76,26 @@ __device__ __forceinline__ bool wide_mask_bit(const uint32_t* mask_bits, int wor
     return (mask_bits[static_cast<size_t>(t) * words + (g >> 5)] >> (g & 31)) & 1u;
 }
 
+// Which K-axis kernel serves a prefill call is decided on the device, without a host read-back:
+// the per-group kernel (Algorithm 3: only active (tile, group) blocks, scatter-reduce into the
+// output) is chosen when the padded active fraction  sum_g ceil(counts[g]/128)*128 / (T*NG)  is at
+// most thr_q / 1024, the owner-computes kernel otherwise.  Every kernel of the pair evaluates this
+// same integer predicate when it starts; the one that is not chosen returns at once.
+// thr_q < 0: never the per-group kernel; thr_q >= 4096: always.  Warp-collective (all 32 lanes).
+#define WIDE_KAXIS_NEVER (-1)
+#define WIDE_KAXIS_ALWAYS 4096
+#ifdef __CUDACC__
+__device__ __forceinline__ bool wide_kaxis_group_chosen(const int32_t* __restrict__ counts, int NG, int T, int thr_q) {
+    if (counts == nullptr || thr_q < 0) return false;
+    if (thr_q >= WIDE_KAXIS_ALWAYS) return true;
+    long long tiles = 0;
+    for (int g = threadIdx.x & 31; g < NG; g += 32) tiles += (counts[g] + 127) >> 7;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
+    return tiles * 128 * 1024 <= static_cast<long long>(thr_q) * T * NG;
+}
+#endif
+
 // ---- launchers (each returns WIDE_OK or WIDE_ERR_CUDA; arguments already validated)
 int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, int T, int D,
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
@@ -97,19 +117,31 @@ int wide_launch_ffn_simt(wide_ctx* ctx, cudaStream_t s, const void* x, const voi
 int wide_launch_oproj_simt(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int dtype, int T, int D,
                            int K, int G, const uint32_t* mask_bits, void* y, int out_dtype);
 
-// tcgen05 prefill path (bf16).  `h` is scratch [T, Dff] bf16.
+// tcgen05 prefill path (bf16).  `h` is scratch [T, Dff] bf16, `acc` scratch [T, D] fp32 (used when
+// the per-group K-axis kernel reduces in fp32 towards a bf16 output).
 int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg,
                                const void* wu, const void* wd, int T, int D, int Dff, int G,
                                const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
                                const int32_t* token_order, const int32_t* token_rank, void* y,
-                               int out_dtype, void* h);
+                               int out_dtype, void* h, void* acc, unsigned flags);
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
                           int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out);
-// `a_masked` is scratch [T, K] bf16.
+// `a_masked` is scratch [T, K] bf16, `acc` scratch [T, D] fp32.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
-                                 int D, int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
-                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked,
-                                 bool input_masked);
+                                 int D, int K, int G, const uint32_t* mask_bits, const int32_t* perm,
+                                 const int32_t* counts, const int32_t* token_order,
+                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked, void* acc,
+                                 unsigned flags);
+
+// Per-group GEMM-K (Algorithm 3) and its helpers, csrc/gemmk_group.cu.
+int wide_launch_kaxis_prep(wide_ctx* ctx, cudaStream_t s, const int32_t* counts, int NG, int T, int thr_q, void* zero_ptr,
+                           size_t zero_bytes, const void* a, const uint32_t* mask_bits, const int32_t* token_rank, int K,
+                           int G, void* a_masked);
+int wide_launch_gemmk_group_tc(wide_ctx* ctx, cudaStream_t s, const void* A, int lda, const void* B, int T, int N, int K,
+                               int G, const int32_t* perm, const int32_t* counts, const int32_t* a_row_of_token, void* Y,
+                               bool bf16_red, int thr_q, const char* name);
+int wide_launch_kaxis_convert(wide_ctx* ctx, cudaStream_t s, const int32_t* counts, int NG, int T, int thr_q,
+                              const float* acc, void* y_bf16, size_t n_elems);
 
 // tcgen05 decode path (bf16, T <= WIDE_DECODE_MAX_TOKENS).
 size_t wide_decode_workspace(int T, int D, int inner);

@@ -108,10 +108,12 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N, int K,
             int G, void* __restrict__ Y,
             int out_bf16, int ksplit, const __nv_bfloat16* __restrict__ aux_w, int aux_rows,
-            float* __restrict__ aux_norm, int* __restrict__ status, unsigned long long wait_ns) {
+            float* __restrict__ aux_norm, const int32_t* __restrict__ sel_counts, int sel_thr,
+            int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
+    if (wide_kaxis_group_chosen(sel_counts, K / G, T, sel_thr)) return;   // the per-group kernel runs instead
     SmemLayout L = carve_smem<kBBytes>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -322,9 +324,10 @@ __global__ void __launch_bounds__(192, 1)
 down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N,
                int K, int G, void* __restrict__ Y,
-               int out_bf16, int n_n, int box_n, unsigned* __restrict__ queue, int* __restrict__ status,
-               unsigned long long wait_ns) {
+               int out_bf16, int n_n, int box_n, unsigned* __restrict__ queue, const int32_t* __restrict__ sel_counts,
+               int sel_thr, int* __restrict__ status, unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
+    if (wide_kaxis_group_chosen(sel_counts, K / G, T, sel_thr)) return;   // the per-group kernel runs instead
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(base + kStages2 * kStage2Bytes);
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + kStages2);
@@ -939,21 +942,6 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
     }
 }
 
-// H~[t, c] = M[t, c/G] ? a[t, c] : 0   (16-byte pieces; G*2 bytes is a multiple of 16)
-__global__ void __launch_bounds__(256) mask_rows_kernel(const uint4* __restrict__ a, const uint32_t* __restrict__ mask_bits,
-                                                        const int32_t* __restrict__ token_rank, int words, int T, int K,
-                                                        int G, uint4* __restrict__ out) {
-    const int vec_per_row = K / 8, vec_per_group = G / 8;
-    const long long total = static_cast<long long>(T) * vec_per_row;
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int t = static_cast<int>(i / vec_per_row);
-        const int g = static_cast<int>(i % vec_per_row) / vec_per_group;
-        const long long o = token_rank ? static_cast<long long>(token_rank[t]) * vec_per_row + (i % vec_per_row) : i;
-        out[o] = wide_mask_bit(mask_bits, words, t, g) ? a[i] : make_uint4(0u, 0u, 0u, 0u);
-    }
-}
-
 // --------------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -977,7 +965,8 @@ bool make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uin
 template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                 int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down",
-                int ksplit = 1, float* aux_norm = nullptr, const int32_t* order = nullptr) {
+                int ksplit = 1, float* aux_norm = nullptr, const int32_t* order = nullptr,
+                const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER) {
     CUtensorMap tmA, tmB;
     if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
@@ -989,7 +978,7 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, name);
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
-                                            ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm,
+                                            ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm, sel_counts, sel_thr,
                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
@@ -1014,14 +1003,16 @@ double pick_down256_tiling(int sm, int T, int N, int* n_n_out, int* wmax_out) {
 // Picks the tile height for the down / output projection: 256-row tiles move fewer bytes per FLOP
 // (about 0.8 of the time per row), 128-row tiles quantise better over the SMs.
 int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
-                     int N, int K, int G, void* Y, int out_dtype, const int32_t* order) {
+                     int N, int K, int G, void* Y, int out_dtype, const int32_t* order,
+                     const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER) {
     const int sm = ctx->sm_count;
     const int t128 = ((T + 127) / 128) * ((N + 255) / 256);
     int n_n = (N + 255) / 256, wmax = 256;
     const double cost128 = static_cast<double>((t128 + sm - 1) / sm);
     const double cost256 = pick_down256_tiling(sm, T, N, &n_n, &wmax) * 2.0 * 0.8;
     if (cost128 <= cost256)
-        return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype, -1, "prefill_down", 1, nullptr, order);
+        return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype, -1, "prefill_down", 1, nullptr, order,
+                                sel_counts, sel_thr);
     CUtensorMap tmA, tmB;
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, 256) || !make_tmap_bf16(ctx, &tmB, B, N, K, wmax)) return WIDE_ERR_CUDA;
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2));
@@ -1030,8 +1021,8 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
     down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
-                                             n_n, wmax, reinterpret_cast<unsigned*>(ctx->d_status) + 8, ctx->d_status,
-                                             ctx->wait_ns);
+                                             n_n, wmax, reinterpret_cast<unsigned*>(ctx->d_status) + 8, sel_counts, sel_thr,
+                                             ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -1050,6 +1041,73 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
+// Which K-axis kernel a prefill call uses.  Measured on the 13B output projection and on the 8B down
+// projection (T = 4096): the per-group kernel (Algorithm 3) costs c * p of the owner-computes kernel's
+// time, p = padded active fraction, with c = 1.35 (G = 512, bf16 sums), 2.1 (256, bf16), 3.5 (256,
+// fp32 sums incl. clearing and converting the scratch), 3.7 (128, bf16): c = 0.6 + 380 * (bytes / 2) / G
+// fits all four.  The first term is the tensor work (128 x 256 tiles move more operand bytes per
+// FLOP than the owner kernel's 256 x 256), the second the T*k*N partial sums that go through the
+// L2's reduction units.  The per-group kernel is taken when c * p <= 0.9.  Group sizes below 256
+// take part in the device-side choice only when the caller opts into bf16 sums; otherwise the choice
+// would add two empty launches to every call that stays with the owner-computes kernel.
+struct KaxisPlan {
+    int thr_q;       // threshold of wide_kaxis_group_chosen
+    bool bf16_red;   // reduce straight into the bf16 output
+    bool use_acc;    // reduce in fp32 into scratch, then convert
+};
+
+KaxisPlan plan_kaxis(int G, int NG, int out_dtype, bool have_perm, unsigned flags) {
+    KaxisPlan p;
+    p.bf16_red = out_dtype == WIDE_BF16 && ((flags & WIDE_FLAG_REDUCE_BF16) || NG <= 16);
+    p.use_acc = out_dtype == WIDE_BF16 && !p.bf16_red;
+    if (!have_perm || (flags & WIDE_FLAG_KAXIS_OWNER)) {
+        p.thr_q = WIDE_KAXIS_NEVER;
+    } else if (flags & WIDE_FLAG_KAXIS_GROUP) {
+        p.thr_q = WIDE_KAXIS_ALWAYS;
+    } else if (G >= 256 || (G >= 128 && (flags & WIDE_FLAG_REDUCE_BF16))) {
+        const double c = 0.6 + 380.0 * (p.bf16_red ? 1.0 : 2.0) / G;
+        p.thr_q = static_cast<int>(1024.0 * 0.9 / c);
+    } else {
+        p.thr_q = WIDE_KAXIS_NEVER;
+    }
+    return p;
+}
+
+// The K-axis product y = A (.)_G M  B^T shared by the down projection and the output projection.
+//   a_rows      [T, K] rows the per-group kernel gathers (row a_row_of_token[t] holds token t)
+//   a_owner     [T, K] operand of the owner-computes kernel: zeros for inactive pairs, rows in
+//               `order`; when a_unmasked is given it is written here first (masking pass)
+int launch_kaxis(wide_ctx* ctx, cudaStream_t s, const KaxisPlan& plan, const void* a_rows, const int32_t* a_row_of_token,
+                 const void* a_unmasked, void* a_owner, const void* B, int T, int N, int K, int G,
+                 const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts, const int32_t* order,
+                 const int32_t* rank, void* y, int out_dtype, void* acc, const char* group_name) {
+    const int NG = K / G;
+    int rc;
+    if (plan.thr_q == WIDE_KAXIS_NEVER) {
+        if (a_unmasked) {
+            rc = wide_launch_kaxis_prep(ctx, s, nullptr, NG, T, plan.thr_q, nullptr, 0, a_unmasked, mask_bits, rank, K, G, a_owner);
+            if (rc != WIDE_OK) return rc;
+        }
+        return launch_down_auto(ctx, s, a_owner, B, mask_bits, T, N, K, G, y, out_dtype, order);
+    }
+    void* target = plan.use_acc ? acc : y;
+    const size_t target_bytes = static_cast<size_t>(T) * N * (plan.bf16_red ? 2 : 4);
+    const bool always = plan.thr_q >= WIDE_KAXIS_ALWAYS;
+    rc = wide_launch_kaxis_prep(ctx, s, counts, NG, T, plan.thr_q, target, target_bytes, always ? nullptr : a_unmasked,
+                                mask_bits, rank, K, G, a_owner);
+    if (rc != WIDE_OK) return rc;
+    rc = wide_launch_gemmk_group_tc(ctx, s, a_rows, K, B, T, N, K, G, perm, counts, a_row_of_token, target, plan.bf16_red,
+                                    plan.thr_q, group_name);
+    if (rc != WIDE_OK) return rc;
+    if (!always) {
+        rc = launch_down_auto(ctx, s, a_owner, B, mask_bits, T, N, K, G, y, out_dtype, order, counts, plan.thr_q);
+        if (rc != WIDE_OK) return rc;
+    }
+    if (plan.use_acc) return wide_launch_kaxis_convert(ctx, s, counts, NG, T, plan.thr_q, static_cast<const float*>(acc), y,
+                                                       static_cast<size_t>(T) * N);
+    return WIDE_OK;
+}
+
 }  // namespace
 
 bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
@@ -1060,15 +1118,18 @@ bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base
 int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
                                const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
                                const int32_t* perm, const int32_t* counts, const int32_t* token_order,
-                               const int32_t* token_rank, void* y, int out_dtype, void* h) {
+                               const int32_t* token_rank, void* y, int out_dtype, void* h, void* acc, unsigned flags) {
     if (T == 0) return WIDE_OK;
     // H [T, Dff] is kept in clustered token order when token_order / token_rank are given (row
     // token_rank[t] holds token t), else in token order.  Inactive (token, group) pairs of H must
-    // read as zero in the down projection: the gate/up kernel's epilogue warps write those zeros.
+    // read as zero in the owner-computes down projection: the gate/up kernel's epilogue warps write
+    // those zeros.  The per-group down projection gathers active rows only.
     int rc = (G == 64) ? launch_gateup<64, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h)
                        : launch_gateup<128, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h);
     if (rc != WIDE_OK) return rc;
-    return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, y, out_dtype, token_order);
+    const KaxisPlan plan = plan_kaxis(G, Dff / G, out_dtype, true, flags);
+    return launch_kaxis(ctx, s, plan, h, token_rank, nullptr, h, wd, T, D, Dff, G, mask_bits, perm, counts, token_order,
+                        token_rank, y, out_dtype, acc, "prefill_down_group");
 }
 
 // y[t, gG:(g+1)G] = x_t W[gG:(g+1)G, :]^T for active (t, g), exact zeros elsewhere (Algorithm 2 with a
@@ -1081,23 +1142,20 @@ int wide_launch_linear_mn_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const
 }
 
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T, int D,
-                                 int K, int G, const uint32_t* mask_bits, const int32_t* token_order,
-                                 const int32_t* token_rank, void* y, int out_dtype, void* a_masked,
-                                 bool input_masked) {
+                                 int K, int G, const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
+                                 const int32_t* token_order, const int32_t* token_rank, void* y, int out_dtype,
+                                 void* a_masked, void* acc, unsigned flags) {
     if (T == 0) return WIDE_OK;
-    // an input that already has zeros for the inactive pairs is the GEMM operand as it stands
-    if (input_masked) return launch_down_auto(ctx, s, a, wo, mask_bits, T, D, K, G, y, out_dtype, nullptr);
-    const int words = (K / G + 31) / 32;
-    const long long total = static_cast<long long>(T) * (K / 8);
-    long long blocks = (total + 255) / 256;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    {
-    WideLaunch l(ctx, s, "prefill_mask_rows");
-    mask_rows_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(static_cast<const uint4*>(a), mask_bits, token_rank, words,
-                                                              T, K, G, static_cast<uint4*>(a_masked));
-    }
-    if (cudaGetLastError() != cudaSuccess) return WIDE_ERR_CUDA;
-    return launch_down_auto(ctx, s, a_masked, wo, mask_bits, T, D, K, G, y, out_dtype, token_order);
+    const KaxisPlan plan = plan_kaxis(G, K / G, out_dtype, perm != nullptr && counts != nullptr, flags);
+    // The per-group kernel gathers active rows of the input as it stands.  The owner-computes kernel
+    // needs zeros for the inactive pairs: an input that already has them is its operand as it
+    // stands (tokens in their own order), any other input goes through the masking pass first (and
+    // lands in clustered token order when one is given).
+    if (flags & WIDE_FLAG_INPUT_MASKED)
+        return launch_kaxis(ctx, s, plan, a, nullptr, nullptr, const_cast<void*>(a), wo, T, D, K, G, mask_bits, perm, counts,
+                            nullptr, nullptr, y, out_dtype, acc, "prefill_oproj_group");
+    return launch_kaxis(ctx, s, plan, a, nullptr, a, a_masked, wo, T, D, K, G, mask_bits, perm, counts, token_order,
+                        token_rank, y, out_dtype, acc, "prefill_oproj_group");
 }
 
 // scores (fp32) = x[T, D] * w_router[NG, D]^T on the tensor cores, K split `ksplit` ways: slab ks
