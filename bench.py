@@ -661,6 +661,100 @@ def run_ours(args):
     return line
 
 
+# ------------------------------------------------------------------------------- group-sharded FFN
+def run_group_sharded(args):
+    """--shard groups: tensor parallelism over the pruned dimension.  Every rank holds the gate / up
+    rows and the down columns of its contiguous range of groups, routes all tokens (replicated),
+    slices the mask to its range, runs reorder + wide_ffn on its shard with an fp32 output, and the
+    parts are summed by one NCCL reduce-scatter over the token rows (Eq. 10: the K-axis product is a
+    sum over groups).  Total work is fixed as N grows (strong scaling)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_28418_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    cfg = make_config(args)
+    peaks = load_peaks()
+    ctx = binding.Context(local)
+    T, NG, G = cfg.tokens, cfg.n_groups, cfg.group
+    if T % world:
+        raise SystemExit("--shard groups needs tokens divisible by the number of ranks")
+    case = synth.make_ffn_case(cfg, 0)                      # the same inputs on every rank
+    g0, g1 = binding.group_range(NG, world, rank)
+    c0, c1 = g0 * G, g1 * G
+    x = binding.upload(case["x"], "bf16")
+    w_router = binding.upload(case["w_router"], "bf16")
+    wg, wu = binding.upload(case["w_gate"][c0:c1], "bf16"), binding.upload(case["w_up"][c0:c1], "bf16")
+    wd = binding.upload(np.ascontiguousarray(case["w_down"][:, c0:c1]), "bf16")
+    bits = torch.empty((T, (NG + 31) // 32), dtype=torch.int32, device=dev)
+    local_bits = torch.empty((T, max(1, (g1 - g0 + 31) // 32)), dtype=torch.int32, device=dev)
+    part = torch.empty((T, cfg.hidden), dtype=torch.float32, device=dev)
+    rows = torch.empty((T // world, cfg.hidden), dtype=torch.float32, device=dev)
+    y = torch.empty((T // world, cfg.hidden), dtype=torch.bfloat16, device=dev)
+    state = {"meta": None}
+
+    def step():
+        binding.wide_route(ctx, x, w_router, NG, cfg.k, mask_bits=bits)
+        binding.wide_mask_slice(ctx, bits, NG, g0, g1, out=local_bits)
+        if T > binding.DECODE_MAX_TOKENS:
+            state["meta"] = binding.wide_reorder(ctx, local_bits, g1 - g0, 128, out=state["meta"])
+        binding.wide_ffn(ctx, x, wg, wu, wd, G, local_bits, state["meta"], y=part)
+        if world > 1:
+            dist.reduce_scatter_tensor(rows, part, op=dist.ReduceOp.SUM)
+            y.copy_(rows)
+        else:
+            y.copy_(part)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during warm-up")
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    sync_all()
+    ms_total = reduce_max_ms(e0.elapsed_time(e1), world, dev)
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        tfl = flops_ffn_active(cfg) / (ms_step * 1e-3) / 1e12
+        rec = config_record(cfg, "ffn", world, args.flush_l2)
+        rec["parallelism"] = (f"group-sharded x{world}: each rank holds the weights of a contiguous range of groups, routing "
+                              "replicated, fp32 parts summed by one NCCL reduce-scatter over token rows")
+        print(json.dumps({
+            "metric": METRIC, "value": T * args.steps / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": rec,
+            "launch": "direct launches", "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": roofline_record("whole step (all ranks)", "tensor", tfl, {**peaks, "bf16_tflops": peaks["bf16_tflops"] * world}),
+            "note": "the multi-GPU form of this mode has not been run on more than one GPU in this build"}))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------------------- attention op
 def run_attn(args):
     """--op attn: route (attention router) -> reorder -> head-group-masked causal attention on the
@@ -875,6 +969,9 @@ def main():
     ap.add_argument("--group", type=int, default=0)
     ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn", "qproj"],
                     help="oproj, qproj and attn need a workload with an attention half")
+    ap.add_argument("--shard", default="tokens", choices=["tokens", "groups"],
+                    help="multi-GPU partition: token shards with replicated weights (no collective), or group "
+                         "shards (tensor parallel over the pruned dimension) with one reduce-scatter per step")
     ap.add_argument("--premasked", action="store_true",
                     help="oproj: feed an attention output that already has zeros for inactive pairs")
     ap.add_argument("--kaxis", default="auto", choices=["auto", "group", "owner"],
@@ -892,6 +989,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard == "groups":
+        run_group_sharded(args)
     elif args.op == "attn":
         run_attn(args)
     else:

@@ -229,6 +229,23 @@ WIDE_API int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits
                  int32_t* token_order, int32_t* token_rank);
 
 /*
+ * wide_mask_slice -- the columns [group_begin, group_end) of a routing mask as a mask of their own
+ * (bit g - group_begin of the output row = bit g of the input row, unused high bits 0).
+ *
+ * This is the mask a rank needs when the groups are sharded over GPUs (tensor parallelism over the
+ * pruned dimension): Eq. 10 writes the K-axis product as a sum over groups, so the rank that holds
+ * the gate / up rows and the down (or output-projection) columns of groups [group_begin, group_end)
+ * computes its part of y by calling wide_reorder, wide_ffn / wide_oproj on ITS weight shard
+ * (d_ff = (group_end - group_begin) * group, contiguous) with the sliced mask and an fp32 output;
+ * the parts of all ranks add up to the full result (one reduce-scatter or all-reduce, the
+ * caller's).  Routing itself is replicated: every rank scores all groups.
+ *   mask_bits [tokens, ceil(n_groups/32)], out_bits out [tokens, ceil((group_end-group_begin)/32)]
+ * Errors: INVALID_ARG (null pointer, range outside [0, n_groups]), UNSUPPORTED_SHAPE.
+ */
+WIDE_API int wide_mask_slice(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
+                             int group_begin, int group_end, uint32_t* out_bits);
+
+/*
  * wide_ffn -- Eq. 3:  y = ((silu(x Wg^T) * (x Wu^T)) (.)_G M) Wd^T.
  * Gate/up columns and down rows of inactive (token, group) pairs are skipped (block level) or
  * contribute exact zeros (inside an active tile).

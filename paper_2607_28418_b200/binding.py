@@ -27,7 +27,8 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, 
 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
            "wide_profile_end", "wide_launch_count", "wide_selftest_wait", "wide_strerror",
-           "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_ffn",
+           "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_mask_slice",
+           "wide_ffn",
            "wide_oproj", "wide_attn", "wide_qproj", "wide_unpermute"]
 
 _c_void_p, _c_int, _c_size_t, _c_uint = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
@@ -69,6 +70,7 @@ def load_library() -> ctypes.CDLL:
                                _c_size_t, _c_uint]
     lib.wide_route_static.argtypes = lib.wide_route.argtypes[:15] + [_c_uint]
     lib.wide_reorder.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int] + [_c_void_p] * 10
+    lib.wide_mask_slice.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_void_p]
     lib.wide_ffn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int,
                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                              _c_void_p, _c_int, _c_void_p, _c_size_t, _c_uint]
@@ -264,6 +266,24 @@ def wide_reorder(ctx: Context, mask_bits: torch.Tensor, n_groups: int, tile_m: i
                               _ptr(out["n_work"]), _ptr(out["union_list"]), _ptr(out["n_union"]),
                               _ptr(out["offsets"]), _ptr(out.get("token_order")), _ptr(out.get("token_rank")))
     _check(rc, "wide_reorder")
+    return out
+
+
+def group_range(n_groups: int, world: int, rank: int):
+    """Groups [begin, end) owned by `rank` when n_groups are dealt to `world` ranks in contiguous,
+    balanced ranges (the first n_groups % world ranks hold one group more)."""
+    base, rem = divmod(n_groups, world)
+    begin = rank * base + min(rank, rem)
+    return begin, begin + base + (1 if rank < rem else 0)
+
+
+def wide_mask_slice(ctx: Context, mask_bits: torch.Tensor, n_groups: int, group_begin: int, group_end: int,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    T = mask_bits.shape[0]
+    if out is None:
+        out = torch.empty((T, max(1, (group_end - group_begin + 31) // 32)), dtype=torch.int32, device=mask_bits.device)
+    rc = ctx.lib.wide_mask_slice(ctx.handle, _stream(), _ptr(mask_bits), T, n_groups, group_begin, group_end, _ptr(out))
+    _check(rc, "wide_mask_slice")
     return out
 
 

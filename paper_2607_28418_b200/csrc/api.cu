@@ -251,6 +251,16 @@ int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tok
                                token_rank);
 }
 
+int wide_mask_slice(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups, int group_begin,
+                    int group_end, uint32_t* out_bits) {
+    if (!ctx || !mask_bits || !out_bits) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || n_groups <= 0 || group_begin < 0 || group_end < group_begin || group_end > n_groups)
+        return WIDE_ERR_INVALID_ARG;
+    if (n_groups > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    return wide_launch_mask_slice(ctx, static_cast<cudaStream_t>(stream), mask_bits, tokens, n_groups, group_begin,
+                                  group_end, out_bits);
+}
+
 int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
              const void* w_down, int dtype, int tokens, int hidden, int d_ff, int group,
              const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,

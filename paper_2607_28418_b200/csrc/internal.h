@@ -107,6 +107,9 @@ int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits
                         int32_t* work_list, int32_t* n_work, int32_t* union_list, int32_t* n_union,
                         int32_t* offsets, int32_t* token_order, int32_t* token_rank);
 
+int wide_launch_mask_slice(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG, int g_begin, int g_end,
+                           uint32_t* out);
+
 int wide_launch_unpermute(wide_ctx* ctx, cudaStream_t s, const void* src, const int32_t* perm, const int32_t* counts,
                           const int32_t* offsets, int T, int NG, int G, int elem_bytes, void* dst);
 

@@ -268,7 +268,37 @@ __global__ void __launch_bounds__(256) unpermute_kernel(const uint4* __restrict_
     }
 }
 
+// out[t] = bits [g_begin, g_end) of row t, re-packed from bit 0 (unused high bits 0).
+__global__ void __launch_bounds__(256) mask_slice_kernel(const uint32_t* __restrict__ mask_bits, int T, int words_in,
+                                                         int g_begin, int g_end, int words_out, uint32_t* __restrict__ out) {
+    const long long total = static_cast<long long>(T) * words_out;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int t = static_cast<int>(i / words_out), w = static_cast<int>(i % words_out);
+        const int first = g_begin + 32 * w;                 // global index of this word's bit 0
+        const uint32_t* row = mask_bits + static_cast<size_t>(t) * words_in;
+        const int wi = first >> 5, sh = first & 31;
+        uint32_t lo = row[wi] >> sh;
+        if (sh != 0 && wi + 1 < words_in) lo |= row[wi + 1] << (32 - sh);
+        const int keep = g_end - first;                     // bits of this word inside the range
+        if (keep < 32) lo &= (1u << keep) - 1u;
+        out[i] = lo;
+    }
+}
+
 }  // namespace
+
+int wide_launch_mask_slice(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG, int g_begin, int g_end,
+                           uint32_t* out) {
+    const int words_out = (g_end - g_begin + 31) / 32;
+    const long long total = static_cast<long long>(T) * words_out;
+    if (total == 0) return WIDE_OK;
+    long long blocks = (total + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    WideLaunch l(ctx, s, "mask_slice");
+    mask_slice_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(mask_bits, T, (NG + 31) / 32, g_begin, g_end, words_out, out);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+}
 
 int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
                         int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
