@@ -13,6 +13,8 @@ route_scores          Routing components (Section 3.1): a linear map from the
                       (``route_scores`` + ``mask_topk``) is the fixed-budget reading
                       "each token selects R groups" of Appendix A.
 mask_pair_argmax      Eq. 4, inference branch: bit = [argmax over the class pair = 0].
+route_logits_pair_norm  Eq. 4 applied to the RMSNorm of the hidden state (the router's input in a
+                      pre-norm transformer block); rmsnorm is the textbook definition.
 reorder               Eq. 6 / Algorithm 1 (per-column SortDesc, stable), the predicate
                       of Eq. 7-8 at level 0 (CTA tile), Appendix B's monotone shortcut.
 cluster_tokens        not in the paper: one global token permutation (stable sort by a
@@ -67,6 +69,22 @@ def route_logits_pair(x: ArrayLike, w1: ArrayLike, w2: ArrayLike) -> np.ndarray:
     """Eq. 4: R = reshape(X W1 W2) in [T, N_G, 2]; W1 [D, r], W2 [r, 2 N_G]."""
     logits = (_f64(x) @ _f64(w1)) @ _f64(w2)
     return logits.reshape(logits.shape[0], -1, 2)
+
+
+def rmsnorm(x: ArrayLike, weight: Optional[ArrayLike], eps: float) -> np.ndarray:
+    """RMSNorm of the Llama backbones the paper prunes (Section 4.1): every row divided by the root
+    of its mean square (plus eps), then scaled channel-wise by `weight` (None: no scaling)."""
+    x = _f64(x)
+    y = x / np.sqrt(np.mean(x * x, axis=1, keepdims=True) + float(eps))
+    return y if weight is None else y * _f64(weight)[None, :]
+
+
+def route_logits_pair_norm(x: ArrayLike, norm_weight: Optional[ArrayLike], eps: float, w1: ArrayLike,
+                           w2: ArrayLike) -> np.ndarray:
+    """Eq. 4 on the normalised activation: the router reads the layer's input after its RMSNorm
+    (the router "maps the input activation", Section 3.1, and the pruned unit's input is the
+    normalised hidden state), so R = reshape(RMSNorm(x) W1 W2)."""
+    return route_logits_pair(rmsnorm(x, norm_weight, eps), w1, w2)
 
 
 def mask_pair_argmax(logits_pair: np.ndarray) -> np.ndarray:

@@ -4,6 +4,7 @@ None of these re-types the oracle's own formula: they use exact rational brute f
 closed-form routers, a hand-worked fixture, and the invariants the paper states for the
 sorted layout (Section 3.3 and Appendix B).
 """
+import math
 import os
 from fractions import Fraction
 
@@ -306,3 +307,47 @@ def test_packed_layout_matches_hand_worked_fixture():
     back = wo.unpermute(np.array(fx["packed"], dtype=np.float32), np.array(fx["perm"], dtype=np.int32),
                         np.array(fx["counts"][0]), np.array(fx["offsets"][0]), 5, 2)
     assert back.tolist() == fx["scattered"]
+
+
+# ----------------------------------------------------------------------------- pair router on the normalised input
+def test_rmsnorm_matches_plain_loops():
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((5, 12)) * 3.0
+    w = rng.standard_normal(12)
+    got = wo.rmsnorm(x, w, 1e-5)
+    for t in range(5):
+        ms = sum(float(v) ** 2 for v in x[t]) / 12
+        for i in range(12):
+            assert abs(got[t, i] - x[t, i] / math.sqrt(ms + 1e-5) * w[i]) <= 1e-14 * (1 + abs(got[t, i]))
+    # a row of unit mean square and no weight passes through (eps = 0)
+    u = np.ones((1, 7))
+    assert np.allclose(wo.rmsnorm(u, None, 0.0), u, rtol=0, atol=0)
+
+
+def test_pair_router_on_normalised_input_by_loops_and_scale_invariance():
+    rng = np.random.default_rng(22)
+    T, D, r, NG = 6, 10, 3, 4
+    x = rng.standard_normal((T, D))
+    g = rng.standard_normal(D)
+    w1 = rng.standard_normal((D, r))
+    w2 = rng.standard_normal((r, 2 * NG))
+    eps = 1e-6
+    logits = wo.route_logits_pair_norm(x, g, eps, w1, w2)
+    assert logits.shape == (T, NG, 2)
+    for t in range(T):
+        rms = math.sqrt(sum(float(v) ** 2 for v in x[t]) / D + eps)
+        xh = [float(x[t, i]) / rms * float(g[i]) for i in range(D)]
+        u = [sum(xh[i] * float(w1[i, c]) for i in range(D)) for c in range(r)]
+        for n in range(2 * NG):
+            ref = sum(u[c] * float(w2[c, n]) for c in range(r))
+            assert abs(logits[t, n // 2, n % 2] - ref) <= 1e-12 * (1 + abs(ref))
+    mask = wo.mask_pair_argmax(logits)
+    # the decision ignores a positive scale of the row: the normalisation's 1/rms drops out, and so
+    # does any rescaling of a token
+    unscaled = wo.mask_pair_argmax(wo.route_logits_pair(x * g[None, :], w1, w2))
+    assert (mask == unscaled).all()
+    assert (wo.mask_pair_argmax(wo.route_logits_pair_norm(x * np.array([[0.01], [3.0], [1.0], [250.0], [7.0], [0.5]]),
+                                                          g, 0.0, w1, w2)) == mask).all()
+    # an all-zero token has all-zero logits: every pair ties, class 0 wins, everything executes
+    z = wo.mask_pair_argmax(wo.route_logits_pair_norm(np.zeros((1, D)), g, eps, w1, w2))
+    assert z.all()
