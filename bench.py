@@ -755,6 +755,48 @@ def run_group_sharded(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------- router forms
+def run_route_forms(args):
+    """--op route: the three router forms on the workload's shape, each replayed as a graph:
+    single linear + top-k, Eq. 4 (bottleneck pair-argmax) with the weight work inside every call, and
+    Eq. 4 on the RMSNorm of the hidden state with the weight work prepared once."""
+    import torch
+
+    from paper_2607_28418_b200 import binding
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    cfg = make_config(args)
+    ctx = binding.Context(0)
+    case = synth.make_ffn_case(cfg, 0)
+    pr = synth.make_pair_router(cfg, 0, rank=16)
+    x, wr = binding.upload(case["x"], "bf16"), binding.upload(case["w_router"], "bf16")
+    w1, w2 = binding.upload(pr["w1"], "bf16"), binding.upload(pr["w2"], "bf16")
+    gamma = binding.upload(synth.round_to_bf16((1.0 + 0.1 * np.random.default_rng(1).standard_normal(cfg.hidden)).astype(np.float32)), "bf16")
+    NG = cfg.n_groups
+    bits = torch.empty((cfg.tokens, (NG + 31) // 32), dtype=torch.int32, device="cuda")
+    prepared = binding.wide_route_pair_prepare(ctx, w1, w2, gamma, NG)
+    forms = {
+        "topk": lambda: binding.wide_route(ctx, x, wr, NG, cfg.k, mask_bits=bits),
+        "pair_argmax": lambda: binding.wide_route(ctx, x, w1, NG, mode=binding.ROUTE_PAIR_ARGMAX, w2=w2, rank=16, mask_bits=bits),
+        "pair_argmax_rmsnorm_prepared": lambda: binding.wide_route_pair_norm(ctx, x, w1, w2, gamma, 1e-5, prepared, NG, mask_bits=bits),
+    }
+    out = {}
+    for name, fn in forms.items():
+        for _ in range(3):
+            fn()
+        g = graph_of(torch, fn)
+        g()
+        out[name + "_us"] = round(event_ms(torch, g, max(20, args.steps)) * 1e3, 2)
+        ctx.profile_begin(64)
+        fn()
+        out[name + "_kernels_us"] = {k: round(v["total_ms"] * 1e3, 1) for k, v in ctx.profile_end().items()}
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set")
+    print(json.dumps({"op": "route", "config": config_record(cfg, "route", 1), "rank": 16, **out}))
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------- attention op
 def run_attn(args):
     """--op attn: route (attention router) -> reorder -> head-group-masked causal attention on the
@@ -967,7 +1009,7 @@ def main():
     ap.add_argument("--router", default="", choices=["", "random", "clustered", "clustered_corr"])
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--group", type=int, default=0)
-    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn", "qproj"],
+    ap.add_argument("--op", default="ffn", choices=["ffn", "oproj", "attn", "qproj", "route"],
                     help="oproj, qproj and attn need a workload with an attention half")
     ap.add_argument("--shard", default="tokens", choices=["tokens", "groups"],
                     help="multi-GPU partition: token shards with replicated weights (no collective), or group "
@@ -989,6 +1031,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.op == "route":
+        run_route_forms(args)
     elif args.shard == "groups":
         run_group_sharded(args)
     elif args.op == "attn":

@@ -195,6 +195,41 @@ WIDE_API int wide_route_static(wide_ctx* ctx, void* stream, const void* x, int d
                                const int32_t* k_per_token, uint32_t* mask_bits, float* scores, unsigned flags);
 
 /*
+ * wide_route_pair_prepare / wide_route_pair_norm -- Eq. 4 (Section 3.1, routing components) with the
+ * router reading the layer's input through its RMSNorm, the weight-only work done once.
+ *
+ *   xh[t,:] = x[t,:] / sqrt(mean_i x[t,i]^2 + eps) * norm_weight      (norm_weight NULL: no scaling)
+ *   l = (xh W1) W2,  token t executes group g iff l[t,2g] >= l[t,2g+1]
+ *
+ * The caller passes the UN-normalised hidden state: 1 / rms is a positive factor of a whole row and
+ * cannot change which logit of a pair is larger, so the decision is taken on (x * norm_weight) W1 W2
+ * and the factor only scales the logits that are returned.  norm_weight is folded into W1 by
+ * wide_route_pair_prepare, which also forms, once per weight set,
+ *   - diag(norm_weight) W1, transposed, as a pair of bf16 matrices (value and rounding remainder:
+ *     the tensor-core product then misses the exact one by 2^-18 of its size at most), and
+ *   - d_g = diag(norm_weight) W1 (W2[:,2g] - W2[:,2g+1]) in fp64 for every group,
+ * so that a call is three launches: the bottleneck product on the tensor cores (fp32), the logits
+ * with an error bound per pair, and one exact fp64 dot product x . d_g for each pair the bound
+ * cannot decide (an exact tie falls back to the definition in fp64).  The selection equals the
+ * fp64 decision on the exact input products.
+ *   x [tokens, hidden] bf16; w1 [hidden, rank], w2 [rank, 2*n_groups], norm_weight [hidden] bf16
+ *   prepared: device buffer of wide_route_pair_prepared_bytes(hidden, rank, n_groups), written by
+ *       prepare, read by every later call with the same weights and shapes
+ *   scores out fp32 [tokens, 2*n_groups] or NULL: the logits of the normalised input
+ *   workspace: wide_route_pair_norm_workspace_bytes(tokens, rank)
+ * Needs hidden % 64 == 0, hidden <= 16384, rank % 8 == 0, rank <= 32, n_groups <= 192.
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, ALIGNMENT, WORKSPACE, CUDA.
+ */
+WIDE_API size_t wide_route_pair_prepared_bytes(int hidden, int rank, int n_groups);
+WIDE_API size_t wide_route_pair_norm_workspace_bytes(int tokens, int rank);
+WIDE_API int wide_route_pair_prepare(wide_ctx* ctx, void* stream, const void* w1, const void* w2, const void* norm_weight,
+                                     int hidden, int rank, int n_groups, void* prepared, size_t prepared_bytes);
+WIDE_API int wide_route_pair_norm(wide_ctx* ctx, void* stream, const void* x, int tokens, int hidden, const void* w1,
+                                  const void* w2, int rank, int n_groups, const void* norm_weight, float eps,
+                                  const void* prepared, uint32_t* mask_bits, float* scores, void* workspace,
+                                  size_t workspace_bytes);
+
+/*
  * wide_reorder -- mask reordering, Eq. 6 / Algorithm 1, and the level-0 predicate of Eq. 7-8.
  * For each group g the rows are sorted by mask value, descending and STABLE (active rows in
  * ascending token order, then inactive rows in ascending token order).

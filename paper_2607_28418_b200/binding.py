@@ -27,7 +27,9 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, 
 
 EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns", "wide_profile_begin",
            "wide_profile_end", "wide_launch_count", "wide_selftest_wait", "wide_strerror",
-           "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_reorder", "wide_mask_slice",
+           "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_route_pair_prepared_bytes",
+           "wide_route_pair_norm_workspace_bytes", "wide_route_pair_prepare", "wide_route_pair_norm", "wide_reorder",
+           "wide_mask_slice",
            "wide_ffn",
            "wide_oproj", "wide_attn", "wide_qproj", "wide_unpermute"]
 
@@ -69,6 +71,13 @@ def load_library() -> ctypes.CDLL:
                                _c_int, _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                                _c_size_t, _c_uint]
     lib.wide_route_static.argtypes = lib.wide_route.argtypes[:15] + [_c_uint]
+    lib.wide_route_pair_prepared_bytes.argtypes = [_c_int] * 3
+    lib.wide_route_pair_prepared_bytes.restype = _c_size_t
+    lib.wide_route_pair_norm_workspace_bytes.argtypes = [_c_int] * 2
+    lib.wide_route_pair_norm_workspace_bytes.restype = _c_size_t
+    lib.wide_route_pair_prepare.argtypes = [_c_void_p] * 5 + [_c_int] * 3 + [_c_void_p, _c_size_t]
+    lib.wide_route_pair_norm.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p, _c_void_p, _c_int, _c_int,
+                                         _c_void_p, ctypes.c_float, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_size_t]
     lib.wide_reorder.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int] + [_c_void_p] * 10
     lib.wide_mask_slice.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_void_p]
     lib.wide_ffn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int,
@@ -85,7 +94,8 @@ def load_library() -> ctypes.CDLL:
     lib.wide_unpermute.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                    _c_int, _c_int, _c_int, _c_void_p]
     for name in EXPORTS:
-        if name not in ("wide_strerror", "wide_workspace_bytes"):
+        if name not in ("wide_strerror", "wide_workspace_bytes", "wide_route_pair_prepared_bytes",
+                        "wide_route_pair_norm_workspace_bytes"):
             getattr(lib, name).restype = _c_int
     _lib = lib
     return lib
@@ -219,6 +229,35 @@ def wide_route(ctx: Context, x: torch.Tensor, w_router: torch.Tensor, n_groups: 
                             n_groups, mode, k, _ptr(k_per_token), _ptr(mask_bits), _ptr(scores), _ptr(ws),
                             ws.numel(), flags)
     _check(rc, "wide_route")
+    return mask_bits, scores
+
+
+def wide_route_pair_prepare(ctx: Context, w1: torch.Tensor, w2: torch.Tensor, norm_weight: Optional[torch.Tensor],
+                            n_groups: int) -> torch.Tensor:
+    """Once per weight set: the prepared buffer wide_route_pair_norm reads."""
+    D, rank = w1.shape
+    nbytes = int(ctx.lib.wide_route_pair_prepared_bytes(D, rank, n_groups))
+    prepared = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=w1.device)
+    rc = ctx.lib.wide_route_pair_prepare(ctx.handle, _stream(), _ptr(w1), _ptr(w2), _ptr(norm_weight), D, rank, n_groups,
+                                         _ptr(prepared), prepared.numel())
+    _check(rc, "wide_route_pair_prepare")
+    return prepared
+
+
+def wide_route_pair_norm(ctx: Context, x: torch.Tensor, w1: torch.Tensor, w2: torch.Tensor, norm_weight: Optional[torch.Tensor],
+                         eps: float, prepared: torch.Tensor, n_groups: int, want_scores: bool = False,
+                         mask_bits: Optional[torch.Tensor] = None):
+    """Eq. 4 on RMSNorm(x): returns (mask_bits, logits of the normalised input or None)."""
+    T, D = x.shape
+    rank = w1.shape[1]
+    if mask_bits is None:
+        mask_bits = torch.empty((T, (n_groups + 31) // 32), dtype=torch.int32, device=x.device)
+    scores = torch.empty((T, 2 * n_groups), dtype=torch.float32, device=x.device) if want_scores else None
+    ws = ctx.workspace(int(ctx.lib.wide_route_pair_norm_workspace_bytes(T, rank)), slot=1)
+    rc = ctx.lib.wide_route_pair_norm(ctx.handle, _stream(), _ptr(x), T, D, _ptr(w1), _ptr(w2), rank, n_groups,
+                                      _ptr(norm_weight), float(eps), _ptr(prepared), _ptr(mask_bits), _ptr(scores), _ptr(ws),
+                                      ws.numel())
+    _check(rc, "wide_route_pair_norm")
     return mask_bits, scores
 
 

@@ -236,6 +236,41 @@ int wide_route(wide_ctx* ctx, void* stream, const void* x, int dtype, int tokens
                              n_groups, mode, k, k_per_token, mask_bits, scores, workspace, flags);
 }
 
+size_t wide_route_pair_prepared_bytes(int hidden, int rank, int n_groups) {
+    if (hidden <= 0 || rank <= 0 || n_groups <= 0) return 0;
+    return wide_route_pair_prepared_size(hidden, rank, n_groups);
+}
+
+size_t wide_route_pair_norm_workspace_bytes(int tokens, int rank) {
+    if (tokens < 0 || rank <= 0) return 0;
+    return wide_route_pair_norm_workspace(tokens, rank);
+}
+
+int wide_route_pair_prepare(wide_ctx* ctx, void* stream, const void* w1, const void* w2, const void* norm_weight, int hidden,
+                            int rank, int n_groups, void* prepared, size_t prepared_bytes) {
+    if (!ctx || !w1 || !w2 || !prepared || hidden <= 0 || rank <= 0 || n_groups <= 0) return WIDE_ERR_INVALID_ARG;
+    if (!wide_route_pair_norm_supported(hidden, rank, n_groups) || !ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(w1) || !wide_aligned16(w2) || !wide_aligned16(prepared) || (norm_weight && !wide_aligned16(norm_weight)))
+        return WIDE_ERR_ALIGNMENT;
+    if (prepared_bytes < wide_route_pair_prepared_size(hidden, rank, n_groups)) return WIDE_ERR_WORKSPACE;
+    return wide_launch_route_pair_prepare(ctx, static_cast<cudaStream_t>(stream), w1, w2, norm_weight, hidden, rank, n_groups,
+                                          prepared);
+}
+
+int wide_route_pair_norm(wide_ctx* ctx, void* stream, const void* x, int tokens, int hidden, const void* w1, const void* w2,
+                         int rank, int n_groups, const void* norm_weight, float eps, const void* prepared,
+                         uint32_t* mask_bits, float* scores, void* workspace, size_t workspace_bytes) {
+    if (!ctx || !x || !w1 || !w2 || !prepared || !mask_bits) return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || rank <= 0 || n_groups <= 0 || !(eps >= 0.f)) return WIDE_ERR_INVALID_ARG;
+    if (!wide_route_pair_norm_supported(hidden, rank, n_groups) || !ctx->encode_tiled) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(x) || !wide_aligned16(w1) || !wide_aligned16(w2) || !wide_aligned16(prepared) ||
+        !wide_aligned16(workspace) || (norm_weight && !wide_aligned16(norm_weight)))
+        return WIDE_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < wide_route_pair_norm_workspace(tokens, rank)) return WIDE_ERR_WORKSPACE;
+    return wide_launch_route_pair_norm(ctx, static_cast<cudaStream_t>(stream), x, tokens, hidden, w1, w2, rank, n_groups,
+                                       norm_weight, eps, const_cast<void*>(prepared), mask_bits, scores, workspace);
+}
+
 int wide_reorder(wide_ctx* ctx, void* stream, const uint32_t* mask_bits, int tokens, int n_groups,
                  int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map, int32_t* work_list,
                  int32_t* n_work, int32_t* union_list, int32_t* n_union, int32_t* offsets, int32_t* token_order,

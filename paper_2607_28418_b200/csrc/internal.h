@@ -101,6 +101,15 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
                       const void* w_router, const void* w2, int rank, int NG, int mode, int k,
                       const int32_t* k_per_token, uint32_t* mask_bits, float* scores, void* ws, unsigned flags);
 size_t wide_route_workspace(int T, int NG, int rank);
+// Eq. 4 on the RMSNorm of the hidden state, weight-only work prepared once (csrc/route.cu)
+size_t wide_route_pair_prepared_size(int D, int rank, int NG);
+size_t wide_route_pair_norm_workspace(int T, int rank);
+bool wide_route_pair_norm_supported(int D, int rank, int NG);
+int wide_launch_route_pair_prepare(wide_ctx* ctx, cudaStream_t s, const void* w1, const void* w2, const void* gamma, int D,
+                                   int rank, int NG, void* prepared);
+int wide_launch_route_pair_norm(wide_ctx* ctx, cudaStream_t s, const void* x, int T, int D, const void* w1, const void* w2,
+                                int rank, int NG, const void* gamma, float eps, void* prepared, uint32_t* mask_bits,
+                                float* scores, void* ws);
 
 int wide_launch_reorder(wide_ctx* ctx, cudaStream_t s, const uint32_t* mask_bits, int T, int NG,
                         int tile_m, int32_t* perm, int32_t* counts, uint8_t* tile_map,
@@ -128,7 +137,7 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const int32_t* token_order, const int32_t* token_rank, void* y,
                                int out_dtype, void* h, void* acc, unsigned flags);
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
-                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out);
+                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out, int* chain_out);
 // `a_masked` is scratch [T, K] bf16, `acc` scratch [T, D] fp32.
 int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                  int D, int K, int G, const uint32_t* mask_bits, const int32_t* perm,

@@ -108,7 +108,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N, int K,
             int G, void* __restrict__ Y,
             int out_bf16, int ksplit, const __nv_bfloat16* __restrict__ aux_w, int aux_rows,
-            float* __restrict__ aux_norm, const int32_t* __restrict__ sel_counts, int sel_thr,
+            float* __restrict__ aux_norm, const int32_t* __restrict__ sel_counts, int sel_thr, int acc_split,
             int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
@@ -191,9 +191,10 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * kAccCols;
                 uint32_t accumulate = 0;
+                int steps_done = 0;
                 for (int g = 0; g < NG && ok; ++g) {
                     if (!((act[g >> 5] >> (g & 31)) & 1u) || (only >= 0 && g != only)) continue;
-                    for (int kk = 0; kk < ksub; ++kk, ++it) {
+                    for (int kk = 0; kk < ksub; ++kk, ++it, ++steps_done) {
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1;
                         if (!mbar_wait(L.full + 8 * s, ph, wait_ns, L.abort_flag)) { ok = false; break; }
@@ -201,6 +202,18 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         const uint32_t a_addr = smem_u32(L.stage_base + s * kStageBytes);
                         const uint64_t adesc = umma_desc_sw128(a_addr);
                         const uint64_t bdesc = umma_desc_sw128(a_addr + kABytes);
+                        if (acc_split > 1) {
+                            // score mode: the k-steps go round-robin to acc_split accumulators (one tile
+                            // per CTA, so they may take the whole tensor memory), which shortens every
+                            // fp32 accumulation chain by that factor; the epilogue adds them up
+                            const uint32_t d_acc = tmem_base + (steps_done % acc_split) * BN;
+#pragma unroll
+                            for (int k4 = 0; k4 < kBK / 16; ++k4)
+                                umma_bf16(d_acc, adesc + 2 * k4, bdesc + 2 * k4, idesc, (steps_done >= acc_split || k4 > 0) ? 1u : 0u);
+                            accumulate = 1;
+                            umma_commit(L.empty + 8 * s);
+                            continue;
+                        }
 #pragma unroll
                         for (int k4 = 0; k4 < kBK / 16; ++k4) {
                             umma_bf16(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, accumulate);
@@ -242,6 +255,13 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (any) {
                     tmem_ld_32x32(taddr + c0, r);
                     tmem_ld_wait();
+                    for (int a = 1; a < acc_split; ++a) {
+                        uint32_t r2[32];
+                        tmem_ld_32x32(taddr + a * BN + c0, r2);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+                    }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) r[i] = 0u;
@@ -966,7 +986,7 @@ template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                 int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down",
                 int ksplit = 1, float* aux_norm = nullptr, const int32_t* order = nullptr,
-                const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER) {
+                const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, int acc_split = 1) {
     CUtensorMap tmA, tmB;
     if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
@@ -979,7 +999,7 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     WideLaunch l(ctx, s, name);
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                             ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm, sel_counts, sel_thr,
-                                            ctx->d_status, ctx->wait_ns);
+                                            acc_split, ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -1163,7 +1183,7 @@ int wide_launch_oproj_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* a, c
 // 32, columns >= NG are zeros (weight rows past NG are zero-filled by the TMA).  The same launch
 // writes ||w_g|| (rounded up) to wnorm[0..NG).  Returns the ksplit it used through *ksplit_out.
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
-                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out) {
+                          int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out, int* chain_out) {
     const int n_m = (T + kBM - 1) / kBM;
     int ksplit = 1;
     // more CTAs while each keeps >= 8 k-steps, the slabs fit, and everything is co-resident
@@ -1171,10 +1191,16 @@ int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const vo
            n_m * ksplit * 2 + (NG + 5) / 6 <= ctx->sm_count)
         ksplit *= 2;
     *ksplit_out = ksplit;
+    // Every CTA has one tile here (the grid is the tile count plus the norm CTAs), so the k-steps of
+    // a slab can be spread over several accumulators: up to 4 of 128 columns or 2 of 256.
+    const int ksteps = D / ksplit / kBK;
+    int acc = ld <= 128 ? 4 : 2;
+    while (acc > 1 && ksteps < 2 * acc) acc >>= 1;
+    *chain_out = (D / ksplit + acc - 1) / acc + acc + ksplit;
     if (T == 0) return WIDE_OK;
     if (ld <= 128)
         return launch_down<128>(ctx, s, x, w_router, nullptr, T, ld, D, D / ksplit, scores, WIDE_F32, NG,
-                                "route_scores_tc", ksplit, wnorm);
+                                "route_scores_tc", ksplit, wnorm, nullptr, nullptr, WIDE_KAXIS_NEVER, acc);
     return launch_down<256>(ctx, s, x, w_router, nullptr, T, ld, D, D / ksplit, scores, WIDE_F32, NG,
-                            "route_scores_tc", ksplit, wnorm);
+                            "route_scores_tc", ksplit, wnorm, nullptr, nullptr, WIDE_KAXIS_NEVER, acc);
 }

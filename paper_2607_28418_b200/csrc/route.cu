@@ -107,10 +107,11 @@ __global__ void __launch_bounds__(256) pair_select_kernel(const double* __restri
 
 // ---------------------------------------------------------------------------- fast path (bf16)
 // Scores come from the tensor cores in fp32 (exact products, fp32 accumulation), as `nsplit`
-// partial slabs over K that are summed here in fp32.  Their error is bounded by
-//   eps_t = kAccumErr * (D / nsplit + nsplit) * ||x_t|| * max_g ||w_g||
-// (a per-element accumulation error along each slab's chain plus the slab sum, times the
-// Cauchy-Schwarz bound on the sum of absolute products).  A group whose fp32 score is further
+// partial slabs over K that are summed here in fp32; inside a slab the score GEMM spreads its
+// k-steps over `a` accumulators that it adds up at the end.  Their error is bounded by
+//   eps_t = kAccumErr * chain * ||x_t|| * max_g ||w_g||,   chain = D / (nsplit * a) + a + nsplit
+// (a per-element accumulation error along each accumulator's chain plus the two short sums, times
+// the Cauchy-Schwarz bound on the sum of absolute products).  A group whose fp32 score is further
 // than 2*eps_t from the selection boundary keeps its fp32 decision; the few groups inside that
 // band get their score recomputed exactly in fp64, and the band is re-ranked on those exact
 // values.  The result equals the fp64 decision of the slow path provided the accumulator loses at
@@ -171,7 +172,7 @@ __global__ void __launch_bounds__(64 * kSelTokens, 8)   // every CTA of a 2048-t
 select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
                    const __nv_bfloat16* __restrict__ w, const float* __restrict__ wnorm, int T, int NG, int D, int k,
                    const int32_t* __restrict__ k_per_token, uint32_t* __restrict__ mask_bits,
-                   float* __restrict__ scores_out) {
+                   float* __restrict__ scores_out, int chain) {
     __shared__ float s_xsq[kSelTokens];
     __shared__ int s_nb[kSelTokens];
     __shared__ int s_band[kSelTokens][kBandMax];
@@ -288,7 +289,7 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
     // band half-width 2 * eps_t (a little slack for the fp32 evaluation of the bound itself)
     int nb = 0, m_hi = 0;
     if (select_warp && boundary) {
-        const float steps = static_cast<float>((D + nsplit - 1) / nsplit + nsplit);
+        const float steps = static_cast<float>(chain);
         const float tau = 2.f * kAccumErr * steps * sqrtf(s_xsq[tt]) * 1.0001f * wmax;
 #pragma unroll
         for (int j = 0; j < KPL; ++j) {
@@ -374,9 +375,9 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
 template <int KPL>
 void launch_select_band(cudaStream_t s, int T, const float* sc32, int ksplit, int ld, const __nv_bfloat16* x,
                         const __nv_bfloat16* w, const float* wn, int NG, int D, int k, const int32_t* k_per_token,
-                        uint32_t* mask_bits, float* scores) {
+                        uint32_t* mask_bits, float* scores, int chain) {
     select_band_kernel<KPL><<<(T + kSelTokens - 1) / kSelTokens, 64 * kSelTokens, 0, s>>>(
-        sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores);
+        sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores, chain);
 }
 
 // ---------------------------------------------------------------------------- fast pair-argmax path (bf16)
@@ -408,7 +409,7 @@ transpose_w1_kernel(const __nv_bfloat16* __restrict__ w1, int D, int rank, int N
 // Block = 128 rows i x 32 groups.
 __global__ void __launch_bounds__(128)
 pair_delta_kernel(const __nv_bfloat16* __restrict__ w1, const __nv_bfloat16* __restrict__ w2, int D, int rank, int NG,
-                  double* __restrict__ d64, float* __restrict__ dn2) {
+                  double* __restrict__ d64, float* __restrict__ dn2, const __nv_bfloat16* __restrict__ gamma = nullptr) {
     __shared__ double delta[kPairMaxRank][32];
     __shared__ float sq[32];
     const int tid = threadIdx.x, g0 = blockIdx.y * 32, i = blockIdx.x * 128 + tid;
@@ -421,9 +422,10 @@ pair_delta_kernel(const __nv_bfloat16* __restrict__ w1, const __nv_bfloat16* __r
     if (tid < 32) sq[tid] = 0.f;
     __syncthreads();
     double w[kPairMaxRank];
+    const double gi = (gamma && i < D) ? static_cast<double>(__bfloat162float(gamma[i])) : 1.0;   // row i of diag(gamma) W1
 #pragma unroll
     for (int c = 0; c < kPairMaxRank; ++c)
-        w[c] = (c < rank && i < D) ? static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])) : 0.0;
+        w[c] = (c < rank && i < D) ? gi * static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])) : 0.0;
     for (int gg = 0; gg < 32 && g0 + gg < NG; ++gg) {
         double a = 0.0;
 #pragma unroll
@@ -444,15 +446,20 @@ pair_delta_kernel(const __nv_bfloat16* __restrict__ w1, const __nv_bfloat16* __r
 __global__ void __launch_bounds__(128)
 pair_band_kernel(const float* __restrict__ u_slabs, int nsplit, int ld, const __nv_bfloat16* __restrict__ x,
                  const __nv_bfloat16* __restrict__ w2, const float* __restrict__ wnorm, int T, int NG, int D, int rank,
-                 uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out, uint32_t* __restrict__ close_bits) {
+                 uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out, uint32_t* __restrict__ close_bits,
+                 int chain, int split = 0, float norm_eps = -1.f) {
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
     if (t >= T) return;
     const int words = (NG + 31) >> 5;
     const size_t slab = static_cast<size_t>(T) * ld;
+    // split: the bottleneck weights were given as a bf16 pair (hi in columns [0, rank), lo behind them)
     float u = 0.f;
     if (lane < rank)
-        for (int ks = 0; ks < nsplit; ++ks) u += __ldg(u_slabs + ks * slab + static_cast<size_t>(t) * ld + lane);
+        for (int ks = 0; ks < nsplit; ++ks) {
+            u += __ldg(u_slabs + ks * slab + static_cast<size_t>(t) * ld + lane);
+            if (split) u += __ldg(u_slabs + ks * slab + static_cast<size_t>(t) * ld + rank + lane);
+        }
     // ||x_t||
     float xsq = 0.f;
     const uint4* xv = reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * D);
@@ -468,9 +475,14 @@ pair_band_kernel(const float* __restrict__ u_slabs, int nsplit, int ld, const __
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
     // error bound of u_c (see the top-k form), then of the fp32 product below
-    const float steps = static_cast<float>((D + nsplit - 1) / nsplit + nsplit);
-    const float eu = lane < rank ? kAccumErr * steps * sqrtf(xsq) * 1.0001f * __ldg(wnorm + lane) : 0.f;
+    const float steps = static_cast<float>(chain);
+    float eu = lane < rank ? kAccumErr * steps * sqrtf(xsq) * 1.0001f * __ldg(wnorm + lane) : 0.f;
+    if (split && lane < rank)   // the lo product's accumulation error, the hi + lo sum, and what the pair leaves out (2^-18 |w|)
+        eu += sqrtf(xsq) * 1.0001f * (kAccumErr * steps * __ldg(wnorm + rank + lane) + 7.6293945e-6f * __ldg(wnorm + lane)) +
+              kAccumErr * fabsf(u);
     const float au = fabsf(u);
+    // the logits of the normalised input differ from these by the positive factor 1 / rms(x_t)
+    const float out_scale = norm_eps >= 0.f ? rsqrtf(xsq / static_cast<float>(D) + norm_eps) : 1.f;
     if (lane == 0) close_bits[static_cast<size_t>(t) * 32 + 31] = __float_as_uint(sqrtf(xsq) * 1.0001f);
     for (int j = 0; j < words; ++j) {
         const int g = 32 * j + lane;
@@ -498,8 +510,8 @@ pair_band_kernel(const float* __restrict__ u_slabs, int nsplit, int ld, const __
             close_bits[static_cast<size_t>(t) * 32 + j] = cword;
         }
         if (scores_out && g < NG) {
-            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = l0;
-            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = l1;
+            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = l0 * out_scale;
+            scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = l1 * out_scale;
         }
     }
 }
@@ -509,7 +521,8 @@ __global__ void __launch_bounds__(128)
 pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w1,
                   const __nv_bfloat16* __restrict__ w2, const double* __restrict__ d64, const float* __restrict__ dn2,
                   int T, int D, int rank, int NG, const uint32_t* __restrict__ close_bits,
-                  uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out) {
+                  uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out,
+                  const __nv_bfloat16* __restrict__ gamma = nullptr, float norm_eps = -1.f) {
     __shared__ double s_part[4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int words = (NG + 31) >> 5;
@@ -518,6 +531,7 @@ pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __re
         if (!__any_sync(0xffffffffu, lane < words && cw != 0u)) continue;      // the same in all four warps
         const __nv_bfloat16* xr = x + static_cast<size_t>(t) * D;
         const float xnorm = __uint_as_float(__shfl_sync(0xffffffffu, cw, 31));
+        const float out_scale = norm_eps >= 0.f ? rsqrtf(xnorm * xnorm / static_cast<float>(D) + norm_eps) : 1.f;
         bool long_way = false;
         for (int j = 0; j < words; ++j) {
             uint32_t bits = __shfl_sync(0xffffffffu, cw, j);
@@ -555,8 +569,8 @@ pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __re
                     // keep the pair's mean, set its difference to the exact one
                     float* sp = scores_out + static_cast<size_t>(t) * 2 * NG + 2 * g;
                     const float mid = 0.5f * (sp[0] + sp[1]);
-                    sp[0] = mid + 0.5f * static_cast<float>(m);
-                    sp[1] = mid - 0.5f * static_cast<float>(m);
+                    sp[0] = mid + 0.5f * static_cast<float>(m) * out_scale;
+                    sp[1] = mid - 0.5f * static_cast<float>(m) * out_scale;
                 }
             }
             if (threadIdx.x == 0) mask_bits[static_cast<size_t>(t) * words + j] = word;
@@ -566,9 +580,11 @@ pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __re
             double uu = 0.0;   // lane c ends up with u_c
             for (int c = 0; c < rank; ++c) {
                 double a = 0.0;
-                for (int i = lane; i < D; i += 32)
-                    a = fma(static_cast<double>(__bfloat162float(xr[i])),
-                            static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])), a);
+                for (int i = lane; i < D; i += 32) {
+                    double xi = static_cast<double>(__bfloat162float(xr[i]));
+                    if (gamma) xi *= static_cast<double>(__bfloat162float(gamma[i]));   // exact: 16 significant bits
+                    a = fma(xi, static_cast<double>(__bfloat162float(w1[static_cast<size_t>(i) * rank + c])), a);
+                }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
                 if (lane == c) uu = a;
@@ -586,11 +602,29 @@ pair_exact_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __re
                 const unsigned word = __ballot_sync(0xffffffffu, g < NG && l0 >= l1);
                 if (lane == 0) mask_bits[static_cast<size_t>(t) * words + j] = word;
                 if (scores_out && g < NG) {
-                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = static_cast<float>(l0);
-                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = static_cast<float>(l1);
+                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g] = static_cast<float>(l0) * out_scale;
+                    scores_out[static_cast<size_t>(t) * 2 * NG + 2 * g + 1] = static_cast<float>(l1) * out_scale;
                 }
             }
         }
+    }
+}
+
+// Prepared form of the bottleneck weights for wide_route_pair_norm: row c of w1t is column c of
+// diag(gamma) W1 rounded to bf16 (hi), row rank + c what that rounding left over, again in bf16 (lo).
+// gamma[i] * W1[i][c] has 16 significant bits, so it is exact in fp32 and hi + lo misses it by at
+// most 2^-18 of its size.
+__global__ void __launch_bounds__(256)
+pair_prepare_w1_kernel(const __nv_bfloat16* __restrict__ w1, const __nv_bfloat16* __restrict__ gamma, int D, int rank, int NG,
+                       __nv_bfloat16* __restrict__ w1t, float* __restrict__ dn2) {
+    for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < NG; g += gridDim.x * blockDim.x) dn2[g] = 0.f;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < static_cast<long long>(D) * rank;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int c = static_cast<int>(i / D), d = static_cast<int>(i % D);
+        const float p = __bfloat162float(w1[static_cast<size_t>(d) * rank + c]) * (gamma ? __bfloat162float(gamma[d]) : 1.f);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(p);
+        w1t[i] = hi;
+        w1t[static_cast<size_t>(rank) * D + i] = __float2bfloat16_rn(p - __bfloat162float(hi));
     }
 }
 
@@ -603,6 +637,82 @@ void launch_gemm_f64(wide_ctx* ctx, cudaStream_t s, const TA* A, const TB* B, do
 }
 
 }  // namespace
+
+// ---- Eq. 4 on the RMSNorm of the hidden state, with the weight-only work done once (prepare)
+namespace {
+struct PairPrepared {
+    __nv_bfloat16* w1t;   // [2 rank, D]
+    double* d64;          // [NG, D]
+    float* dn2;           // [NG]
+};
+PairPrepared carve_prepared(void* base, int D, int rank, int NG) {
+    char* b = static_cast<char*>(base);
+    PairPrepared p;
+    p.w1t = reinterpret_cast<__nv_bfloat16*>(b);
+    b += wide_align_up(static_cast<size_t>(2) * rank * D * 2, 256);
+    p.d64 = reinterpret_cast<double*>(b);
+    b += wide_align_up(static_cast<size_t>(NG) * D * sizeof(double), 256);
+    p.dn2 = reinterpret_cast<float*>(b);
+    return p;
+}
+}  // namespace
+
+size_t wide_route_pair_prepared_size(int D, int rank, int NG) {
+    return wide_align_up(static_cast<size_t>(2) * rank * D * 2, 256) + wide_align_up(static_cast<size_t>(NG) * D * sizeof(double), 256) +
+           wide_align_up(static_cast<size_t>(NG) * sizeof(float), 256);
+}
+
+bool wide_route_pair_norm_supported(int D, int rank, int NG) {
+    return D % 64 == 0 && D <= 16384 && rank <= kPairMaxRank && rank % 8 == 0 && NG <= 192;
+}
+
+int wide_launch_route_pair_prepare(wide_ctx* ctx, cudaStream_t s, const void* w1, const void* w2, const void* gamma, int D,
+                                   int rank, int NG, void* prepared) {
+    const PairPrepared p = carve_prepared(prepared, D, rank, NG);
+    const __nv_bfloat16* w1b = static_cast<const __nv_bfloat16*>(w1);
+    const __nv_bfloat16* gb = static_cast<const __nv_bfloat16*>(gamma);
+    {
+        WideLaunch l(ctx, s, "route_pair_prepare_w1");
+        pair_prepare_w1_kernel<<<64, 256, 0, s>>>(w1b, gb, D, rank, NG, p.w1t, p.dn2);
+    }
+    WideLaunch l(ctx, s, "route_pair_delta");
+    pair_delta_kernel<<<dim3((D + 127) / 128, (NG + 31) / 32), 128, 0, s>>>(w1b, static_cast<const __nv_bfloat16*>(w2), D, rank,
+                                                                             NG, p.d64, p.dn2, gb);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+}
+
+size_t wide_route_pair_norm_workspace(int T, int rank) {
+    const int ld = (2 * rank + 31) / 32 * 32;
+    return wide_align_up(static_cast<size_t>(T) * ld * sizeof(float) * kMaxSlabs, 256) + wide_align_up(static_cast<size_t>(T) * 128, 256) + 1024;
+}
+
+int wide_launch_route_pair_norm(wide_ctx* ctx, cudaStream_t s, const void* x, int T, int D, const void* w1, const void* w2,
+                                int rank, int NG, const void* gamma, float eps, void* prepared, uint32_t* mask_bits,
+                                float* scores, void* ws) {
+    if (T == 0) return WIDE_OK;
+    const PairPrepared p = carve_prepared(prepared, D, rank, NG);
+    const int ld = (2 * rank + 31) / 32 * 32;
+    char* wsb = static_cast<char*>(ws);
+    float* slabs = reinterpret_cast<float*>(wsb);
+    const size_t off1 = wide_align_up(static_cast<size_t>(T) * ld * sizeof(float) * kMaxSlabs, 256);
+    uint32_t* close_bits = reinterpret_cast<uint32_t*>(wsb + off1);
+    float* wn = reinterpret_cast<float*>(wsb + off1 + wide_align_up(static_cast<size_t>(T) * 128, 256));
+    const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+    const __nv_bfloat16* w2b = static_cast<const __nv_bfloat16*>(w2);
+    int ksplit = 1, chain = D;
+    const int rc = wide_launch_scores_tc(ctx, s, x, p.w1t, T, 2 * rank, ld, D, slabs, wn, kMaxSlabs, &ksplit, &chain);
+    if (rc != WIDE_OK) return rc;
+    {
+        WideLaunch l(ctx, s, "route_pair_band");
+        pair_band_kernel<<<(T + 3) / 4, 128, 0, s>>>(slabs, ksplit, ld, xb, w2b, wn, T, NG, D, rank, mask_bits, scores, close_bits,
+                                                      chain, 1, eps);
+    }
+    WideLaunch l(ctx, s, "route_pair_exact");
+    const int grid = T < 16 * ctx->sm_count ? T : 16 * ctx->sm_count;
+    pair_exact_kernel<<<grid, 128, 0, s>>>(xb, static_cast<const __nv_bfloat16*>(w1), w2b, p.d64, p.dn2, T, D, rank, NG,
+                                           close_bits, mask_bits, scores, static_cast<const __nv_bfloat16*>(gamma), eps);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
+}
 
 size_t wide_route_workspace(int T, int NG, int rank) {
     // fp64 scores [T, NG] (TOPK) or logits [T, 2NG] plus bottleneck activations [T, rank] (PAIR);
@@ -627,15 +737,15 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
         int max_split = static_cast<int>(part0 / (static_cast<size_t>(T) * ld * sizeof(float)));
         if (max_split > kMaxSlabs) max_split = kMaxSlabs;
         if (max_split < 1) max_split = 1;
-        int ksplit = 1;
-        const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32, wn, max_split, &ksplit);
+        int ksplit = 1, chain = D;
+        const int rc = wide_launch_scores_tc(ctx, s, x, w_router, T, NG, ld, D, sc32, wn, max_split, &ksplit, &chain);
         if (rc != WIDE_OK) return rc;
         WideLaunch l(ctx, s, "route_select_band");
         const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
         const __nv_bfloat16* wb = static_cast<const __nv_bfloat16*>(w_router);
         switch ((NG + 31) / 32) {   // mask words per token = groups held per lane
 #define WIDE_SEL_CASE(n) \
-    case n: launch_select_band<n>(s, T, sc32, ksplit, ld, xb, wb, wn, NG, D, k, k_per_token, mask_bits, scores); break;
+    case n: launch_select_band<n>(s, T, sc32, ksplit, ld, xb, wb, wn, NG, D, k, k_per_token, mask_bits, scores, chain); break;
             WIDE_SEL_CASE(1) WIDE_SEL_CASE(2) WIDE_SEL_CASE(3) WIDE_SEL_CASE(4)
             WIDE_SEL_CASE(5) WIDE_SEL_CASE(6) WIDE_SEL_CASE(7) WIDE_SEL_CASE(8)
 #undef WIDE_SEL_CASE
@@ -675,13 +785,13 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
             WideLaunch l(ctx, s, "route_pair_delta");
             pair_delta_kernel<<<dim3((D + 127) / 128, (NG + 31) / 32), 128, 0, s>>>(w1b, w2b, D, rank, NG, d64, dn2);
         }
-        int ksplit = 1;
-        const int rc = wide_launch_scores_tc(ctx, s, x, w1t, T, rank, ld, D, slabs, wn, max_split, &ksplit);
+        int ksplit = 1, chain = D;
+        const int rc = wide_launch_scores_tc(ctx, s, x, w1t, T, rank, ld, D, slabs, wn, max_split, &ksplit, &chain);
         if (rc != WIDE_OK) return rc;
         {
             WideLaunch l(ctx, s, "route_pair_band");
             pair_band_kernel<<<(T + 3) / 4, 128, 0, s>>>(slabs, ksplit, ld, xb, w2b, wn, T, NG, D, rank, mask_bits, scores,
-                                                          close_bits);
+                                                          close_bits, chain);
         }
         WideLaunch l(ctx, s, "route_pair_exact");
         const int grid = T < 16 * ctx->sm_count ? T : 16 * ctx->sm_count;
