@@ -355,7 +355,7 @@ attn_decode_ring_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         for (int t = warp; t < ntiles; t += kRingConsumers) {
             const int st = t % kRingStages;
             const uint32_t ph = (t / kRingStages) & 1;
-            if (!mbar_wait(full + 8 * st, ph, wait_ns, &s_abort)) break;
+            if (!mbar_wait_warp(full + 8 * st, ph, wait_ns, &s_abort)) break;
             const uint8_t* kt = ring + st * 2 * kTileBytes;
             const uint8_t* vt = kt + kTileBytes;
             {
@@ -626,7 +626,7 @@ attn_decode_ring_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __gri
         for (int t = warp; t < ntiles; t += kRingConsumers) {
             const int st = t % kRingStages;
             const uint32_t ph = (t / kRingStages) & 1;
-            if (!mbar_wait(full + 8 * st, ph, wait_ns, &s_abort)) break;
+            if (!mbar_wait_warp(full + 8 * st, ph, wait_ns, &s_abort)) break;
             const uint32_t kt = smem_u32(ring + st * 2 * kTileBytes), vt = kt + kTileBytes;
             const int c0 = j0 + t * kRingKeys;
             // S = Q K^T: four 8-key tiles, kKS k-steps.  One x4 load = (k-step ks, columns +0 / +8) and (ks + 1, +0 / +8)

@@ -274,7 +274,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
         int last = -1;
         for (int t = grp; t < NT; t += 2) {
             const uint32_t ph = (t >> 1) & 1;
-            if (!mbar_wait(s_full + 8 * b, ph, wait_ns, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(s_full + 8 * b, ph, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const int j0 = t * kKV;
             const bool edge = j0 + kKV - 1 > lim;     // this row needs element-wise predicates here
@@ -301,7 +301,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2e;
             // the previous PV of this group has to be complete before P is overwritten or O rescaled
-            if (last >= 0 && !mbar_wait(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
+            if (last >= 0 && !mbar_wait_warp(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
             float alpha = 1.f;
             const bool raise = mx > mref + kRaise || (mref == -CUDART_INF_F && mx > mref);
             if (raise) {
@@ -356,7 +356,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             mbar_arrive(p_ready + 8 * b);
             last = t;
         }
-        if (ok && last >= 0) ok = mbar_wait(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag);
+        if (ok && last >= 0) ok = mbar_wait_warp(pv_full + 8 * b, (last >> 1) & 1, wait_ns, abort_flag);
         tc_fence_after_sync();
         if (NT > 0) cp_async_wait_all();
         const float mrow = mref;

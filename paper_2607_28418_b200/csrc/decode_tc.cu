@@ -127,6 +127,21 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// The same barrier of the four epilogue warps, carrying an AND over a flag of every thread: a wait
+// that one warp gave up must take all four out of the pass together, or the others would stand at
+// the next barrier for good.
+__device__ __forceinline__ bool epilogue_bar_and(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(flag ? 1u : 0u)
+        : "memory");
+    return out != 0;
+}
 
 // All CTAs of the (co-resident) grid meet here; used once per launch.  bar[0] counts arrivals
 // (a fire-and-forget red after a fence; thread 0 then polls with acquire loads), bar[1] departures:
@@ -329,29 +344,31 @@ __device__ bool epilogue_pass(int mode, const DecodeArgs& a, Pipe& P, const int*
         float* out = (mode == MODE_GATEUP ? (mat ? a.up : a.gate) : a.yacc) + static_cast<size_t>(row) * a.NT;
         const int buf = P.tc & 1;
         const uint32_t tph = (P.tc >> 1) & 1;
-        if (!mbar_wait(P.tfull + 8 * buf, tph, a.wait_ns, P.abort_flag)) return false;
-        tc_fence_after_sync();
-        const uint32_t taddr = P.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccColsD;
-        for (int c0 = 0; c0 < a.NT; c0 += 16) {
-            uint32_t r[16];
-            tmem_ld_32x16(taddr + c0, r);
-            tmem_ld_wait();
-            if (live) {
+        const bool got = mbar_wait_warp(P.tfull + 8 * buf, tph, a.wait_ns, P.abort_flag);
+        if (got) {
+            tc_fence_after_sync();
+            const uint32_t taddr = P.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccColsD;
+            for (int c0 = 0; c0 < a.NT; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x16(taddr + c0, r);
+                tmem_ld_wait();
+                if (live) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v)
-                    if (c0 / 4 + v < nb4)
-                        red_add_v4(out + c0 + 4 * v, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    for (int v = 0; v < 4; ++v)
+                        if (c0 / 4 + v < nb4)
+                            red_add_v4(out + c0 + 4 * v, __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                       __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                }
             }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(P.tempty + 8 * buf);
+            ++P.tc;
         }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(P.tempty + 8 * buf);
-        ++P.tc;
 
         // ticket: has every piece of this block been added?
         __threadfence();
-        epilogue_bar_sync();
+        if (!epilogue_bar_and(got)) return false;
         if (e == 0) {
             unsigned* tk;
             int expected;

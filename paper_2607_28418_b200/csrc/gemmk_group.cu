@@ -222,7 +222,7 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
             for (int kk = 0; kk < ksub; ++kk, ++it) {
                 const int s = it % kStagesK;
                 const uint32_t ph = (it / kStagesK) & 1;
-                if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
                 const uint32_t a_dst = smem_u32(base + s * kStageBytes);
                 const size_t koff = static_cast<size_t>(kk) * (kBK * 2);
 #pragma unroll
@@ -259,7 +259,7 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
             const int j = m * kBM + q * 32 + lane;
             const int tok = j < counts[g] ? perm[static_cast<size_t>(g) * T + j] : -1;
             const int buf = tc & 1;
-            if (!mbar_wait(tfull + 8 * buf, (tc >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(tfull + 8 * buf, (tc >> 1) & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
 #pragma unroll 1

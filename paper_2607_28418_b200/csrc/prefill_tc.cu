@@ -244,7 +244,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int g = 0; g < NG; ++g) any = any || ((act[g >> 5] >> (g & 31)) & 1u);
             const int buf = tc & 1;
             const uint32_t tph = (tc >> 1) & 1;
-            if (!mbar_wait(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(L.tfull + 8 * buf, tph, wait_ns, L.abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const int pos = m * kBM + q * 32 + lane;              // row position of the tile
             const int row = (order && pos < T) ? order[pos] : pos;  // token that owns this output row
@@ -522,7 +522,7 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tile_mask(m, act);
             bool any = false;
             for (int g = 0; g < NG; ++g) any = any || ((act[g >> 5] >> (g & 31)) & 1u);
-            if (!mbar_wait(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
@@ -822,7 +822,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             for (int k = 0; k < nk; ++k, ++it) {
                 const int s = it % kStagesG;
                 const uint32_t ph = (it / kStagesG) & 1;
-                if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
                 const uint32_t a_dst = smem_u32(base + s * kStageBytes);
                 const size_t koff = static_cast<size_t>(k) * (kBK * 2);
 #pragma unroll
@@ -898,7 +898,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                 if (tok >= 0 && token_rank) tok = token_rank[tok];   // H rows are kept in clustered token order
                 tokh[half] = tok;
             }
-            if (!mbar_wait(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             for (int half = 0; half < w.rows / kBM; ++half) {
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 256 + chalf * kCh;

@@ -71,6 +71,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
     }
 }
 
+// The same wait for a warp whose 32 lanes all wait on the same barrier, with ONE outcome for the
+// warp.  Lanes poll on their own, so when a wait is given up (the limit runs out, or another warp has
+// flagged an abort) some lanes can see the barrier complete while others give up; a warp split that
+// way would go on to warp-wide instructions (tcgen05.ld/st .sync.aligned, votes, shuffles, named
+// barriers) with part of its lanes missing, and those wait without any limit.  Every lane of the
+// warp must call this, in converged code.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned long long limit_ns,
+                                               volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns, abort_flag) ? 1 : 0) != 0;
+}
+
 // ------------------------------------------------------------------------------- proxies / fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
