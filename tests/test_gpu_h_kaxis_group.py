@@ -144,3 +144,26 @@ def test_flag_combinations_are_validated_on_the_host(ctx):
     with pytest.raises(binding.WideError) as e:      # the per-group kernel needs the permutation
         binding.wide_oproj(ctx, a, w, G, bits, None, flags=binding.FLAG_FORCE_PREFILL | binding.FLAG_KAXIS_GROUP)
     assert e.value.code == binding.ERR_INVALID_ARG
+
+
+def test_per_group_kernel_narrow_output_and_empty_batch(ctx):
+    """An output narrower than one 256-column block, and a call with no tokens at all."""
+    from paper_2607_28418_b200 import binding
+    T, D, K, G, k = 200, 128, 1024, 256, 2
+    mask = synth.random_mask(4, T, K // G, k)
+    y, ref = _oproj(ctx, T, D, K, G, mask, binding.FLAG_FORCE_PREFILL | binding.FLAG_KAXIS_GROUP, seed=2)
+    assert_close(y, ref, "hidden 128")
+    # an empty batch, through the C ABI itself (torch hands out null pointers for empty tensors, and
+    # the entry points refuse null pointers): nothing is launched, the output is left alone
+    import ctypes
+    a = torch.zeros((1, K), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((D, K), dtype=torch.bfloat16, device="cuda")
+    small = torch.zeros((8,), dtype=torch.int32, device="cuda")
+    y0 = torch.full((1, D), 3.0, dtype=torch.bfloat16, device="cuda")
+    ws = ctx.workspace(1 << 20)
+    vp = lambda t: ctypes.c_void_p(t.data_ptr())
+    rc = ctx.lib.wide_oproj(ctx.handle, ctypes.c_void_p(torch.cuda.current_stream().cuda_stream), vp(a), vp(w), binding.BF16,
+                            0, D, K, G, vp(small), vp(small), vp(small), None, None, vp(y0), binding.BF16, vp(ws), ws.numel(),
+                            binding.FLAG_FORCE_PREFILL | binding.FLAG_KAXIS_GROUP)
+    torch.cuda.synchronize()
+    assert rc == 0 and (y0 == 3.0).all().item() and ctx.status() == 0
