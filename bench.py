@@ -701,12 +701,35 @@ def run_group_sharded(args):
     rows = torch.empty((T // world, cfg.hidden), dtype=torch.float32, device=dev)
     y = torch.empty((T // world, cfg.hidden), dtype=torch.bfloat16, device=dev)
     state = {"meta": None}
+    shard_ptrs = None
+    if args.fused:
+        # the fp32 shard of every rank, peer-mapped: the down projection adds into them directly
+        if world > 1:
+            import torch.distributed._symmetric_memory as symm_mem
+            rows = symm_mem.empty((T // world, cfg.hidden), dtype=torch.float32, device=dev)
+            handle = symm_mem.rendezvous(rows, dist.group.WORLD)
+            shard_ptrs = [int(p) for p in handle.buffer_ptrs]
+        else:
+            shard_ptrs = [rows.data_ptr()]
+        token = torch.zeros((1,), dtype=torch.float32, device=dev)
+
+    def rank_barrier():
+        # stream-ordered: a one-element all-reduce on the stream the kernels run on
+        if world > 1:
+            dist.all_reduce(token)
 
     def step():
         binding.wide_route(ctx, x, w_router, NG, cfg.k, mask_bits=bits)
         binding.wide_mask_slice(ctx, bits, NG, g0, g1, out=local_bits)
         if T > binding.DECODE_MAX_TOKENS:
             state["meta"] = binding.wide_reorder(ctx, local_bits, g1 - g0, 128, out=state["meta"])
+        if args.fused and T > binding.DECODE_MAX_TOKENS:
+            rows.zero_()
+            rank_barrier()                       # every shard is zero before any rank adds to it
+            binding.wide_ffn_tp(ctx, x, wg, wu, wd, G, local_bits, state["meta"], shard_ptrs, T // world)
+            rank_barrier()                       # every rank's adds have landed
+            y.copy_(rows)
+            return
         binding.wide_ffn(ctx, x, wg, wu, wd, G, local_bits, state["meta"], y=part)
         if world > 1:
             dist.reduce_scatter_tensor(rows, part, op=dist.ReduceOp.SUM)
@@ -742,7 +765,9 @@ def run_group_sharded(args):
         tfl = flops_ffn_active(cfg) / (ms_step * 1e-3) / 1e12
         rec = config_record(cfg, "ffn", world, args.flush_l2)
         rec["parallelism"] = (f"group-sharded x{world}: each rank holds the weights of a contiguous range of groups, routing "
-                              "replicated, fp32 parts summed by one NCCL reduce-scatter over token rows")
+                              "replicated, " + ("the down projection adds its rows into the owner ranks' fp32 shards over peer "
+                                                "memory (reduce-scatter fused into the kernel)" if args.fused else
+                                                "fp32 parts summed by one NCCL reduce-scatter over token rows"))
         print(json.dumps({
             "metric": METRIC, "value": T * args.steps / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
@@ -1014,6 +1039,8 @@ def main():
     ap.add_argument("--shard", default="tokens", choices=["tokens", "groups"],
                     help="multi-GPU partition: token shards with replicated weights (no collective), or group "
                          "shards (tensor parallel over the pruned dimension) with one reduce-scatter per step")
+    ap.add_argument("--fused", action="store_true",
+                    help="--shard groups: fuse the reduce-scatter into the down projection (adds over peer memory)")
     ap.add_argument("--premasked", action="store_true",
                     help="oproj: feed an attention output that already has zeros for inactive pairs")
     ap.add_argument("--kaxis", default="auto", choices=["auto", "group", "owner"],

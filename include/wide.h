@@ -305,6 +305,32 @@ WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_
              void* workspace, size_t workspace_bytes, unsigned flags);
 
 /*
+ * wide_ffn_tp -- the FFN part of one rank when the groups are sharded over GPUs, with the
+ * reduce-scatter of the parts fused into the down projection (Eq. 10 summed over this rank's groups;
+ * the sum over ranks is a reduce-scatter over token rows).  Prefill sizes, tensor-core path only.
+ *
+ * x, w_gate, w_up, w_down, mask_bits_local, perm, counts, token_order, token_rank: as for wide_ffn on
+ * this rank's weight shard (d_ff_local = this rank's groups * group; the mask sliced with
+ * wide_mask_slice and reordered with wide_reorder).
+ *   y_shards   HOST array of `world` DEVICE pointers: y_shards[r] = the fp32 shard
+ *              [rows_per_rank, hidden] of rank r, which owns token rows [r * rows_per_rank,
+ *              (r+1) * rows_per_rank); peer-mapped memory of the other GPUs for r != this rank
+ *              (read when the call is made, not kept).  world <= 8, world * rows_per_rank >= tokens.
+ * The down projection's epilogue adds every row of this rank's part into the shard of the rank
+ * that owns the row (red.global.add.f32 over peer memory: plain peer stores, no multicast, no TMA on
+ * peer memory).  The caller synchronises the ranks twice: every shard must be ZERO before any
+ * rank's call starts, and a shard is complete when the calls of ALL ranks have finished.  A token
+ * tile none of whose tokens uses any of this rank's groups sends nothing.
+ * Errors: INVALID_ARG, UNSUPPORTED_SHAPE (anything the tensor-core prefill path of wide_ffn does not
+ * take), ALIGNMENT, WORKSPACE (wide_workspace_bytes(WIDE_OP_FFN, ...) is enough), CUDA.
+ */
+WIDE_API int wide_ffn_tp(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,
+                         const void* w_down, int dtype, int tokens, int hidden, int d_ff_local, int group,
+                         const uint32_t* mask_bits_local, const int32_t* perm, const int32_t* counts,
+                         const int32_t* token_order, const int32_t* token_rank, float* const* y_shards, int world,
+                         int rows_per_rank, void* workspace, size_t workspace_bytes);
+
+/*
  * wide_oproj -- Eq. 2 / Eq. 10:  y[t,:] = sum_{g : M[t,g]=1} a[t, gG:(g+1)G] Wo[:, gG:(g+1)G]^T,
  * a = attention output flattened head-major [tokens, attn_dim], group g = channels [gG, (g+1)G).
  *   perm, counts: outputs of wide_reorder for this mask, or both NULL.  The prefill path has two

@@ -29,7 +29,7 @@ EXPORTS = ["wide_create", "wide_destroy", "wide_status", "wide_set_wait_limit_ns
            "wide_profile_end", "wide_launch_count", "wide_selftest_wait", "wide_strerror",
            "wide_version", "wide_workspace_bytes", "wide_route", "wide_route_static", "wide_route_pair_prepared_bytes",
            "wide_route_pair_norm_workspace_bytes", "wide_route_pair_prepare", "wide_route_pair_norm", "wide_reorder",
-           "wide_mask_slice",
+           "wide_mask_slice", "wide_ffn_tp",
            "wide_ffn",
            "wide_oproj", "wide_attn", "wide_qproj", "wide_unpermute"]
 
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.wide_ffn.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int,
                              _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
                              _c_void_p, _c_int, _c_void_p, _c_size_t, _c_uint]
+    lib.wide_ffn_tp.argtypes = [_c_void_p] * 6 + [_c_int] * 5 + [_c_void_p] * 6 + [_c_int, _c_int, _c_void_p, _c_size_t]
     lib.wide_oproj.argtypes = [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_int,
                                _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int,
                                _c_void_p, _c_size_t, _c_uint]
@@ -324,6 +325,24 @@ def wide_mask_slice(ctx: Context, mask_bits: torch.Tensor, n_groups: int, group_
     rc = ctx.lib.wide_mask_slice(ctx.handle, _stream(), _ptr(mask_bits), T, n_groups, group_begin, group_end, _ptr(out))
     _check(rc, "wide_mask_slice")
     return out
+
+
+def wide_ffn_tp(ctx: Context, x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, group: int,
+                mask_bits_local: torch.Tensor, meta: Dict[str, torch.Tensor], shard_ptrs, rows_per_rank: int):
+    """One rank's group-sharded FFN part, added straight into the fp32 shards of the ranks that own
+    the token rows.  ``shard_ptrs``: one device address per rank (ints), e.g. ``t.data_ptr()`` of a
+    local tensor for this rank and the peer-mapped addresses of the others."""
+    T, D = x.shape
+    d_ff = w_gate.shape[0]
+    world = len(shard_ptrs)
+    table = (ctypes.c_void_p * world)(*[ctypes.c_void_p(int(p)) for p in shard_ptrs])
+    nbytes = workspace_bytes(OP_FFN, BF16, T, D, d_ff, group, d_ff // group)
+    ws = ctx.workspace(nbytes, slot=0)
+    rc = ctx.lib.wide_ffn_tp(ctx.handle, _stream(), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _dtype_code(x), T, D,
+                             d_ff, group, _ptr(mask_bits_local), _ptr(meta["perm"]), _ptr(meta["counts"]),
+                             _ptr(meta.get("token_order")), _ptr(meta.get("token_rank")),
+                             ctypes.cast(table, ctypes.c_void_p), world, rows_per_rank, _ptr(ws), ws.numel())
+    _check(rc, "wide_ffn_tp")
 
 
 def wide_ffn(ctx: Context, x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor,

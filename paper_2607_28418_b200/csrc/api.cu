@@ -331,6 +331,31 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
     }
 }
 
+int wide_ffn_tp(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up, const void* w_down,
+                int dtype, int tokens, int hidden, int d_ff_local, int group, const uint32_t* mask_bits_local,
+                const int32_t* perm, const int32_t* counts, const int32_t* token_order, const int32_t* token_rank,
+                float* const* y_shards, int world, int rows_per_rank, void* workspace, size_t workspace_bytes) {
+    if (!ctx || !x || !w_gate || !w_up || !w_down || !mask_bits_local || !perm || !counts || !y_shards)
+        return WIDE_ERR_INVALID_ARG;
+    if (tokens < 0 || hidden <= 0 || d_ff_local <= 0 || group <= 0 || d_ff_local % group != 0) return WIDE_ERR_INVALID_ARG;
+    if (world < 1 || world > 8 || rows_per_rank <= 0 || static_cast<long long>(world) * rows_per_rank < tokens)
+        return WIDE_ERR_INVALID_ARG;
+    if ((token_order == nullptr) != (token_rank == nullptr)) return WIDE_ERR_INVALID_ARG;
+    for (int r = 0; r < world; ++r)
+        if (!y_shards[r] || !wide_aligned16(y_shards[r])) return WIDE_ERR_INVALID_ARG;
+    if (d_ff_local / group > WIDE_MAX_GROUPS) return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (dtype != WIDE_BF16 || hidden % 64 != 0 || (group != 64 && group != 128 && group != 256 && group != 512) ||
+        !ctx->encode_tiled)
+        return WIDE_ERR_UNSUPPORTED_SHAPE;
+    if (!wide_aligned16(x) || !wide_aligned16(w_gate) || !wide_aligned16(w_up) || !wide_aligned16(w_down) ||
+        !wide_aligned16(workspace))
+        return WIDE_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < inner_scratch(dtype, tokens, hidden, d_ff_local)) return WIDE_ERR_WORKSPACE;
+    return wide_launch_ffn_prefill_tp(ctx, static_cast<cudaStream_t>(stream), x, w_gate, w_up, w_down, tokens, hidden,
+                                      d_ff_local, group, mask_bits_local, perm, counts, token_order, token_rank, y_shards,
+                                      world, rows_per_rank, workspace);
+}
+
 int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_o, int dtype,
                int tokens, int hidden, int attn_dim, int group, const uint32_t* mask_bits,
                const int32_t* perm, const int32_t* counts, const int32_t* token_order,

@@ -136,6 +136,10 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
                                const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts,
                                const int32_t* token_order, const int32_t* token_rank, void* y,
                                int out_dtype, void* h, void* acc, unsigned flags);
+int wide_launch_ffn_prefill_tp(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
+                               const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
+                               const int32_t* perm, const int32_t* counts, const int32_t* token_order,
+                               const int32_t* token_rank, float* const* shards, int world, int rows_per_rank, void* h);
 int wide_launch_scores_tc(wide_ctx* ctx, cudaStream_t s, const void* x, const void* w_router, int T, int NG,
                           int ld, int D, float* scores, float* wnorm, int max_split, int* ksplit_out, int* chain_out);
 // `a_masked` is scratch [T, K] bf16, `acc` scratch [T, D] fp32.

@@ -99,6 +99,26 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Output of the down / output projection when the groups are sharded over GPUs (tensor parallelism
+// over the pruned dimension): this rank's tile is a PART of y (Eq. 10 summed over this rank's groups
+// only), and the sum over ranks is a reduce-scatter over token rows.  Fused here: instead of storing
+// its part and handing it to a collective, the epilogue adds every row straight into the fp32 shard
+// of the rank that owns the row, with red.global.add over peer memory (plain peer stores through
+// NVLink; no multicast, no TMA).  base[r] = rank r's shard [rows_per_rank, N] fp32, zero before any
+// rank starts and complete once every rank's kernel has finished (the caller's two barriers).
+// world == 0: ordinary output.
+struct PeerOut {
+    float* base[8];
+    int world;
+    int rows_per_rank;
+};
+
+__device__ __forceinline__ void red_add_f32x4(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
+                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+                 : "memory");
+}
+
 // ======================================================================================= down
 // Y[T, N] = A[T, K] * B[N, K]^T with K split into groups of G; group g is skipped for a token tile
 // when no token of the tile has bit g set (mask_bits == nullptr: nothing is skipped).
@@ -109,7 +129,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             int G, void* __restrict__ Y,
             int out_bf16, int ksplit, const __nv_bfloat16* __restrict__ aux_w, int aux_rows,
             float* __restrict__ aux_norm, const int32_t* __restrict__ sel_counts, int sel_thr, int acc_split,
-            int* __restrict__ status, unsigned long long wait_ns) {
+            const PeerOut peer, int* __restrict__ status, unsigned long long wait_ns) {
     constexpr int kBBytes = BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -267,7 +287,15 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int i = 0; i < 32; ++i) r[i] = 0u;
                 }
                 const int col = n * BN + c0;
-                if (row < T && col + 32 <= N) {
+                if (peer.world > 0) {
+                    // this rank's part of the row, added into the shard of the rank that owns the row
+                    if (any && row < T && col + 32 <= N) {
+                        float* dst = peer.base[row / peer.rows_per_rank] +
+                                     static_cast<size_t>(row % peer.rows_per_rank) * N + col;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) red_add_f32x4(dst + 4 * v, r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                } else if (row < T && col + 32 <= N) {
                     if (out_bf16) {
                         uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(row) * N + col);
 #pragma unroll
@@ -345,7 +373,7 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const uint32_t* __restrict__ mask_bits, const int32_t* __restrict__ order, int words, int T, int N,
                int K, int G, void* __restrict__ Y,
                int out_bf16, int n_n, int box_n, unsigned* __restrict__ queue, const int32_t* __restrict__ sel_counts,
-               int sel_thr, int* __restrict__ status, unsigned long long wait_ns) {
+               int sel_thr, const PeerOut peer, int* __restrict__ status, unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
     if (wide_kaxis_group_chosen(sel_counts, K / G, T, sel_thr)) return;   // the per-group kernel runs instead
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -552,7 +580,15 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     const int col = cbase + c0;
                     const int ncol = whole ? 32 : 16;
-                    if (row < T && col + ncol <= N) {
+                    if (peer.world > 0) {
+                        if (any && row < T && col + ncol <= N) {
+                            float* dst = peer.base[row / peer.rows_per_rank] +
+                                         static_cast<size_t>(row % peer.rows_per_rank) * N + col;
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                if (4 * v < ncol) red_add_f32x4(dst + 4 * v, r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                        }
+                    } else if (row < T && col + ncol <= N) {
                         if (out_bf16) {
                             uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(Y) + static_cast<size_t>(row) * N + col);
 #pragma unroll
@@ -986,7 +1022,8 @@ template <int BN>
 int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                 int N, int K, int G, void* Y, int out_dtype, int b_rows = -1, const char* name = "prefill_down",
                 int ksplit = 1, float* aux_norm = nullptr, const int32_t* order = nullptr,
-                const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, int acc_split = 1) {
+                const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, int acc_split = 1,
+                const PeerOut* peer = nullptr) {
     CUtensorMap tmA, tmB;
     if (b_rows < 0) b_rows = N;  // rows of B that exist; rows up to N beyond them read as zero
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, kBM) || !make_tmap_bf16(ctx, &tmB, B, b_rows, K, BN)) return WIDE_ERR_CUDA;
@@ -999,7 +1036,7 @@ int launch_down(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, con
     WideLaunch l(ctx, s, name);
     down_kernel<BN><<<grid, 192, smem, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                             ksplit, static_cast<const __nv_bfloat16*>(B), b_rows, aux_norm, sel_counts, sel_thr,
-                                            acc_split, ctx->d_status, ctx->wait_ns);
+                                            acc_split, peer ? *peer : PeerOut{}, ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -1024,7 +1061,7 @@ double pick_down256_tiling(int sm, int T, int N, int* n_n_out, int* wmax_out) {
 // (about 0.8 of the time per row), 128-row tiles quantise better over the SMs.
 int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                      int N, int K, int G, void* Y, int out_dtype, const int32_t* order,
-                     const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER) {
+                     const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, const PeerOut* peer = nullptr) {
     const int sm = ctx->sm_count;
     const int t128 = ((T + 127) / 128) * ((N + 255) / 256);
     int n_n = (N + 255) / 256, wmax = 256;
@@ -1032,7 +1069,7 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     const double cost256 = pick_down256_tiling(sm, T, N, &n_n, &wmax) * 2.0 * 0.8;
     if (cost128 <= cost256)
         return launch_down<256>(ctx, s, A, B, mask_bits, T, N, K, G, Y, out_dtype, -1, "prefill_down", 1, nullptr, order,
-                                sel_counts, sel_thr);
+                                sel_counts, sel_thr, 1, peer);
     CUtensorMap tmA, tmB;
     if (!make_tmap_bf16(ctx, &tmA, A, T, K, 256) || !make_tmap_bf16(ctx, &tmB, B, N, K, wmax)) return WIDE_ERR_CUDA;
     WIDE_CUDA_CHECK(cudaFuncSetAttribute(down256_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2));
@@ -1042,7 +1079,7 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     WideLaunch l(ctx, s, "prefill_down");
     down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                              n_n, wmax, reinterpret_cast<unsigned*>(ctx->d_status) + 8, sel_counts, sel_thr,
-                                             ctx->d_status, ctx->wait_ns);
+                                             peer ? *peer : PeerOut{}, ctx->d_status, ctx->wait_ns);
     return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
@@ -1154,6 +1191,25 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
     const KaxisPlan plan = plan_kaxis(G, Dff / G, out_dtype, true, flags);
     return launch_kaxis(ctx, s, plan, h, token_rank, nullptr, h, wd, T, D, Dff, G, mask_bits, perm, counts, token_order,
                         token_rank, y, out_dtype, acc, "prefill_down_group");
+}
+
+// Group-sharded FFN part with the reduce-scatter fused into the down projection's epilogue (see
+// PeerOut): gate/up on this rank's groups, then the owner-computes down kernel adding its tiles into
+// the shards of the ranks that own the rows.
+int wide_launch_ffn_prefill_tp(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, const void* wu,
+                               const void* wd, int T, int D, int Dff, int G, const uint32_t* mask_bits,
+                               const int32_t* perm, const int32_t* counts, const int32_t* token_order,
+                               const int32_t* token_rank, float* const* shards, int world, int rows_per_rank, void* h) {
+    if (T == 0) return WIDE_OK;
+    PeerOut peer{};
+    peer.world = world;
+    peer.rows_per_rank = rows_per_rank;
+    for (int r = 0; r < world; ++r) peer.base[r] = shards[r];
+    int rc = (G == 64) ? launch_gateup<64, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h)
+                       : launch_gateup<128, false>(ctx, s, x, wg, wu, T, D, Dff, G, perm, counts, token_rank, h);
+    if (rc != WIDE_OK) return rc;
+    return launch_down_auto(ctx, s, h, wd, mask_bits, T, D, Dff, G, nullptr, WIDE_F32, token_order, nullptr, WIDE_KAXIS_NEVER,
+                            &peer);
 }
 
 // y[t, gG:(g+1)G] = x_t W[gG:(g+1)G, :]^T for active (t, g), exact zeros elsewhere (Algorithm 2 with a

@@ -102,3 +102,36 @@ def test_oproj_parts_add_up(ctx, world, flags):
     torch.cuda.synchronize()
     assert ctx.status() == 0
     assert_close(total, wo.oproj(a, w_o, mask, G), f"O-projection, sum of {world} parts")
+
+
+@pytest.mark.parametrize("T,world", [(640, 2), (640, 4), (1100, 8), (2048, 4)])
+def test_fused_reduce_scatter_adds_every_part_into_the_owners_shard(ctx, T, world):
+    """wide_ffn_tp: the down projection's epilogue adds this rank's part of every token row into the
+    fp32 shard of the rank that owns the row.  The ranks are emulated one after the other on one GPU
+    (the adds are one-sided: no rank waits on another); their shards are separate local buffers, the
+    same instruction that would cross NVLink adds into them.  Shards concatenated = the full FFN."""
+    from paper_2607_28418_b200 import binding
+    cfg = synth.WideConfig("tp", tokens=T, hidden=512, d_ff=4096, group=128, k=12, router="clustered" if world == 8 else "random")
+    case = synth.make_ffn_case(cfg, 7)
+    NG, G = cfg.n_groups, cfg.group
+    mask = wo.mask_topk(wo.route_scores(case["x"], case["w_router"]), cfg.k)
+    bits = bits_to_dev(wo.pack_mask_bits(mask))
+    xd = to_dev(case["x"], "bf16")
+    rows_per_rank = (T + world - 1) // world
+    shards = [torch.zeros((rows_per_rank, cfg.hidden), dtype=torch.float32, device="cuda") for _ in range(world)]
+    ptrs = [t.data_ptr() for t in shards]
+    for r in range(world):
+        g0, g1 = binding.group_range(NG, world, r)
+        c0, c1 = g0 * G, g1 * G
+        wg, wu = to_dev(case["w_gate"][c0:c1], "bf16"), to_dev(case["w_up"][c0:c1], "bf16")
+        wd = to_dev(np.ascontiguousarray(case["w_down"][:, c0:c1]), "bf16")
+        local_bits = binding.wide_mask_slice(ctx, bits, NG, g0, g1)
+        meta = binding.wide_reorder(ctx, local_bits, g1 - g0, 128)
+        binding.wide_ffn_tp(ctx, xd, wg, wu, wd, G, local_bits, meta, ptrs, rows_per_rank)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    y = torch.cat(shards, dim=0)[:T]
+    ref = wo.ffn(case["x"], case["w_gate"], case["w_up"], case["w_down"], mask, G)
+    assert_close(y, ref, f"fused reduce-scatter, {world} ranks")
+    if world * rows_per_rank > T:
+        assert (torch.cat(shards, dim=0)[T:] == 0).all().item()     # rows past the batch are never touched
