@@ -291,7 +291,7 @@ def cublas_dense_context(torch, d, reps=10):
             "dense_tflops": 6.0 * x.shape[0] * wg.shape[0] * x.shape[1] / (ms * 1e-3) / 1e12}
 
 
-def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 32, 64), replays=300):
+def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 16, 32, 64), replays=300):
     """Llama-3-8B-shaped decode FFN (hidden 4096, d_ff 14336, 112 groups of 128, top-56, random
     router) at each batch size: the FFN call replayed as a graph over two rotating copies of the
     weights (704 MB > 4x L2, so every replay streams from HBM), and the whole step (route + FFN)."""
@@ -343,6 +343,41 @@ def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 32, 64), 
     return {"workload": "llama8b_decode", "router": "random", "k": cfg.k, "n_groups": cfg.n_groups,
             "bytes": "union groups x 3 x group x hidden x 2 B (gate, up, down weights)", "peak": peaks["hbm_gbs"],
             "peak_source": peaks["source"], "replays": replays, "clocks": clocks, "points": out}
+
+
+def oproj_13b_record(torch, binding, ctx, peaks, replays=50):
+    """Llama-2-13B-shaped head-group-masked output projection (T = 4096, 40 heads of 128 in 10 groups,
+    top-5): the wide_oproj call alone as a graph, with the library's own choice of K-axis kernel and
+    with the owner-computes kernel forced, and with every group active (the dense run of the same
+    call)."""
+    cfg = synth.CONFIGS["llama13b_layer"]
+    case = synth.make_oproj_case(cfg, 0)
+    d = {k: binding.upload(v, "bf16") for k, v in case.items()}
+    T, NG, G = cfg.tokens, cfg.attn_n_groups, cfg.attn_group
+    y = torch.empty((T, cfg.hidden), dtype=torch.bfloat16, device=d["x"].device)
+    out = {"workload": "llama13b_layer", "op": "oproj", "tokens": T, "n_groups": NG, "group": G}
+    for k in (cfg.attn_k, NG):
+        bits, _ = binding.wide_route(ctx, d["x"], d["w_router_attn"], NG, k)
+        meta = binding.wide_reorder(ctx, bits, NG, 128)
+        for name, flags in (("auto", 0), ("owner", binding.FLAG_KAXIS_OWNER)):
+            def call():
+                binding.wide_oproj(ctx, d["attn_out"], d["w_o"], G, bits, meta, y=y, flags=flags)
+            for _ in range(3):
+                call()
+            g = graph_of(torch, call)
+            g()
+            ms = event_ms(torch, g, replays)
+            tag = f"k{k}_{name}"
+            out[tag + "_ms"] = ms
+            if k == cfg.attn_k:
+                tfl = 2.0 * T * k * G * cfg.hidden / (ms * 1e-3) / 1e12
+                out[tag + "_active_tflops"] = tfl
+                out[tag + "_frac_of_bf16_peak"] = tfl / peaks["bf16_tflops"]
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during the O-projection record")
+    out["speedup_vs_all_groups_active"] = out[f"k{NG}_auto_ms"] / out[f"k{cfg.attn_k}_auto_ms"]
+    out["ideal"] = NG / cfg.attn_k
+    return out
 
 
 # ------------------------------------------------------------------------------- our arm
@@ -581,13 +616,14 @@ def run_ours(args):
         step()
 
     # ---- extra records of the default single-GPU run: seconds-long replay, cuBLAS context, decode sweep
-    sustained = cublas = decode_rec = None
+    sustained = cublas = decode_rec = oproj_rec = None
     if world == 1 and not decode and not args.no_extras:
         sustained = sustained_record(torch, run_step, ms_total / args.steps, T, flops_ffn_active(cfg, oproj), peaks, local)
         if not oproj:
             cublas = cublas_dense_context(torch, d)
             if cfg.name == "llama7b_prefill":
                 decode_rec = decode_sweep(torch, binding, ctx, peaks, local)
+                oproj_rec = oproj_13b_record(torch, binding, ctx, peaks)
 
     # ---- roofline of the dominant kernel (largest share of the timed region)
     kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
@@ -646,6 +682,8 @@ def run_ours(args):
             line["cublas_dense_context"] = cublas
         if decode_rec:
             line["decode"] = decode_rec
+        if oproj_rec:
+            line["oproj_13b"] = oproj_rec
         if world == 1 and not args.no_cpu_baseline and not oproj:
             sample = min(T, args.oracle_tokens)
             _, ms1 = time_oracle(case, cfg, sample, 1, 0)
