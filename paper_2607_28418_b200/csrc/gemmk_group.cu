@@ -32,7 +32,15 @@ namespace {
 
 using namespace wptx;
 
-constexpr int kStagesK = 4;
+// bf16 sums: 4 stages, 8 epilogue warps.  fp32 sums move twice the bytes per item through a chain of
+// dependent steps (TMEM load, staging, reduction), which made the epilogue the longer leg of the TMEM
+// double buffer (tensor pipe 24 % active); that variant trades a ring stage for four more epilogue warps.
+template <bool kBf16Red> struct KCfg {
+    static constexpr int kStages = kBf16Red ? 4 : 3;
+    static constexpr int kEpiWarps = kBf16Red ? 8 : 12;
+    static constexpr int kThreads = 32 * (6 + kEpiWarps);   // TMA, MMA, 4 gather warps, epilogue warps
+    static constexpr int kStaging = kEpiWarps * 4096;       // 32 rows x 128 B per epilogue warp
+};
 constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kBN = 256;
@@ -40,9 +48,9 @@ constexpr int kABytes = kBM * kBK * 2;          // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;          // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;  // 48 KB
 constexpr int kAccCols = 256;
-constexpr int kThreadsK = 448;                  // TMA, MMA, 4 gather warps, 8 epilogue warps
-constexpr int kStagingBytes = 8 * 4096;         // 32 rows x 128 B per epilogue warp
-constexpr int kSmemK = kStagesK * kStageBytes + kStagingBytes + (2 * kStagesK + 4) * 8 + 16 + 1024;
+template <bool kBf16Red> constexpr int smem_k() {
+    return KCfg<kBf16Red>::kStages * kStageBytes + KCfg<kBf16Red>::kStaging + (2 * KCfg<kBf16Red>::kStages + 4) * 8 + 16 + 1024;
+}
 
 __device__ __forceinline__ void red_add_v4_f32(void* p, uint4 v) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(v.x)),
@@ -79,13 +87,16 @@ struct ItemMap {
 };
 
 template <bool kBf16Red>
-__global__ void __launch_bounds__(kThreadsK, 1)
+__global__ void __launch_bounds__(KCfg<kBf16Red>::kThreads, 1)
 gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16* __restrict__ A, int lda,
                    const int32_t* __restrict__ perm, const int32_t* __restrict__ counts,
                    const int32_t* __restrict__ a_row_of_token, int NG, int T, int N, int G, void* __restrict__ Y,
                    int thr_q, int* __restrict__ status, unsigned long long wait_ns) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ int s_off[WIDE_MAX_GROUPS + 1];
+    constexpr int kStagesK = KCfg<kBf16Red>::kStages;
+    constexpr int kEpiWarps = KCfg<kBf16Red>::kEpiWarps;
+    constexpr int kStagingBytes = KCfg<kBf16Red>::kStaging;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (!wide_kaxis_group_chosen(counts, NG, T, thr_q)) return;   // the owner-computes kernel runs instead
 
@@ -104,7 +115,7 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull + 8 * b, 1);
-            mbar_init(tempty + 8 * b, 8);
+            mbar_init(tempty + 8 * b, kEpiWarps);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -240,14 +251,17 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
         cp_async_wait_all();
         if (!ok && lane == 0) atomicExch(status, WIDE_ERR_TIMEOUT);
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 6..13)
-        // Warps w and w + 4 share a TMEM lane quarter and split the accumulator's columns in two.
+        // ------------------------------------------------------------------ epilogue (warps 6 ..)
+        // Warps w, w + 4 (, w + 8) share a TMEM lane quarter and split the accumulator's columns.
         // Thread = accumulator row (TMEM lane).  A chunk is 128 bytes of an output row (32 fp32 or
         // 64 bf16 columns): the thread writes its row's chunk into the warp's staging tile (16-byte
         // pieces, piece v of row r in slot v ^ (r & 7)), then the warp reads it back 4 rows x 8
         // pieces at a time and reduces whole 128-byte lines into Y.
         const int q = warp & 3;
-        const int chalf = (warp - 6) >> 2;
+        const int part = (warp - 6) >> 2;
+        // column range of this warp: halves of 128, or thirds of 96 / 96 / 64
+        const int col_lo = kEpiWarps == 8 ? part * 128 : part * 96;
+        const int col_hi = kEpiWarps == 8 ? col_lo + 128 : (part == 2 ? kBN : col_lo + 96);
         uint4* stage = reinterpret_cast<uint4*>(staging + (warp - 6) * 4096);
         constexpr int kEsz = kBf16Red ? 2 : 4;
         constexpr int kChunkCols = 128 / kEsz;
@@ -263,7 +277,7 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
 #pragma unroll 1
-            for (int c0 = chalf * (kBN / 2); c0 < (chalf + 1) * (kBN / 2); c0 += kChunkCols) {
+            for (int c0 = col_lo; c0 < col_hi; c0 += kChunkCols) {
                 uint32_t r[32];
                 tmem_ld_32x32(taddr + c0, r);
                 if constexpr (kBf16Red) {
@@ -289,7 +303,7 @@ gemmk_group_kernel(const __grid_constant__ CUtensorMap tmB, const __nv_bfloat16*
                     for (int v = 0; v < 8; ++v)
                         stage[lane * 8 + (v ^ (lane & 7))] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                 }
-                if (c0 + kChunkCols >= (chalf + 1) * (kBN / 2)) {
+                if (c0 + kChunkCols >= col_hi) {
                     // the accumulator has been read out: hand it back before the last reductions
                     tc_fence_before_sync();
                     __syncwarp();
@@ -389,13 +403,13 @@ int wide_launch_gemmk_group_tc(wide_ctx* ctx, cudaStream_t s, const void* A, int
     const int NG = K / G;
     WideLaunch l(ctx, s, name);
     if (bf16_red) {
-        WIDE_CUDA_CHECK(cudaFuncSetAttribute(gemmk_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemK));
-        gemmk_group_kernel<true><<<ctx->sm_count, kThreadsK, kSmemK, s>>>(
+        WIDE_CUDA_CHECK(cudaFuncSetAttribute(gemmk_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_k<true>()));
+        gemmk_group_kernel<true><<<ctx->sm_count, KCfg<true>::kThreads, smem_k<true>(), s>>>(
             tmB, static_cast<const __nv_bfloat16*>(A), lda, perm, counts, a_row_of_token, NG, T, N, G, Y, thr_q,
             ctx->d_status, ctx->wait_ns);
     } else {
-        WIDE_CUDA_CHECK(cudaFuncSetAttribute(gemmk_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemK));
-        gemmk_group_kernel<false><<<ctx->sm_count, kThreadsK, kSmemK, s>>>(
+        WIDE_CUDA_CHECK(cudaFuncSetAttribute(gemmk_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_k<false>()));
+        gemmk_group_kernel<false><<<ctx->sm_count, KCfg<false>::kThreads, smem_k<false>(), s>>>(
             tmB, static_cast<const __nv_bfloat16*>(A), lda, perm, counts, a_row_of_token, NG, T, N, G, Y, thr_q,
             ctx->d_status, ctx->wait_ns);
     }
