@@ -41,7 +41,7 @@
 extern "C" {
 #endif
 
-#define WIDE_VERSION 100
+#define WIDE_VERSION 110
 
 #if defined(__GNUC__)
 #define WIDE_API __attribute__((visibility("default")))

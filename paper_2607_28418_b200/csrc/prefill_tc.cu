@@ -1100,13 +1100,14 @@ int launch_gateup(wide_ctx* ctx, cudaStream_t s, const void* x, const void* wg, 
 
 // Which K-axis kernel a prefill call uses.  Measured on the 13B output projection and on the 8B down
 // projection (T = 4096): the per-group kernel (Algorithm 3) costs c * p of the owner-computes kernel's
-// time, p = padded active fraction, with c = 1.35 (G = 512, bf16 sums), 2.05 (512, fp32 sums incl.
-// clearing and converting the scratch), 2.1 (256, bf16), 3.5 (256, fp32), 3.7 (128, bf16):
-// c = 0.6 + 380 * (bytes / 2) / G fits all five.  The first term is the tensor work (128 x 256 tiles move more operand bytes per
-// FLOP than the owner kernel's 256 x 256), the second the T*k*N partial sums that go through the
-// L2's reduction units.  The per-group kernel is taken when c * p <= 0.9.  Group sizes below 256
-// take part in the device-side choice only when the caller opts into bf16 sums; otherwise the choice
-// would add two empty launches to every call that stays with the owner-computes kernel.
+// time, p = padded active fraction, with c = 1.35 (G = 512, bf16 sums), 2.1 (256, bf16), 3.7 (128, bf16),
+// 2.0 (512, fp32 sums incl. clearing and converting the scratch), 3.1 (256, fp32), 5.5 (128, fp32):
+// c = 0.6 + beta / G with beta = 380 for bf16 sums and 640 for fp32 sums fits all six.  The first term is
+// the tensor work (128 x 256 tiles move more operand bytes per FLOP than the owner kernel's 256 x 256),
+// the second the T*k*N partial sums that go through the L2's reduction units.  The per-group kernel is
+// taken when c * p <= 0.9.  Group sizes below 256 take part in the device-side choice only when the
+// caller opts into bf16 sums; otherwise the choice would add two empty launches to every call that
+// stays with the owner-computes kernel.
 struct KaxisPlan {
     int thr_q;       // threshold of wide_kaxis_group_chosen
     bool bf16_red;   // reduce straight into the bf16 output
@@ -1126,7 +1127,7 @@ KaxisPlan plan_kaxis(int G, int NG, int out_dtype, bool have_perm, unsigned flag
     } else if (flags & WIDE_FLAG_KAXIS_GROUP) {
         p.thr_q = WIDE_KAXIS_ALWAYS;
     } else if (G >= 256 || (G >= 128 && (flags & WIDE_FLAG_REDUCE_BF16))) {
-        const double c = 0.6 + 380.0 * (p.bf16_red ? 1.0 : 2.0) / G;
+        const double c = 0.6 + (p.bf16_red ? 380.0 : 640.0) / G;
         p.thr_q = static_cast<int>(1024.0 * 0.9 / c);
     } else {
         p.thr_q = WIDE_KAXIS_NEVER;
