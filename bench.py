@@ -380,6 +380,38 @@ def oproj_13b_record(torch, binding, ctx, peaks, replays=50):
     return out
 
 
+def attn_13b_record(torch, binding, ctx, peaks, replays=30):
+    """Llama-2-13B-shaped head-group-masked causal attention, prefill (one sequence of 4096 positions,
+    40 heads of 128 in 10 groups, top-5): the wide_attn call alone as a graph; FLOPs counted per
+    active (token, head) pair over its visible keys."""
+    cfg = synth.CONFIGS["llama13b_layer"]
+    T, hd = cfg.tokens, 128
+    H, hpg, NG, k = cfg.attn_dim // hd, cfg.attn_group // hd, cfg.attn_n_groups, cfg.attn_k
+    oc = synth.make_oproj_case(cfg, 0)
+    ac = synth.make_attn_case(0, T, T, H, H, hd)
+    x, wr = binding.upload(oc["x"], "bf16"), binding.upload(oc["w_router_attn"], "bf16")
+    q, kk, v = (binding.upload(ac[n].reshape(T, H * hd), "bf16") for n in ("q", "k", "v"))
+    bits, _ = binding.wide_route(ctx, x, wr, NG, k)
+    meta = binding.wide_reorder(ctx, bits, NG, 128)
+    o = torch.empty_like(q)
+
+    def call():
+        binding.wide_attn(ctx, q, kk, v, H, H, hpg, meta, causal=True, o=o)
+    for _ in range(3):
+        call()
+    g = graph_of(torch, call)
+    g()
+    ms = event_ms(torch, g, replays)
+    if ctx.status() != 0:
+        raise RuntimeError("device status word set during the attention record")
+    mask = np.unpackbits(bits.cpu().numpy().view(np.uint8), axis=1, bitorder="little")[:, :NG].astype(bool)
+    flops = float((mask.sum(axis=1) * hpg * 4.0 * hd * (np.arange(T) + 1.0)).sum())
+    tfl = flops / (ms * 1e-3) / 1e12
+    return {"workload": "llama13b_layer", "op": "attn", "tokens": T, "heads": H, "head_dim": hd, "n_groups": NG, "k": k,
+            "ms": ms, "active_gflop": flops / 1e9, "active_tflops": tfl, "frac_of_bf16_peak": tfl / peaks["bf16_tflops"],
+            "frac_of_nominal_peak": tfl / NOMINAL_PEAKS["bf16_tflops"]}
+
+
 # ------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -616,7 +648,7 @@ def run_ours(args):
         step()
 
     # ---- extra records of the default single-GPU run: seconds-long replay, cuBLAS context, decode sweep
-    sustained = cublas = decode_rec = oproj_rec = None
+    sustained = cublas = decode_rec = oproj_rec = attn_rec = None
     if world == 1 and not decode and not args.no_extras:
         sustained = sustained_record(torch, run_step, ms_total / args.steps, T, flops_ffn_active(cfg, oproj), peaks, local)
         if not oproj:
@@ -624,6 +656,7 @@ def run_ours(args):
             if cfg.name == "llama7b_prefill":
                 decode_rec = decode_sweep(torch, binding, ctx, peaks, local)
                 oproj_rec = oproj_13b_record(torch, binding, ctx, peaks)
+                attn_rec = attn_13b_record(torch, binding, ctx, peaks)
 
     # ---- roofline of the dominant kernel (largest share of the timed region)
     kernels = {n: {"launches": v["launches"], "total_ms": round(v["total_ms"], 4),
@@ -684,6 +717,8 @@ def run_ours(args):
             line["decode"] = decode_rec
         if oproj_rec:
             line["oproj_13b"] = oproj_rec
+        if attn_rec:
+            line["attn_13b"] = attn_rec
         if world == 1 and not args.no_cpu_baseline and not oproj:
             sample = min(T, args.oracle_tokens)
             _, ms1 = time_oracle(case, cfg, sample, 1, 0)
