@@ -35,7 +35,7 @@ NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the part's data-s
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries,
 # keyed by (kernel, workload) -> (bytes, the summary under profiles/ it was read from).
 NCU_TRAFFIC_BYTES = {
-    ("prefill_gateup", "llama7b_prefill"): (355.4e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
+    ("prefill_gateup", "llama7b_prefill"): (292.3e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
     ("prefill_down", "llama7b_prefill"): (140.1e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
     # decode: captured at batch 8 (union 111 groups, 357.3 MB); traffic is proportional to the union
     ("decode_ffn_fused", "llama8b_decode"): (357.3e6 / 111, "profiles/decode_llama8b_batch8_fused_kernel.md"),

@@ -783,6 +783,9 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
             bool ok = true;
             GuSched sched(s_dbl, s_sgl, n_gs);
             GuItem w;
+            // A group's weight tile is read by the few CTAs that run the group's items side by side and
+            // is dead afterwards: it should leave L2 before x (which every item gathers from) and H.
+            const uint64_t wpol = l2_policy_evict_first();
             while (ok && sched.next(w)) {
                 const int crow = (w.gs / nsub) * G + (w.gs % nsub) * kItemCh;
                 for (int k = 0; k < nk; ++k, ++it) {
@@ -791,8 +794,8 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, wait_ns, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(full + 8 * s, kBBytes);
                     const uint32_t b_dst = smem_u32(base + s * kStageBytes) + kAB;
-                    tma_load_2d(b_dst, &tmG, k * kBK, crow, full + 8 * s);
-                    tma_load_2d(b_dst + BN * kBK * 2, &tmU, k * kBK, kLinear ? crow + BN : crow, full + 8 * s);
+                    tma_load_2d_hint(b_dst, &tmG, k * kBK, crow, full + 8 * s, wpol);
+                    tma_load_2d_hint(b_dst + BN * kBK * 2, &tmU, k * kBK, kLinear ? crow + BN : crow, full + 8 * s, wpol);
                 }
             }
             if (!ok) { report_timeout(status); abort_grace(); }
