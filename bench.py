@@ -39,6 +39,8 @@ NCU_TRAFFIC_BYTES = {
     ("prefill_down", "llama7b_prefill"): (140.1e6, "profiles/prefill_llama7b_gateup_down_kernels.md"),
     # decode: captured at batch 8 (union 111 groups, 357.3 MB); traffic is proportional to the union
     ("decode_ffn_fused", "llama8b_decode"): (357.3e6 / 111, "profiles/decode_llama8b_batch8_fused_kernel.md"),
+    # captured at batch 1 (union 56 groups, 180.4 MB)
+    ("decode_ffn_gemv", "llama8b_decode"): (180.4e6 / 56, "profiles/decode_llama8b_batch1_gemv_kernel.md"),
 }
 
 
@@ -291,7 +293,7 @@ def cublas_dense_context(torch, d, reps=10):
             "dense_tflops": 6.0 * x.shape[0] * wg.shape[0] * x.shape[1] / (ms * 1e-3) / 1e12}
 
 
-def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 16, 32, 64), replays=300):
+def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 16, 32, 64), replays=300, flags=0):
     """Llama-3-8B-shaped decode FFN (hidden 4096, d_ff 14336, 112 groups of 128, top-56, random
     router) at each batch size: the FFN call replayed as a graph over two rotating copies of the
     weights (704 MB > 4x L2, so every replay streams from HBM), and the whole step (route + FFN)."""
@@ -312,7 +314,7 @@ def decode_sweep(torch, binding, ctx, peaks, gpu_index, batches=(1, 8, 16, 32, 6
 
         def ffn(c):
             w = wsets[c]
-            binding.wide_ffn(ctx, x, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, None, y=y)
+            binding.wide_ffn(ctx, x, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, None, y=y, flags=flags)
 
         def whole(c):
             binding.wide_route(ctx, x, d["w_router"], cfg.n_groups, cfg.k, mask_bits=bits)
@@ -467,6 +469,7 @@ def run_ours(args):
         wsets.append({k: d[k].clone() for k in wkeys})
 
     kflags = {"auto": 0, "group": binding.FLAG_KAXIS_GROUP, "owner": binding.FLAG_KAXIS_OWNER}[args.kaxis]
+    dflags = binding.FLAG_DECODE_TC if args.decode_tc else 0
     if args.reduce_bf16:
         kflags |= binding.FLAG_REDUCE_BF16
 
@@ -475,10 +478,10 @@ def run_ours(args):
             binding.wide_qproj(ctx, x_in, w["w_q"], cfg.group, meta, y=y_out)
         elif oproj:
             binding.wide_oproj(ctx, d["attn_out"], w["w_o"], cfg.group, bits, meta, y=y_out,
-                               flags=(binding.FLAG_INPUT_MASKED if args.premasked else 0) | (0 if decode else kflags))
+                               flags=(binding.FLAG_INPUT_MASKED if args.premasked else 0) | (dflags if decode else kflags))
         else:
             binding.wide_ffn(ctx, x_in, w["w_gate"], w["w_up"], w["w_down"], cfg.group, bits, meta, y=y_out,
-                             flags=0 if decode else kflags)
+                             flags=dflags if decode else kflags)
     calls = {"n": 0}
 
     def step(k=cfg.k, slot=0, copy=None):
@@ -1119,6 +1122,8 @@ def main():
     ap.add_argument("--kaxis", default="auto", choices=["auto", "group", "owner"],
                     help="prefill K-axis kernel (down / output projection): per-group scatter-reduce, owner-computes, "
                          "or the library's own choice")
+    ap.add_argument("--decode-tc", action="store_true",
+                    help="decode with one or two tokens: the tensor-core kernel instead of the matrix-vector kernel")
     ap.add_argument("--reduce-bf16", action="store_true", help="per-group K-axis kernel: add partial sums in bf16")
     ap.add_argument("--kv-len", type=int, default=0, help="attn: number of keys (default: the workload's tokens)")
     ap.add_argument("--flush-l2", action="store_true")

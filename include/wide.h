@@ -41,7 +41,7 @@
 extern "C" {
 #endif
 
-#define WIDE_VERSION 110
+#define WIDE_VERSION 111
 
 #if defined(__GNUC__)
 #define WIDE_API __attribute__((visibility("default")))
@@ -91,8 +91,12 @@ extern "C" {
 #define WIDE_FLAG_REDUCE_BF16 64u   /* per-group form with a bf16 output: add the partial sums (one per active
                                       group of a token) in bf16 straight into the output instead of in fp32
                                       scratch; halves the reduction traffic.  Default when n_groups <= 16 */
+#define WIDE_FLAG_DECODE_TC 128u    /* decode path with at most WIDE_DECODE_GEMV_MAX_TOKENS tokens: take the
+                                      tensor-core kernel instead of the matrix-vector kernel (the GEMV
+                                      dispatch for tiny M of Appendix B), which is the default there */
 
 #define WIDE_DECODE_MAX_TOKENS 64
+#define WIDE_DECODE_GEMV_MAX_TOKENS 2
 #define WIDE_MAX_GROUPS 256
 
 typedef struct wide_ctx wide_ctx;
@@ -295,7 +299,10 @@ WIDE_API int wide_mask_slice(wide_ctx* ctx, void* stream, const uint32_t* mask_b
  *       is the same either way, block skipping in the down projection is not.
  *   y  out [tokens, hidden] of out_dtype
  * Tensor-core paths need dtype bf16, hidden % 64 == 0, group in {64,128,256,512}; other shapes
- * need WIDE_FLAG_SIMT (hidden % 4 == 0, group % 4 == 0).
+ * need WIDE_FLAG_SIMT (hidden % 4 == 0, group % 4 == 0).  The decode path serves up to
+ * WIDE_DECODE_GEMV_MAX_TOKENS tokens with matrix-vector products on the CUDA cores (each needed
+ * weight byte read once by plain loads) and more with the tensor-core kernel; WIDE_FLAG_DECODE_TC
+ * takes the latter for any token count.  Same shapes, same results within the tolerance.
  * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, ALIGNMENT, WORKSPACE, CUDA.
  */
 WIDE_API int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, const void* w_up,

@@ -21,7 +21,9 @@ ROUTE_TOPK, ROUTE_PAIR_ARGMAX = 0, 1
 OP_ROUTE, OP_REORDER, OP_FFN, OP_OPROJ, OP_UNPERMUTE = 0, 1, 2, 3, 4
 FLAG_NONE, FLAG_SIMT, FLAG_FORCE_PREFILL, FLAG_FORCE_DECODE, FLAG_INPUT_MASKED = 0, 1, 2, 4, 8
 FLAG_KAXIS_GROUP, FLAG_KAXIS_OWNER, FLAG_REDUCE_BF16 = 16, 32, 64
+FLAG_DECODE_TC = 128
 DECODE_MAX_TOKENS = 64
+DECODE_GEMV_MAX_TOKENS = 2
 MAX_GROUPS = 256
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 

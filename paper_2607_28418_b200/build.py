@@ -21,7 +21,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libwide.so")
 
-SOURCES = ["api.cu", "route.cu", "reorder.cu", "ffn_simt.cu", "prefill_tc.cu", "gemmk_group.cu", "decode_tc.cu", "attn_tc.cu", "attn_decode.cu", "selftest.cu"]
+SOURCES = ["api.cu", "route.cu", "reorder.cu", "ffn_simt.cu", "prefill_tc.cu", "gemmk_group.cu", "decode_tc.cu", "decode_gemv.cu", "attn_tc.cu", "attn_decode.cu", "selftest.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

@@ -326,6 +326,9 @@ int wide_ffn(wide_ctx* ctx, void* stream, const void* x, const void* w_gate, con
             return wide_launch_ffn_prefill_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
                                               perm, counts, token_order, token_rank, y, out_dtype, workspace, acc, flags);
         default:
+            if (!(flags & WIDE_FLAG_DECODE_TC) && wide_decode_gemv_fits(true, tokens, hidden, d_ff, group))
+                return wide_launch_decode_gemv(ctx, s, true, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group,
+                                               mask_bits, y, out_dtype, workspace);
             return wide_launch_ffn_decode_tc(ctx, s, x, w_gate, w_up, w_down, tokens, hidden, d_ff, group, mask_bits,
                                              y, out_dtype, workspace);
     }
@@ -386,6 +389,9 @@ int wide_oproj(wide_ctx* ctx, void* stream, const void* attn_out, const void* w_
             return wide_launch_oproj_prefill_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, perm,
                                                 counts, token_order, token_rank, y, out_dtype, workspace, acc, flags);
         default:
+            if (!(flags & WIDE_FLAG_DECODE_TC) && wide_decode_gemv_fits(false, tokens, hidden, attn_dim, group))
+                return wide_launch_decode_gemv(ctx, s, false, attn_out, nullptr, nullptr, w_o, tokens, hidden, attn_dim,
+                                               group, mask_bits, y, out_dtype, workspace);
             return wide_launch_oproj_decode_tc(ctx, s, attn_out, w_o, tokens, hidden, attn_dim, group, mask_bits, y,
                                                out_dtype, workspace);
     }

@@ -18,7 +18,7 @@ struct wide_ctx {
     int device;
     int sm_count;
     int* d_status;          // [0] device status word (WIDE_OK or WIDE_ERR_TIMEOUT), [1] reorder ticket,
-                            // [4..5] grid-barrier counters of the decode kernel, [8..9] tile queue of the
+                            // [4..5] grid-barrier counters of the decode kernels, [6] channel pool of the GEMV decode kernel, [8..9] tile queue of the
                             // 256-row down projection (16 ints in all)
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
@@ -167,6 +167,13 @@ int wide_launch_ffn_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* x, cons
 int wide_launch_oproj_decode_tc(wide_ctx* ctx, cudaStream_t s, const void* a, const void* wo, int T,
                                 int D, int K, int G, const uint32_t* mask_bits, void* y,
                                 int out_dtype, void* ws);
+
+// CUDA-core decode path for at most WIDE_DECODE_GEMV_MAX_TOKENS tokens (csrc/decode_gemv.cu).  `act` is x
+// (FFN) or the attention output (O-projection, wg = wu = nullptr); `ws` as for the tensor-core kernel.
+bool wide_decode_gemv_fits(bool is_ffn, int T, int D, int inner, int G);
+int wide_launch_decode_gemv(wide_ctx* ctx, cudaStream_t s, bool is_ffn, const void* act, const void* wg, const void* wu,
+                            const void* wd, int T, int D, int inner, int G, const uint32_t* mask_bits, void* y,
+                            int out_dtype, void* ws);
 
 // 2-D bf16 row-major [rows, cols] tensor map, box = [box_rows, 64 columns], 128-byte swizzle.
 bool wide_make_tmap_bf16(const wide_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
