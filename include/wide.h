@@ -41,7 +41,7 @@
 extern "C" {
 #endif
 
-#define WIDE_VERSION 111
+#define WIDE_VERSION 112
 
 #if defined(__GNUC__)
 #define WIDE_API __attribute__((visibility("default")))
@@ -159,8 +159,10 @@ WIDE_API size_t wide_workspace_bytes(int op, int dtype, int tokens, int hidden, 
  * depend on summation order.  (bf16, TOPK, hidden % 64 == 0: scores come from the tensor cores in
  * fp32 and every group closer to the selection boundary than an error bound is re-scored exactly
  * in fp64.  The bound assumes that the tensor-core accumulator loses at most 2^-23 of the running
- * sum per accumulated element; the parity tests check the measured error against it.  Other
- * cases, and WIDE_FLAG_SIMT, compute all scores in fp64.)
+ * sum per accumulated element; the parity tests check the measured error against it.  With at
+ * most WIDE_DECODE_MAX_TOKENS tokens the same is done in one launch on the CUDA cores, fp32 sums
+ * of hidden / 32-long chains with the same kind of bound; WIDE_FLAG_FORCE_PREFILL takes the
+ * tensor-core form there too.  Other cases, and WIDE_FLAG_SIMT, compute all scores in fp64.)
  *   x          [tokens, hidden]  dtype
  *   mask_bits  out uint32 [tokens, W]
  *   scores     out fp32 [tokens, n_groups] (TOPK) or [tokens, 2*n_groups] (PAIR), may be NULL

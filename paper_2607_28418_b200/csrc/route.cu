@@ -159,6 +159,49 @@ __device__ __forceinline__ double warp_dot_f64(const __nv_bfloat16* __restrict__
     return r;
 }
 
+// The same for two weight rows at once: x is read once and the two chains of fp64 multiply-adds (the
+// slow part: this GPU issues about two of them per clock and SM) run side by side.
+__device__ __forceinline__ void warp_dot_f64_x2(const __nv_bfloat16* __restrict__ xrow, const __nv_bfloat16* __restrict__ wrow0,
+                                                const __nv_bfloat16* __restrict__ wrow1, int nch, int lane, double& r0, double& r1) {
+    constexpr int kB = 4;
+    const uint4* xv = reinterpret_cast<const uint4*>(xrow);
+    const uint4* wv0 = reinterpret_cast<const uint4*>(wrow0);
+    const uint4* wv1 = reinterpret_cast<const uint4*>(wrow1);
+    double a0[4] = {0.0, 0.0, 0.0, 0.0}, a1[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int base = 0; base < nch; base += 32 * kB) {
+        uint4 a[kB], b0[kB], b1[kB];
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {
+            const int i = base + lane + 32 * j;
+            a[j] = i < nch ? __ldg(xv + i) : make_uint4(0u, 0u, 0u, 0u);
+            b0[j] = i < nch ? __ldg(wv0 + i) : make_uint4(0u, 0u, 0u, 0u);
+            b1[j] = i < nch ? __ldg(wv1 + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {
+            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a[j]);
+            const __nv_bfloat162* bh0 = reinterpret_cast<const __nv_bfloat162*>(&b0[j]);
+            const __nv_bfloat162* bh1 = reinterpret_cast<const __nv_bfloat162*>(&b1[j]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 fa = __bfloat1622float2(ah[e]), f0 = __bfloat1622float2(bh0[e]), f1 = __bfloat1622float2(bh1[e]);
+                const double xa = static_cast<double>(fa.x), xb = static_cast<double>(fa.y);
+                a0[e] = fma(xa, static_cast<double>(f0.x), a0[e]);
+                a0[e] = fma(xb, static_cast<double>(f0.y), a0[e]);
+                a1[e] = fma(xa, static_cast<double>(f1.x), a1[e]);
+                a1[e] = fma(xb, static_cast<double>(f1.y), a1[e]);
+            }
+        }
+    }
+    r0 = (a0[0] + a0[1]) + (a0[2] + a0[3]);
+    r1 = (a1[0] + a1[1]) + (a1[2] + a1[3]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        r0 += __shfl_xor_sync(0xffffffffu, r0, o);
+        r1 += __shfl_xor_sync(0xffffffffu, r1, o);
+    }
+}
+
 // Two warps per token, two tokens per CTA.  What bounds this kernel is the length of one warp's
 // chain of dependent instructions and load round trips, not throughput, so the two independent
 // halves of the work run side by side: the SELECT warp sums the score slabs and finds the kt-th
@@ -378,6 +421,309 @@ void launch_select_band(cudaStream_t s, int T, const float* sc32, int ksplit, in
                         uint32_t* mask_bits, float* scores, int chain) {
     select_band_kernel<KPL><<<(T + kSelTokens - 1) / kSelTokens, 64 * kSelTokens, 0, s>>>(
         sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores, chain);
+}
+
+// ---------------------------------------------------------------------------- small batches (decode), top-k
+// One launch for at most kRsMaxTokens tokens.  A CTA takes eight tokens, eight groups and one of KS
+// slices of the hidden dimension: the tokens' slices of x sit in shared memory, a warp streams its
+// slice of one row of the router weight once (one round trip) and forms fp32 partial scores against all
+// eight tokens on the CUDA cores (a lane accumulates every 32nd 16-byte piece, the lanes' sums are added
+// by shuffles), with its part of ||w_g||^2 and ||x_t||^2 on the side.  Partial scores and norms go to
+// the scratch; the CTA that arrives last for a tile of tokens (a ticket per tile, put back to zero by
+// that CTA) selects: one warp per token adds the KS partials in a fixed order and then runs the same
+// bitwise search for the k-th largest score, the same band of half-width 2 * eps_t around the boundary
+// and the same exact fp64 re-scoring of the band's members as select_band_kernel, here with
+//   eps_t = 1.01 * 2^-24 * (D / (32 KS) + 5 + KS) * ||x_t|| * max_g ||w_g||:
+// every score is the end of a chain of at most D / (32 KS) fused multiply-adds in a lane, five shuffle
+// additions and KS - 1 additions of the partials, each an IEEE operation rounded to nearest (relative
+// error 2^-24, unlike the tensor core's unspecified accumulator), so its error is at most
+// gamma_n * sum |x_i w_i| with n the chain length, and the sum is at most ||x|| ||w|| (Cauchy-Schwarz);
+// the factor 1.01 covers the second-order terms of gamma_n.  The norms of the weight rows are the same for every
+// tile of tokens: every tile writes them, with the same bits, to the same place.
+constexpr int kRsTokens = 8;
+constexpr int kRsGroups = 8;
+constexpr int kRsMaxTokens = 64;
+
+// scratch of the one-launch router, in floats: partial scores [KS][T][NG], partial ||w||^2 [KS][NG],
+// partial ||x||^2 [T][KS]
+__host__ __device__ inline size_t route_small_floats(int T, int NG, int KS) {
+    return static_cast<size_t>(KS) * (static_cast<size_t>(T) * NG + NG + T);
+}
+
+template <int KPL>
+__global__ void __launch_bounds__(32 * kRsGroups)
+route_small_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w, int T, int NG, int D, int k,
+                   const int32_t* __restrict__ k_per_token, uint32_t* __restrict__ mask_bits, float* __restrict__ scores_out,
+                   float* __restrict__ scratch, int KS, int ppq, unsigned* __restrict__ tickets) {
+    extern __shared__ uint4 rs_smem[];   // x slices of the tile's tokens, bf16 [kRsTokens][ppq pieces]
+    __shared__ int s_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nch = D / 8;
+    const int chunk = blockIdx.x / KS, kq = blockIdx.x - chunk * KS;
+    const int q_lo = min(nch, kq * ppq), q_hi = min(nch, q_lo + ppq);   // this slice's pieces of a row
+    const int t0 = blockIdx.y * kRsTokens;
+    const int nt = min(kRsTokens, T - t0);
+    float* slab = scratch;                                          // [KS][T][NG]
+    float* wsq_part = scratch + static_cast<size_t>(KS) * T * NG;   // [KS][NG]
+    float* xsq_part = wsq_part + static_cast<size_t>(KS) * NG;      // [T][KS]
+    const uint4* x4 = reinterpret_cast<const uint4*>(x);
+    for (int tt = warp; tt < kRsTokens; tt += kRsGroups) {
+        for (int p = lane; p < ppq; p += 32)
+            rs_smem[tt * ppq + p] = (tt < nt && q_lo + p < q_hi) ? __ldg(x4 + static_cast<size_t>(t0 + tt) * nch + q_lo + p)
+                                                                 : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncthreads();
+
+    // ---- partial scores of this warp's group against the tile's tokens
+    const int g = chunk * kRsGroups + warp;
+    if (g < NG) {
+        const uint4* w4 = reinterpret_cast<const uint4*>(w + static_cast<size_t>(g) * D) + q_lo;
+        float acc[kRsTokens];
+#pragma unroll
+        for (int tt = 0; tt < kRsTokens; ++tt) acc[tt] = 0.f;
+        float wsq = 0.f;
+        for (int base = 0; base < q_hi - q_lo; base += 32 * kBatch) {
+            uint4 wv[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int i = base + lane + 32 * j;
+                wv[j] = i < q_hi - q_lo ? __ldg(w4 + i) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int i = base + lane + 32 * j;
+                if (i < q_hi - q_lo) {
+                    const uint32_t ww[4] = {wv[j].x, wv[j].y, wv[j].z, wv[j].w};
+                    float wf[8];
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        wf[2 * p] = __uint_as_float(ww[p] << 16);
+                        wf[2 * p + 1] = __uint_as_float(ww[p] & 0xffff0000u);
+                        wsq = fmaf(wf[2 * p], wf[2 * p], fmaf(wf[2 * p + 1], wf[2 * p + 1], wsq));
+                    }
+#pragma unroll
+                    for (int tt = 0; tt < kRsTokens; ++tt) {
+                        if (tt < nt) {
+                            const uint4 xv = rs_smem[tt * ppq + i];
+                            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                            for (int p = 0; p < 4; ++p) {
+                                acc[tt] = fmaf(wf[2 * p], __uint_as_float(xw[p] << 16), acc[tt]);
+                                acc[tt] = fmaf(wf[2 * p + 1], __uint_as_float(xw[p] & 0xffff0000u), acc[tt]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wsq += __shfl_xor_sync(0xffffffffu, wsq, o);
+#pragma unroll
+        for (int tt = 0; tt < kRsTokens; ++tt) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[tt] += __shfl_xor_sync(0xffffffffu, acc[tt], o);
+            if (lane == tt && tt < nt) slab[(static_cast<size_t>(kq) * T + t0 + tt) * NG + g] = acc[tt];
+        }
+        if (lane == 0) wsq_part[kq * NG + g] = wsq;   // the same bits from every tile of tokens
+    }
+    if (chunk == 0 && warp < nt) {
+        // this slice's part of ||x_t||^2, token t0 + warp
+        float xsq = 0.f;
+        for (int p = lane; p < ppq; p += 32) {
+            const uint4 xv = rs_smem[warp * ppq + p];
+            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float a = __uint_as_float(xw[q] << 16), b = __uint_as_float(xw[q] & 0xffff0000u);
+                xsq = fmaf(a, a, fmaf(b, b, xsq));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) xsq += __shfl_xor_sync(0xffffffffu, xsq, o);
+        if (lane == 0) xsq_part[(t0 + warp) * KS + kq] = xsq;
+    }
+
+    // ---- the CTA that completes the tile's scores selects
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned old = atomicAdd(tickets + blockIdx.y, 1u);
+        s_last = old + 1u == gridDim.x ? 1 : 0;
+        if (s_last) tickets[blockIdx.y] = 0u;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    const int t = t0 + warp;
+    if (warp >= nt) return;
+    const int words = (NG + 31) >> 5;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const int kt = min(max(k_per_token ? k_per_token[t] : k, 0), NG);
+    const bool boundary = kt > 0 && kt < NG;
+    // (the partials are read with loops of fixed length, so that all loads are on their way before the first sum)
+    float xsq = 0.f;
+    {
+        float part[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) part[q] = q < KS ? __ldcg(xsq_part + t * KS + q) : 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) xsq += part[q];
+    }
+
+    float sv[KPL];
+    uint32_t key[KPL];   // 0 for slots past NG, >= 1 for real groups
+    bool sel[KPL], in_band[KPL];
+    float wmax = 0.f, v_k = 0.f, v_k1 = 0.f;
+    float sp[KPL][4], wp[KPL][4];
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+        const int gg = 32 * j + lane;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const bool live = gg < NG && q < KS;
+            sp[j][q] = live ? __ldcg(slab + (static_cast<size_t>(q) * T + t) * NG + gg) : 0.f;
+            wp[j][q] = live ? __ldcg(wsq_part + q * NG + gg) : 0.f;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+        const int gg = 32 * j + lane;
+        float v = 0.f, wn = 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {   // slices beyond KS add an exact zero
+            v += sp[j][q];
+            wn += wp[j][q];
+        }
+        v += 0.0f;  // -0 -> +0
+        sv[j] = v;
+        const uint32_t u = __float_as_uint(v);
+        const uint32_t ord = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+        key[j] = gg < NG ? max(ord, 1u) : 0u;
+        wmax = fmaxf(wmax, wn);
+        sel[j] = kt == NG && gg < NG;
+        in_band[j] = false;
+        if (scores_out && gg < NG) scores_out[static_cast<size_t>(t) * NG + gg] = v;
+    }
+    int nb = 0, m_hi = 0;
+    if (boundary) {
+        wmax = sqrtf(__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(wmax)))) * 1.0001f;  // norms are >= 0
+        // kt-th largest key, two bits per step: the three candidates of a step are counted side by side, so
+        // the chain of dependent steps is half as long as a bit-by-bit search's
+        uint32_t key_k = 0u;
+#pragma unroll 4
+        for (int bit = 30; bit >= 0; bit -= 2) {
+            const uint32_t c1 = key_k | (1u << bit), c2 = key_k | (2u << bit), c3 = key_k | (3u << bit);
+            int n1 = 0, n2 = 0, n3 = 0;
+#pragma unroll
+            for (int j = 0; j < KPL; ++j) {
+                n1 += __popc(__ballot_sync(0xffffffffu, key[j] >= c1));
+                n2 += __popc(__ballot_sync(0xffffffffu, key[j] >= c2));
+                n3 += __popc(__ballot_sync(0xffffffffu, key[j] >= c3));
+            }
+            key_k = n3 >= kt ? c3 : (n2 >= kt ? c2 : (n1 >= kt ? c1 : key_k));
+        }
+        int n_gt = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, key[j] > key_k));
+        const int need = kt - n_gt;   // how many of the groups tied at key_k are taken (>= 1)
+        int n_tie = 0;
+        uint32_t below = 0u;          // largest key under key_k
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            const bool tie = key[j] == key_k;
+            const uint32_t b = __ballot_sync(0xffffffffu, tie);
+            sel[j] = key[j] > key_k || (tie && n_tie + __popc(b & lt_mask) < need);
+            n_tie += __popc(b);
+            if (key[j] < key_k) below = max(below, key[j]);
+        }
+        below = __reduce_max_sync(0xffffffffu, below);
+        v_k = __uint_as_float((key_k & 0x80000000u) ? (key_k & 0x7fffffffu) : ~key_k);
+        v_k1 = n_tie > need ? v_k : __uint_as_float((below & 0x80000000u) ? (below & 0x7fffffffu) : ~below);
+        // band half-width 2 * eps_t (a little slack for the fp32 evaluation of the bound itself)
+        // ppq / 4 >= D / (32 KS) multiply-adds per lane; 1.001: the bound itself is evaluated in fp32 from
+        // norms that were summed in fp32
+        const float tau = 2.f * 1.01f * 5.9604645e-8f * static_cast<float>(ppq / 4 + 5 + KS) * sqrtf(xsq) * 1.001f * wmax;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            const bool valid = key[j] != 0u;
+            in_band[j] = valid && (sel[j] ? (sv[j] - v_k1 <= tau) : (v_k - sv[j] <= tau));
+            nb += __popc(__ballot_sync(0xffffffffu, in_band[j]));
+            m_hi += __popc(__ballot_sync(0xffffffffu, in_band[j] && sel[j]));
+        }
+    }
+    if (nb > 0) {   // then the band holds at least the two groups on either side of the boundary
+        // exact scores of the band's members, two at a time (the same value whichever way a member is paired:
+        // each dot product has its own accumulators and the same order of operations)
+        double ex[KPL];
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) ex[j] = 0.0;
+        const __nv_bfloat16* xrow = x + static_cast<size_t>(t) * D;
+        int pend = -1;   // a member waiting for a partner
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            uint32_t bits = __ballot_sync(0xffffffffu, in_band[j]);
+            while (bits) {
+                const int h = 32 * j + __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (pend < 0) {
+                    pend = h;
+                    continue;
+                }
+                double e0, e1;
+                warp_dot_f64_x2(xrow, w + static_cast<size_t>(pend) * D, w + static_cast<size_t>(h) * D, nch, lane, e0, e1);
+#pragma unroll
+                for (int jj = 0; jj < KPL; ++jj) {
+                    if (32 * jj + lane == pend) ex[jj] = e0;
+                    if (32 * jj + lane == h) ex[jj] = e1;
+                }
+                pend = -1;
+            }
+        }
+        if (pend >= 0) {
+            const double e = warp_dot_f64(xrow, w + static_cast<size_t>(pend) * D, nch, lane);
+#pragma unroll
+            for (int jj = 0; jj < KPL; ++jj)
+                if (32 * jj + lane == pend) ex[jj] = e;
+        }
+        // band members are re-ranked among themselves on the exact scores
+        int beats[KPL];
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) beats[j] = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {
+            uint32_t bits = __ballot_sync(0xffffffffu, in_band[j]);
+            while (bits) {
+                const int l = __ffs(bits) - 1;
+                bits &= bits - 1;
+                const double u = __shfl_sync(0xffffffffu, ex[j], l);
+                const int h = 32 * j + l;
+#pragma unroll
+                for (int jj = 0; jj < KPL; ++jj) beats[jj] += (u > ex[jj]) || (u == ex[jj] && h < 32 * jj + lane);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < KPL; ++j)
+            if (in_band[j]) sel[j] = beats[j] < m_hi;
+    }
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+        const uint32_t word = __ballot_sync(0xffffffffu, sel[j]);
+        if (lane == 0 && j < words) mask_bits[static_cast<size_t>(t) * words + j] = word;
+    }
+}
+
+template <int KPL>
+int launch_route_small(cudaStream_t s, int T, const __nv_bfloat16* x, const __nv_bfloat16* w, int NG, int D, int k,
+                       const int32_t* k_per_token, uint32_t* mask_bits, float* scores, float* scratch, int KS,
+                       unsigned* tickets) {
+    const int ppq = ((D / 8 + KS - 1) / KS + 31) / 32 * 32;   // 16-byte pieces of a row per slice
+    const int smem = kRsTokens * ppq * 16;
+    if (cudaFuncSetAttribute(route_small_kernel<KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return WIDE_ERR_CUDA;
+    route_small_kernel<KPL><<<dim3((NG + kRsGroups - 1) / kRsGroups * KS, (T + kRsTokens - 1) / kRsTokens), 32 * kRsGroups, smem, s>>>(
+        x, w, T, NG, D, k, k_per_token, mask_bits, scores, scratch, KS, ppq, tickets);
+    return cudaGetLastError() == cudaSuccess ? WIDE_OK : WIDE_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------- fast pair-argmax path (bf16)
@@ -731,6 +1077,25 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
         !(flags & WIDE_FLAG_SIMT)) {
         const int ld = (NG + 31) / 32 * 32;
         float* sc32 = static_cast<float*>(ws);
+        // decode batches: scores and selection in one launch on the CUDA cores, the hidden dimension cut into as
+        // many slices (4, 2 or 1) as the scratch holds partial scores for
+        int KS = 4;
+        while (KS > 1 && route_small_floats(T, NG, KS) * sizeof(float) > wide_route_workspace(T, NG, rank) - 1024) KS >>= 1;
+        if (T <= kRsMaxTokens && !(flags & WIDE_FLAG_FORCE_PREFILL) &&
+            route_small_floats(T, NG, KS) * sizeof(float) <= wide_route_workspace(T, NG, rank) - 1024 &&
+            kRsTokens * ((D / 8 + KS - 1) / KS + 31) * 16 <= 200 * 1024) {
+            WideLaunch l(ctx, s, "route_small");
+            const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+            const __nv_bfloat16* wb = static_cast<const __nv_bfloat16*>(w_router);
+            switch ((NG + 31) / 32) {
+#define WIDE_RS_CASE(n) \
+    case n: return launch_route_small<n>(s, T, xb, wb, NG, D, k, k_per_token, mask_bits, scores, sc32, KS, ctx->d_tickets);
+                WIDE_RS_CASE(1) WIDE_RS_CASE(2) WIDE_RS_CASE(3) WIDE_RS_CASE(4)
+                WIDE_RS_CASE(5) WIDE_RS_CASE(6) WIDE_RS_CASE(7) WIDE_RS_CASE(8)
+#undef WIDE_RS_CASE
+                default: return WIDE_ERR_UNSUPPORTED_SHAPE;
+            }
+        }
         float* wn = reinterpret_cast<float*>(static_cast<char*>(ws) + wide_route_workspace(T, NG, rank) - 1024);
         // as many K-split slabs as the first part of the workspace holds (at most 8)
         const size_t part0 = wide_route_workspace(T, NG, rank) - 1024;
