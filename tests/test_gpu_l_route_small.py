@@ -93,3 +93,26 @@ def test_route_small_repeated_calls_of_different_sizes(ctx):
     for T in (64, 1, 64, 3, 17, 17, 1, 64):
         x = synth.make_activations(rng, T, D, "bf16", "random")
         _check(ctx, x, wr, k, both=False)
+
+
+@pytest.mark.parametrize("T", [3, 40])
+def test_route_small_band_rescoring_with_a_wide_range_of_magnitudes(ctx, T):
+    """Rows that tie exactly or differ by one ulp put most groups in the band, whose members are re-scored
+    exactly; a few elements of x and of the weights are tiny (2^-100, 2^-60) or large (2^20), so that the
+    products of one row span a hundred binary orders of magnitude.  The decision must stay the oracle's."""
+    D, NG, k = 1024, 64, 32
+    rng = np.random.default_rng(77 + T)
+    x = synth.round_to_bf16(rng.standard_normal((T, D)).astype(np.float32))
+    base = synth.round_to_bf16((rng.standard_normal((1, D)) / np.sqrt(D)).astype(np.float32))
+    wr = np.repeat(base, NG, axis=0)
+    for g in range(0, NG, 3):
+        i = int(rng.integers(0, D))
+        wr[g, i] = synth.round_to_bf16(np.array([wr[g, i] * (1 + 2.0 ** -7)], dtype=np.float32))[0]
+    wr[5, 7] = np.float32(2.0 ** -60)
+    wr[6, 9] = np.float32(2.0 ** -100)
+    for t in range(T):
+        if t % 3 == 1:
+            x[t, t % D] = np.float32(2.0 ** -100)
+        if t % 3 == 2:
+            x[t, (5 * t) % D] = np.float32(2.0 ** 20)
+    _check(ctx, synth.round_to_bf16(x), synth.round_to_bf16(wr), k)
