@@ -22,7 +22,8 @@ struct wide_ctx {
                             // 256-row down projection (16 ints in all)
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
-    unsigned* d_tickets;    // 2048 completion counters of the decode path; zero between calls
+    unsigned* d_tickets;    // 2048 completion counters, zero between calls: [0, 1024) and [1024, 1152) the decode FFN /
+                            // O-projection kernel, [2040, 2048) the token tiles of the one-launch router
     float* attn_part;       // partial (m, l, O) of the key slices of the decode attention
     size_t attn_part_bytes;
     unsigned long long wait_ns;  // bound of every device-side wait

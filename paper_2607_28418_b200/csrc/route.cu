@@ -207,8 +207,8 @@ __device__ __forceinline__ void warp_dot_f64_x2(const __nv_bfloat16* __restrict_
 // halves of the work run side by side: the SELECT warp sums the score slabs and finds the kt-th
 // largest, the NORM warp reads the x row for ||x_t||.  Lane l of the select warp holds the groups
 // g = 32*j + l, j < KPL, which is also the layout of the packed mask words.  Scores map to
-// unsigned keys that order like the floats; the kt-th largest key is found by a 32-step binary
-// search on its bits with warp votes (no quadratic rank count), ties at that key go to the lower
+// unsigned keys that order like the floats; the kt-th largest key is found by a 16-step search on
+// its bits, two at a time, with warp votes (no quadratic rank count), ties at that key go to the lower
 // group index.  Band members (rare) are re-scored by all four warps of the CTA.
 template <int KPL>
 __global__ void __launch_bounds__(64 * kSelTokens, 8)   // every CTA of a 2048-token batch resident at once
@@ -296,15 +296,20 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
         }
         if (boundary) {
             wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(wmax)));  // norms are >= 0
-            // kt-th largest key
+            // kt-th largest key, two bits per step: the three candidates of a step are counted side by side,
+            // so the chain of dependent steps is half as long as a bit-by-bit search's
             uint32_t key_k = 0u;
-#pragma unroll 8
-            for (int bit = 31; bit >= 0; --bit) {
-                const uint32_t cand = key_k | (1u << bit);
-                int c = 0;
+#pragma unroll 4
+            for (int bit = 30; bit >= 0; bit -= 2) {
+                const uint32_t c1 = key_k | (1u << bit), c2 = key_k | (2u << bit), c3 = key_k | (3u << bit);
+                int n1 = 0, n2 = 0, n3 = 0;
 #pragma unroll
-                for (int j = 0; j < KPL; ++j) c += __popc(__ballot_sync(0xffffffffu, key[j] >= cand));
-                if (c >= kt) key_k = cand;
+                for (int j = 0; j < KPL; ++j) {
+                    n1 += __popc(__ballot_sync(0xffffffffu, key[j] >= c1));
+                    n2 += __popc(__ballot_sync(0xffffffffu, key[j] >= c2));
+                    n3 += __popc(__ballot_sync(0xffffffffu, key[j] >= c3));
+                }
+                key_k = n3 >= kt ? c3 : (n2 >= kt ? c2 : (n1 >= kt ? c1 : key_k));
             }
             int n_gt = 0;
 #pragma unroll
@@ -1089,7 +1094,7 @@ int wide_launch_route(wide_ctx* ctx, cudaStream_t s, const void* x, int dtype, i
             const __nv_bfloat16* wb = static_cast<const __nv_bfloat16*>(w_router);
             switch ((NG + 31) / 32) {
 #define WIDE_RS_CASE(n) \
-    case n: return launch_route_small<n>(s, T, xb, wb, NG, D, k, k_per_token, mask_bits, scores, sc32, KS, ctx->d_tickets);
+    case n: return launch_route_small<n>(s, T, xb, wb, NG, D, k, k_per_token, mask_bits, scores, sc32, KS, ctx->d_tickets + 2040);
                 WIDE_RS_CASE(1) WIDE_RS_CASE(2) WIDE_RS_CASE(3) WIDE_RS_CASE(4)
                 WIDE_RS_CASE(5) WIDE_RS_CASE(6) WIDE_RS_CASE(7) WIDE_RS_CASE(8)
 #undef WIDE_RS_CASE
