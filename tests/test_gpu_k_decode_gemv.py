@@ -54,13 +54,13 @@ def test_ffn_gemv_and_tensor_core_kernel_match_the_oracle(ctx, B, G, out):
         assert_close(y, ref, f"{name} B{B} G{G} out {out}")
 
 
-@pytest.mark.parametrize("D,Dff,G", [(320, 1280, 64), (576, 2304, 128), (4096, 14336, 128)])
+@pytest.mark.parametrize("D,Dff,G", [(320, 1280, 64), (576, 2304, 128), (4096, 14336, 128), (5120, 13824, 128)])
 def test_ffn_gemv_rows_that_are_not_whole_sweeps(ctx, D, Dff, G):
     """hidden / 8 = 40 or 72 pieces per row (not a multiple of the 32 lanes, nor of a 128-piece batch),
-    unions whose W_down pieces do not fill the last batch; and the full Llama-3-8B shape."""
+    unions whose W_down pieces do not fill the last batch; and the full Llama-3-8B and Llama-2-13B shapes."""
     from paper_2607_28418_b200 import binding
     for B in (1, 2):
-        mask = synth.random_mask(7 * B + D, B, Dff // G, 3 if D < 4096 else 56)
+        mask = synth.random_mask(7 * B + D, B, Dff // G, 3 if D < 4096 else Dff // G // 2)
         y, ref = _ffn(ctx, B, D, Dff, G, mask, binding.FLAG_NONE, seed=D + B)
         assert_close(y, ref, f"B{B} D{D} Dff{Dff} G{G}")
 
