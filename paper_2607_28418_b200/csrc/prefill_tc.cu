@@ -103,8 +103,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // over the pruned dimension): this rank's tile is a PART of y (Eq. 10 summed over this rank's groups
 // only), and the sum over ranks is a reduce-scatter over token rows.  Fused here: instead of storing
 // its part and handing it to a collective, the epilogue adds every row straight into the fp32 shard
-// of the rank that owns the row, with red.global.add over peer memory (plain peer stores through
-// NVLink; no multicast, no TMA).  base[r] = rank r's shard [rows_per_rank, N] fp32, zero before any
+// of the rank that owns the row, with red.global.add over peer memory (plain peer accesses through
+// NVLink issued by the epilogue threads; no bulk or tensor copy touches another GPU's memory).  base[r] = rank r's shard [rows_per_rank, N] fp32, zero before any
 // rank starts and complete once every rank's kernel has finished (the caller's two barriers).
 // world == 0: ordinary output.
 struct PeerOut {
