@@ -57,10 +57,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // abort in *abort_flag); the caller must then leave its loop and go to the kernel's teardown.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns,
                                           volatile int* abort_flag) {
+    // The polling loops stay loops: unrolled, every wait in a kernel is kilobytes of code, and the
+    // threads that spin in them run through it again and again, which pushes the code that does the
+    // work out of the SM's instruction cache.
+#pragma unroll 1
     for (int i = 0; i < 128; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     const uint64_t start = globaltimer_ns();
     while (true) {
+#pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
