@@ -19,7 +19,8 @@ struct wide_ctx {
     int sm_count;
     int* d_status;          // [0] device status word (WIDE_OK or WIDE_ERR_TIMEOUT), [1] reorder ticket,
                             // [4..5] grid-barrier counters of the decode kernels, [6] channel pool of the GEMV decode kernel, [8..9] tile queue of the
-                            // 256-row down projection (16 ints in all)
+                            // 256-row down projection, [10..11] work list of the attention prefill kernel (next item, CTAs done;
+                            // zero between launches) (16 ints in all)
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
     unsigned* d_tickets;    // 2048 completion counters, zero between calls: [0, 1024) and [1024, 1152) the decode FFN /

@@ -73,6 +73,56 @@ def test_attn_one_group_active_per_token_and_custom_scale(ctx):
     assert_close(got, ref, "attn, custom scale")
 
 
+def test_attn_more_items_than_sms_with_uneven_groups(ctx):
+    """The prefill kernel runs one CTA per SM and hands (head, query tile) items out at run time.  Here
+    about 200 items of 1 to 20 key tiles go over the CTAs: three groups with every token, two with
+    half, one with 90 %, one with 37 tokens, one with none (no item at all, rows of exact zeros)."""
+    t, h_q, h_kv, d, hpg = 2560, 16, 4, 128, 2
+    case = synth.make_attn_case(21, t, t, h_q, h_kv, d)
+    rng = np.random.default_rng(22)
+    mask = np.zeros((t, h_q // hpg), dtype=bool)
+    mask[:, [0, 3, 5]] = True
+    mask[:, 1] = rng.random(t) < 0.5
+    mask[:, 6] = rng.random(t) < 0.5
+    mask[rng.choice(t, 37, replace=False), 2] = True
+    mask[:, 7] = rng.random(t) < 0.9
+    got = _run(ctx, case, mask, h_q, h_kv, d, hpg)
+    ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg)
+    head_mask = np.repeat(mask, hpg, axis=1)
+    assert (got.float().cpu().numpy()[~head_mask] == 0.0).all()
+    assert_close(got, ref, "attn, more items than SMs")
+
+
+def test_attn_queries_ahead_of_the_keys(ctx):
+    """T_k < T_q with the causal limit j <= t + T_k - T_q: the first queries see no key at all (exact
+    zero rows, whole query tiles without a key tile), the next ones a single, partly visible key tile."""
+    t_q, t_k, h_q, h_kv, d, hpg = 600, 200, 4, 2, 128, 2
+    case = synth.make_attn_case(23, t_q, t_k, h_q, h_kv, d)
+    for mask in (synth.bernoulli_mask(24, t_q, h_q // hpg, 0.5), np.ones((t_q, h_q // hpg), dtype=bool)):
+        got = _run(ctx, case, mask, h_q, h_kv, d, hpg)
+        ref = wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg)
+        assert (got[: t_q - t_k] == 0.0).all().item()
+        assert_close(got, ref, "attn, T_k < T_q")
+
+
+def test_attn_repeated_and_interleaved_calls_repeat_bit_for_bit(ctx):
+    """The work list's counter is shared state that every launch must leave at zero, whatever the shapes
+    of the calls before; which CTA takes which item may differ from run to run, the bits may not."""
+    shapes = [(300, 300, 8, 2, 128, 4), (1536, 1536, 16, 16, 128, 4), (517, 517, 4, 4, 64, 1)]
+    first = {}
+    for rep in range(3):
+        for sh in shapes:
+            t_q, t_k, h_q, h_kv, d, hpg = sh
+            case = synth.make_attn_case(31, t_q, t_k, h_q, h_kv, d)
+            mask = synth.bernoulli_mask(32, t_q, h_q // hpg, 0.6)
+            got = _run(ctx, case, mask, h_q, h_kv, d, hpg)
+            if sh in first:
+                assert torch.equal(first[sh], got), f"{sh}: call {rep} differs from the first"
+            else:
+                first[sh] = got.clone()
+                assert_close(got, wo.masked_attention(case["q"], case["k"], case["v"], mask, hpg), f"attn {sh}")
+
+
 def test_attn_rejects_bad_arguments(ctx):
     from paper_2607_28418_b200 import binding
     q = torch.zeros((128, 4 * 96), dtype=torch.bfloat16, device="cuda")
