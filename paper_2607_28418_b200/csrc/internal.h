@@ -19,7 +19,7 @@ struct wide_ctx {
     int sm_count;
     int* d_status;          // [0] device status word (WIDE_OK or WIDE_ERR_TIMEOUT), [1] reorder ticket,
                             // [4..5] grid-barrier counters of the decode kernels, [6] channel pool of the GEMV decode kernel, [8..9] tile queue of the
-                            // 256-row down projection, [10..11] work list of the attention prefill kernel (next item, CTAs done;
+                            // 256-row down projection, [10..12] work list of the attention prefill kernel (next item, CTAs done, next block of rows to zero;
                             // zero between launches) (16 ints in all)
     float* decode_acc;      // fp32 accumulators of the decode path; zero between calls
     size_t decode_acc_floats;
