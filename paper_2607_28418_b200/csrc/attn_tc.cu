@@ -173,7 +173,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
     constexpr int kHalfKV = kKV / 2;       // keys of a tile each softmax group takes
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const size_t ldq = static_cast<size_t>(Hq) * HD;
-    const int n_mt = (Tq + kQ - 1) / kQ;
     const int delta = Tk - Tq;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -554,7 +553,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
             // accumulators hold row r in tensor-memory lane r, so a thread reads its row of either one:
             // each group finishes half of the output columns from O[0] and O[1] directly, and only
             // (m, l) go through shared memory.
-            const bool mine = NT > 0, theirs = NT > 0;
+            const bool any = NT > 0;   // an item without a visible key: both accumulators are stale
             if (ok && NT > 0) ok = mbar_wait_warp(pv_full + 8 * ((cnt - 1) & 1), ((cnt - 1) >> 1) & 1, wait_ns, abort_flag);   // the last PV
             // the other group has read this group's (m, l) of the previous item
             if (ok && il > 0) ok = mbar_wait_warp(x_done + 8 * b, (il - 1) & 1, wait_ns, abort_flag);
@@ -580,11 +579,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
                     tmem_ld_32x32(o_addr + keep_c + c0, w0);
                     tmem_ld_32x32(lane_addr + 256 + (1 - b) * HD + keep_c + c0, w1);
                     tmem_ld_wait();
-                    // a group without a key tile in this item: its accumulator is stale (any bits), not zero
+                    // an item without a visible key issued no PV: the accumulators hold stale bits, not zeros
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        w0[i] = mine ? w0[i] : 0u;
-                        w1[i] = theirs ? w1[i] : 0u;
+                        w0[i] = any ? w0[i] : 0u;
+                        w1[i] = any ? w1[i] : 0u;
                     }
                     if (ok && r < n_valid) {
 #pragma unroll
@@ -621,9 +620,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUt
                 if (c >= n_blocks) break;
                 const int g = c % n_groups, first = min(counts[g], Tq) + (c / n_groups) * 32;
                 if (first >= Tq) continue;
-                const int mine = first + lane < Tq ? perm[static_cast<size_t>(g) * Tq + first + lane] : -1;
+                const int my_row = first + lane < Tq ? perm[static_cast<size_t>(g) * Tq + first + lane] : -1;
                 for (int u = 0; u < 32; ++u) {
-                    const int row = __shfl_sync(0xffffffffu, mine, u);
+                    const int row = __shfl_sync(0xffffffffu, my_row, u);
                     if (row < 0) break;
                     uint4* dst = reinterpret_cast<uint4*>(o + row * ldq + static_cast<size_t>(g) * hpg * HD);
                     for (int pc = lane; pc < pieces; pc += 32) dst[pc] = make_uint4(0u, 0u, 0u, 0u);
