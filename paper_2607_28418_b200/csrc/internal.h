@@ -35,6 +35,24 @@ struct wide_ctx {
     int prof_cap, prof_used;
 };
 
+// Launch with the programmatic-serialization attribute: the kernel may start its set-up while the kernel before
+// it in the stream finishes; it calls grid_dep_wait() before it touches global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t wide_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                         Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Counts one kernel launch and, when profiling is on, brackets it with a pair of CUDA events on
 // the launching stream.  Usage: { WideLaunch l(ctx, s, "name"); kernel<<<..., s>>>(...); }
 struct WideLaunch {

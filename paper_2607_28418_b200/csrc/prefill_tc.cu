@@ -415,6 +415,10 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // When this kernel is launched as a programmatic dependent of the gate / up kernel (launch_down_auto), it may
+    // run up to here, and on through its tile masks (mask and token order are older than the gate / up kernel, which
+    // is launched the ordinary way), while that kernel's last CTAs finish; grid_dep_wait() stands before the first load
+    // of H and before the first store to Y.
 
     const int n_m = (T + 255) / 256;
     const int n_tiles = n_m * n_n;
@@ -471,6 +475,7 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t act[kMaskWords];
             tile_mask(m, act);
             if (lane == 0) {
+                if (tc == 0) grid_dep_wait();     // H comes from the kernel before
                 for (int g = 0; g < NG && ok; ++g) {
                     if (!((act[g >> 5] >> (g & 31)) & 1u)) continue;
                     for (int kk = 0; kk < ksub; ++kk, ++it) {
@@ -552,6 +557,8 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int g = 0; g < NG; ++g) any = any || ((act[g >> 5] >> (g & 31)) & 1u);
             if (!mbar_wait_warp(tfull, tc & 1, wait_ns, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
+            if (tc == 0) grid_dep_wait();         // nothing is stored before the kernel before has completed (a tile without
+                                                  // an active group gets here without a load behind it)
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
                 const int pos = m * 256 + half * 128 + q * 32 + lane;
@@ -741,6 +748,7 @@ gateup_kernel(const __grid_constant__ CUtensorMap tmG, const __grid_constant__ C
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
     }
+    grid_dep_launch();   // the down projection behind this kernel may set itself up on SMs that this kernel has left
     if (warp == 2) {
         // prefix sums of doubles and odd tiles per (group, sub-block)
         int dsum = 0, ssum = 0;
@@ -1064,7 +1072,8 @@ double pick_down256_tiling(int sm, int T, int N, int* n_n_out, int* wmax_out) {
 // (about 0.8 of the time per row), 128-row tiles quantise better over the SMs.
 int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B, const uint32_t* mask_bits, int T,
                      int N, int K, int G, void* Y, int out_dtype, const int32_t* order,
-                     const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, const PeerOut* peer = nullptr) {
+                     const int32_t* sel_counts = nullptr, int sel_thr = WIDE_KAXIS_NEVER, const PeerOut* peer = nullptr,
+                     bool after_gateup = false) {
     const int sm = ctx->sm_count;
     const int t128 = ((T + 127) / 128) * ((N + 255) / 256);
     int n_n = (N + 255) / 256, wmax = 256;
@@ -1080,6 +1089,17 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     const int grid = t256 < sm ? t256 : sm;
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
+    if (after_gateup && !sel_counts) {
+        // The kernel before this one in the stream is the gate / up kernel of the same call, which lets its dependents
+        // start as its CTAs leave: this kernel sets itself up and forms its tile masks (from the mask and the token
+        // order, both older than the gate / up kernel) meanwhile, and waits before it loads H or stores anything.
+        // Only then: after any other kernel the early reads could see that kernel's unfinished writes.
+        WIDE_CUDA_CHECK(wide_launch_dependent(down256_kernel, dim3(grid), dim3(192), kSmem2, s, tmA, tmB, mask_bits, order, words, T,
+                                              N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0, n_n, wmax,
+                                              reinterpret_cast<unsigned*>(ctx->d_status) + 8, sel_counts, sel_thr,
+                                              peer ? *peer : PeerOut{}, ctx->d_status, ctx->wait_ns));
+        return WIDE_OK;
+    }
     down256_kernel<<<grid, 192, kSmem2, s>>>(tmA, tmB, mask_bits, order, words, T, N, K, G, Y, out_dtype == WIDE_BF16 ? 1 : 0,
                                              n_n, wmax, reinterpret_cast<unsigned*>(ctx->d_status) + 8, sel_counts, sel_thr,
                                              peer ? *peer : PeerOut{}, ctx->d_status, ctx->wait_ns);
@@ -1145,7 +1165,7 @@ KaxisPlan plan_kaxis(int G, int NG, int out_dtype, bool have_perm, unsigned flag
 int launch_kaxis(wide_ctx* ctx, cudaStream_t s, const KaxisPlan& plan, const void* a_rows, const int32_t* a_row_of_token,
                  const void* a_unmasked, void* a_owner, const void* B, int T, int N, int K, int G,
                  const uint32_t* mask_bits, const int32_t* perm, const int32_t* counts, const int32_t* order,
-                 const int32_t* rank, void* y, int out_dtype, void* acc, const char* group_name) {
+                 const int32_t* rank, void* y, int out_dtype, void* acc, const char* group_name, bool after_gateup = false) {
     const int NG = K / G;
     int rc;
     if (plan.thr_q == WIDE_KAXIS_NEVER) {
@@ -1153,7 +1173,8 @@ int launch_kaxis(wide_ctx* ctx, cudaStream_t s, const KaxisPlan& plan, const voi
             rc = wide_launch_kaxis_prep(ctx, s, nullptr, NG, T, plan.thr_q, nullptr, 0, a_unmasked, mask_bits, rank, K, G, a_owner);
             if (rc != WIDE_OK) return rc;
         }
-        return launch_down_auto(ctx, s, a_owner, B, mask_bits, T, N, K, G, y, out_dtype, order);
+        return launch_down_auto(ctx, s, a_owner, B, mask_bits, T, N, K, G, y, out_dtype, order, nullptr, WIDE_KAXIS_NEVER, nullptr,
+                                after_gateup && !a_unmasked);
     }
     void* target = plan.use_acc ? acc : y;
     const size_t target_bytes = static_cast<size_t>(T) * N * (plan.bf16_red ? 2 : 4);
@@ -1194,7 +1215,7 @@ int wide_launch_ffn_prefill_tc(wide_ctx* ctx, cudaStream_t s, const void* x, con
     if (rc != WIDE_OK) return rc;
     const KaxisPlan plan = plan_kaxis(G, Dff / G, out_dtype, true, flags);
     return launch_kaxis(ctx, s, plan, h, token_rank, nullptr, h, wd, T, D, Dff, G, mask_bits, perm, counts, token_order,
-                        token_rank, y, out_dtype, acc, "prefill_down_group");
+                        token_rank, y, out_dtype, acc, "prefill_down_group", true);
 }
 
 // Group-sharded FFN part with the reduce-scatter fused into the down projection's epilogue (see

@@ -87,6 +87,16 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, un
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns, abort_flag) ? 1 : 0) != 0;
 }
 
+// ------------------------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialization attribute may become resident while the kernel
+// before it in the stream is still running (as soon as every CTA of that kernel has called
+// grid_dep_launch or exited).  Until it has called grid_dep_wait it must not touch global memory: the
+// call returns when the earlier kernel has completed and its writes are visible.  What runs before the
+// call (barrier set-up, tensor-memory allocation) overlaps the earlier kernel's tail.  Both are no-ops
+// in a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------- proxies / fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
