@@ -133,6 +133,7 @@ down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     constexpr int kBBytes = BN * kBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
     extern __shared__ uint8_t smem_raw[];
+    grid_dep_launch();   // as the score GEMM of the router: the selection kernel behind it may be scheduled as CTAs leave
     if (wide_kaxis_group_chosen(sel_counts, K / G, T, sel_thr)) return;   // the per-group kernel runs instead
     SmemLayout L = carve_smem<kBBytes>(smem_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;

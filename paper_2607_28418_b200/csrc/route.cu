@@ -2,6 +2,7 @@
 // top-k reading of Appendix A).  The decision is taken on fp64 sums of exact products so that
 // it does not depend on summation order.
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace {
 
@@ -220,6 +221,7 @@ select_band_kernel(const float* __restrict__ scores, int nsplit, int ld, const _
     __shared__ int s_nb[kSelTokens];
     __shared__ int s_band[kSelTokens][kBandMax];
     __shared__ double s_ex[kSelTokens][kBandMax];
+    wptx::grid_dep_wait();     // the score slabs come from the kernel before (see launch_select_band)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tt = warp >> 1;                       // token slot in the CTA
     const bool select_warp = (warp & 1) == 0;
@@ -424,8 +426,8 @@ template <int KPL>
 void launch_select_band(cudaStream_t s, int T, const float* sc32, int ksplit, int ld, const __nv_bfloat16* x,
                         const __nv_bfloat16* w, const float* wn, int NG, int D, int k, const int32_t* k_per_token,
                         uint32_t* mask_bits, float* scores, int chain) {
-    select_band_kernel<KPL><<<(T + kSelTokens - 1) / kSelTokens, 64 * kSelTokens, 0, s>>>(
-        sc32, ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores, chain);
+    wide_launch_dependent(select_band_kernel<KPL>, dim3((T + kSelTokens - 1) / kSelTokens), dim3(64 * kSelTokens), 0, s, sc32,
+                          ksplit, ld, x, w, wn, T, NG, D, k, k_per_token, mask_bits, scores, chain);
 }
 
 // ---------------------------------------------------------------------------- small batches (decode), top-k
