@@ -637,9 +637,12 @@ down256_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // order.  Two consecutive tiles of the same (group, channel sub-block) form a DOUBLE item: 256
 // gathered rows, two M=128 UMMAs per 16-wide k-slice sharing the weight tile in shared memory
 // (1.5x fewer bytes per FLOP, the ring covers 1.5x more latency).  Doubles are dealt round-robin
-// for as many full rounds as there are; what is left of them is cut back into 128-row SINGLE items
-// and dealt together with the odd last tiles, so that every CTA ends within one single item of the
-// others.  Every CTA derives the same schedule from `counts` alone (prefix sums in shared memory).
+// for as many full rounds as there are.  What is left of them is either cut back into 128-row SINGLE
+// items and dealt together with the odd last tiles, so that every CTA ends within one single item of
+// the others, or (when many doubles are left: a single costs about 0.7 of a double, two of them 1.4)
+// run as one more, partial round of doubles with the odd tiles dealt from the idle CTAs on; whichever
+// ends earlier by that cost model.  Every CTA derives the same schedule from `counts` alone (prefix
+// sums in shared memory).
 // The two accumulators of a double fill TMEM, so an item's epilogue does not overlap the next
 // item's MMAs; it is kept short instead (8 epilogue warps, fast SiLU).
 struct GuItem {
@@ -652,12 +655,18 @@ struct GuSched {
     const int* dbl_off;   // [n_gs + 1] prefix of doubles per (group, sub)
     const int* sgl_off;   // [n_gs + 1] prefix of odd last tiles
     int n_gs, nD, nS, grid, rfull, remD, nS2, pos;
+    bool tail_doubles;    // the doubles left after the full rounds run as doubles
     __device__ GuSched(const int* d, const int* sg, int n) : dbl_off(d), sgl_off(sg), n_gs(n), grid(gridDim.x), pos(0) {
         nD = d[n];
         nS = sg[n];
         rfull = nD / grid;
         remD = nD - rfull * grid;
         nS2 = 2 * remD + nS;
+        // end of the tail in tenths of a double item's time, a single item counted as 7
+        const int cost_cut = 7 * ((nS2 + grid - 1) / grid);
+        const int idle = grid - remD;
+        const int cost_keep = max(7 * ((nS + grid - 1) / grid), 10 + 7 * (nS > idle ? (nS - idle + grid - 1) / grid : 0));
+        tail_doubles = remD > 0 && cost_keep < cost_cut;
     }
     __device__ int find(const int* off, int idx) const {  // largest i with off[i] <= idx
         int lo = 0, hi = n_gs;
@@ -674,6 +683,26 @@ struct GuSched {
             it.gs = find(dbl_off, di);
             it.m = 2 * (di - dbl_off[it.gs]);
             it.rows = 256;
+            ++pos;
+            return true;
+        }
+        if (tail_doubles) {
+            // one partial round of doubles on CTAs 0 .. remD-1, the odd tiles dealt round-robin from CTA remD on
+            const bool has_double = b < remD;
+            if (pos == rfull && has_double) {
+                const int di = rfull * grid + b;
+                it.gs = find(dbl_off, di);
+                it.m = 2 * (di - dbl_off[it.gs]);
+                it.rows = 256;
+                ++pos;
+                return true;
+            }
+            const int q = pos - rfull - (has_double ? 1 : 0);         // singles this CTA has taken
+            const int si = q * grid + (b - remD + grid) % grid;
+            if (si >= nS) return false;
+            it.gs = find(sgl_off, si);
+            it.m = 2 * (dbl_off[it.gs + 1] - dbl_off[it.gs]);            // the odd tile follows the group's doubles
+            it.rows = 128;
             ++pos;
             return true;
         }
@@ -1090,7 +1119,7 @@ int launch_down_auto(wide_ctx* ctx, cudaStream_t s, const void* A, const void* B
     const int grid = t256 < sm ? t256 : sm;
     const int words = (K / G + 31) / 32;
     WideLaunch l(ctx, s, "prefill_down");
-    if (after_gateup && !sel_counts) {
+    if (after_gateup && !sel_counts && !ctx->prof) {   // (per-kernel timing brackets every launch with events: ordinary launches then)
         // The kernel before this one in the stream is the gate / up kernel of the same call, which lets its dependents
         // start as its CTAs leave: this kernel sets itself up and forms its tile masks (from the mask and the token
         // order, both older than the gate / up kernel) meanwhile, and waits before it loads H or stores anything.
